@@ -1,0 +1,201 @@
+"""Python face of the fp64 CPU oracle (ctypes marshalling + the per-step cache semantics).
+
+TEST INFRASTRUCTURE ONLY -- see oracle/__init__.py.  All arithmetic of Eq. 1, Eq. 2,
+Eq. 8 and Eq. 13 lives in ditango_oracle.c; this file only moves numpy arrays in and out
+and keeps the state cache of the selective compute / reuse step (Section 2.2.4, Fig. 6;
+cache timestep t_c of Section 4.2.2; Algorithm 1's t_c bookkeeping).
+
+Q, K, V are numpy uint16 arrays holding bf16 bit patterns in layout [B, L, H, D].
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(_build.build())
+        u16p, i32p, f64p, u8p = (C.POINTER(C.c_uint16), C.POINTER(C.c_int32),
+                                 C.POINTER(C.c_double), C.POINTER(C.c_uint8))
+        L.orc_num_threads.restype = C.c_int
+        L.orc_pair_state.restype = C.c_int
+        L.orc_pair_state.argtypes = [u16p, u16p, u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
+                                     C.c_int, C.c_int, i32p, C.c_int, C.c_int, C.c_int, f64p, f64p]
+        L.orc_full_attention.restype = C.c_int
+        L.orc_full_attention.argtypes = [u16p, u16p, u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
+                                         C.c_int, C.c_int, i32p, C.c_int, f64p, f64p]
+        L.orc_compose2.restype = None
+        L.orc_compose2.argtypes = [f64p, C.c_double, f64p, C.c_double, C.c_int, f64p, f64p]
+        L.orc_merge.restype = None
+        L.orc_merge.argtypes = [f64p, f64p, C.c_int, C.c_int, C.c_int, f64p, f64p]
+        L.orc_contribution.restype = C.c_int
+        L.orc_contribution.argtypes = [f64p, C.c_int, C.c_int, C.c_int, C.c_int, i32p, f64p]
+        L.orc_threshold.restype = None
+        L.orc_threshold.argtypes = [f64p, C.c_int, C.c_double, u8p]
+        L.orc_target_fraction.restype = C.c_int
+        L.orc_target_fraction.argtypes = [f64p, C.c_int, C.c_double, u8p, f64p]
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().orc_num_threads())
+
+
+def _p(a, ct):
+    return a.ctypes.data_as(C.POINTER(ct))
+
+
+def _chk_qkv(q, k, v):
+    for t in (q, k, v):
+        if t.dtype != np.uint16 or t.ndim != 4 or not t.flags.c_contiguous:
+            raise ValueError("q, k, v must be C-contiguous uint16 (bf16 bits) arrays [B, L, H, D]")
+    if not (q.shape == k.shape == v.shape):
+        raise ValueError("q, k, v shapes differ")
+    return q.shape
+
+
+def pair_state(q, k, v, scale, b, h, rows, key_begin, key_end):
+    """Eq. 1 for the listed query rows of (b, h) against keys [key_begin, key_end).
+
+    Returns (OUT [nrows, D], LSE [nrows]) in fp64."""
+    B, L, H, D = _chk_qkv(q, k, v)
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    out = np.empty((rows.size, D), dtype=np.float64)
+    lse = np.empty((rows.size,), dtype=np.float64)
+    rc = lib().orc_pair_state(_p(q, C.c_uint16), _p(k, C.c_uint16), _p(v, C.c_uint16), B, L, H, D,
+                              float(scale), int(b), int(h), _p(rows, C.c_int32), rows.size,
+                              int(key_begin), int(key_end), _p(out, C.c_double), _p(lse, C.c_double))
+    if rc != 0:
+        raise ValueError("orc_pair_state: bad arguments")
+    return out, lse
+
+
+def full_attention(q, k, v, scale, b, h, rows):
+    """softmax(scale * q K^T) V over all L keys for the listed rows of (b, h), fp64."""
+    B, L, H, D = _chk_qkv(q, k, v)
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    out = np.empty((rows.size, D), dtype=np.float64)
+    lse = np.empty((rows.size,), dtype=np.float64)
+    rc = lib().orc_full_attention(_p(q, C.c_uint16), _p(k, C.c_uint16), _p(v, C.c_uint16), B, L, H, D,
+                                  float(scale), int(b), int(h), _p(rows, C.c_int32), rows.size,
+                                  _p(out, C.c_double), _p(lse, C.c_double))
+    if rc != 0:
+        raise ValueError("orc_full_attention: bad arguments")
+    return out, lse
+
+
+def compose2(oa, lsea, ob, lseb):
+    """Eq. 2 for two states of one query row."""
+    oa = np.ascontiguousarray(oa, dtype=np.float64)
+    ob = np.ascontiguousarray(ob, dtype=np.float64)
+    o = np.empty_like(oa)
+    lse = C.c_double()
+    lib().orc_compose2(_p(oa, C.c_double), float(lsea), _p(ob, C.c_double), float(lseb), oa.size,
+                       _p(o, C.c_double), C.byref(lse))
+    return o, lse.value
+
+
+def merge(o_states, lse_states):
+    """Eq. 2 folded over P states per row: o_states [n, P, D], lse_states [n, P]."""
+    o_states = np.ascontiguousarray(o_states, dtype=np.float64)
+    lse_states = np.ascontiguousarray(lse_states, dtype=np.float64)
+    n, P, D = o_states.shape
+    assert lse_states.shape == (n, P)
+    out = np.empty((n, D), dtype=np.float64)
+    lse = np.empty((n,), dtype=np.float64)
+    lib().orc_merge(_p(o_states, C.c_double), _p(lse_states, C.c_double), n, P, D,
+                    _p(out, C.c_double), _p(lse, C.c_double))
+    return out, lse
+
+
+def contribution(lse_states, off):
+    """Eq. 8 per row, averaged to W[i][j]; lse_states [P, B, H, L] fp64, off [P+1]."""
+    lse_states = np.ascontiguousarray(lse_states, dtype=np.float64)
+    P, B, H, L = lse_states.shape
+    off = np.ascontiguousarray(off, dtype=np.int32)
+    assert off.size == P + 1
+    W = np.empty((P, P), dtype=np.float64)
+    rc = lib().orc_contribution(_p(lse_states, C.c_double), B, H, L, P, _p(off, C.c_int32), _p(W, C.c_double))
+    if rc != 0:
+        raise ValueError("orc_contribution: bad partition offsets")
+    return W
+
+
+def threshold(W, eps):
+    """Eq. 13 with the diagonal forced to COMPUTE; returns uint8 [P, P]."""
+    W = np.ascontiguousarray(W, dtype=np.float64)
+    P = W.shape[0]
+    mask = np.empty((P, P), dtype=np.uint8)
+    lib().orc_threshold(_p(W, C.c_double), P, float(eps), _p(mask, C.c_uint8))
+    return mask
+
+
+def target_fraction(W, f):
+    """Percentile choice of eps for a target computed-pair fraction; returns (mask, eps, K)."""
+    W = np.ascontiguousarray(W, dtype=np.float64)
+    P = W.shape[0]
+    mask = np.empty((P, P), dtype=np.uint8)
+    eps = C.c_double()
+    K = lib().orc_target_fraction(_p(W, C.c_double), P, float(f), _p(mask, C.c_uint8), C.byref(eps))
+    return mask, eps.value, int(K)
+
+
+def uniform_offsets(L, P):
+    """off_p = floor(p L / P): contiguous partitions whose sizes differ by at most one."""
+    return np.array([(p * L) // P for p in range(P + 1)], dtype=np.int32)
+
+
+class OracleSession:
+    """Selective compute / reuse over denoising steps for a chosen set of query rows.
+
+    The cache holds, per (query row, KV partition j), the state of the last step at which
+    the pair (partition of the row, j) was computed (t_c); it starts empty (t_c = -1).
+    step(): COMPUTE pairs are recomputed from the step's inputs (Eq. 1) and overwrite
+    their slots; REUSE pairs keep their slots (an empty one is an error); the output is
+    the composition of all P slots (Eq. 2).
+
+    rows_by_bh: dict {(b, h): int array of query rows}; only these rows are evaluated,
+    which is what lets large workloads be checked on a sample.
+    """
+
+    def __init__(self, B, L, H, D, off, scale, rows_by_bh):
+        self.B, self.L, self.H, self.D = B, L, H, D
+        self.off = np.ascontiguousarray(off, dtype=np.int32)
+        self.P = self.off.size - 1
+        self.scale = float(scale)
+        self.rows = {bh: np.ascontiguousarray(r, dtype=np.int32) for bh, r in rows_by_bh.items()}
+        self.part = {bh: np.searchsorted(self.off, r, side="right") - 1 for bh, r in self.rows.items()}
+        self.o = {bh: np.zeros((r.size, self.P, D)) for bh, r in self.rows.items()}
+        self.lse = {bh: np.zeros((r.size, self.P)) for bh, r in self.rows.items()}
+        self.tc = -np.ones((self.P, self.P), dtype=np.int32)
+
+    def step(self, q, k, v, mask, t):
+        mask = np.asarray(mask).reshape(self.P, self.P)
+        for i in range(self.P):
+            for j in range(self.P):
+                if not mask[i, j] and self.tc[i, j] < 0:
+                    raise RuntimeError(f"REUSE of pair ({i},{j}) that was never computed")
+        outs, lses = {}, {}
+        for bh, rows in self.rows.items():
+            b, h = bh
+            for i in range(self.P):
+                sel = np.nonzero(self.part[bh] == i)[0]
+                if sel.size == 0:
+                    continue
+                for j in range(self.P):
+                    if mask[i, j]:
+                        o, l = pair_state(q, k, v, self.scale, b, h, rows[sel],
+                                          int(self.off[j]), int(self.off[j + 1]))
+                        self.o[bh][sel, j, :] = o
+                        self.lse[bh][sel, j] = l
+            outs[bh], lses[bh] = merge(self.o[bh], self.lse[bh])
+        self.tc[mask.astype(bool)] = t
+        return outs, lses
