@@ -1,0 +1,141 @@
+/*
+ * libditango -- selective attention-state path of DiTango on one B200 (sm_100a).
+ *
+ * The token sequence of one attention layer (L tokens) is split into P contiguous
+ * partitions.  For a (query partition i, KV partition j) pair, the attention state is the
+ * partition-normalised output OUT_ij and the log-sum-exp LSE_ij of Eq. 1 (Section 2.2.4).
+ * Per denoising step a plan marks each pair COMPUTE or REUSE (Eq. 11, Eq. 13): COMPUTE pairs
+ * are evaluated from the step's Q, K, V and overwrite their slot of the state cache, REUSE
+ * pairs keep the state of the last step that computed them (t_c, Section 4.2.2), and all P
+ * states of a query row are composed by LSE rescaling (Eq. 2) into the attention output.
+ * The plan comes from the cached LSEs: partition importance weights (Eq. 8), averaged per
+ * pair, thresholded with a strict '>' (Eq. 13); the local (diagonal) pair is always computed
+ * (Section 4.1.2).
+ *
+ * Conventions
+ *   - Plain C ABI.  "device" pointers are CUDA device memory of the context's device,
+ *     "host" pointers are ordinary host memory.  The library never frees or keeps caller
+ *     buffers, except the two cache pointers given to dt_bind_cache.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  dt_attn_states,
+ *     dt_state_merge and dt_plan only enqueue work on it; they do not synchronise.
+ *   - Every function returns a dt_status.  Argument errors are detected before any launch.
+ *     Conditions only the device can see (REUSE of a never-computed pair, a bounded wait
+ *     that ran out) are recorded in a device status word that dt_poll reads.
+ *   - Natural logarithm everywhere an LSE crosses this boundary.
+ *   - Limits: D in {64, 128}; 1 <= P <= 32; bf16 inputs; innermost stride 1.
+ *
+ * Memory layout of the state cache (caller-owned device memory, sized by dt_cache_bytes):
+ *   o_state   [P (KV partition j)][B][H][L][D]   fp32 or bf16 (dt_config.state_dtype)
+ *   lse_state [P (KV partition j)][B][H][L]      fp32
+ * Row l of slot j belongs to pair (i, j) with i the partition that contains l.
+ */
+#ifndef DITANGO_H_
+#define DITANGO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dt_ctx dt_ctx; /* opaque; owns only small device scratch (work list, t_c, partial sums) */
+
+typedef enum {
+    DT_OK = 0,
+    DT_ERR_INVALID_ARG = 1, /* null pointer, bad shape / stride / offsets / alignment           */
+    DT_ERR_UNSUPPORTED = 2, /* D not in {64,128}, P > 32, unknown state dtype, device not sm_100 */
+    DT_ERR_STATE = 3,       /* cache not bound or too small; REUSE of a pair never computed       */
+    DT_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (text in dt_last_error)        */
+    DT_ERR_TIMEOUT = 5      /* a bounded device-side wait expired; the kernel returned normally   */
+} dt_status;
+
+enum { DT_STATE_FP32 = 0, DT_STATE_BF16 = 1 };
+enum { DT_MAX_P = 32 };
+
+typedef struct {
+    int32_t B, H, D, L, P;       /* batch, heads, head dim, tokens, partitions                      */
+    const int32_t *part_offsets; /* host, P+1 ints, off[0]=0 < off[1] < ... < off[P]=L; copied      */
+    float softmax_scale;         /* s in exp(s * q.k); the paper's Eq. 1 leaves it implicit          */
+    int32_t state_dtype;         /* DT_STATE_FP32 or DT_STATE_BF16: storage type of cached OUT_ij    */
+    int32_t device;              /* CUDA device ordinal                                              */
+} dt_config;
+
+/* Create / destroy a context.  dt_create makes `device` current, checks it is sm_100, copies the
+ * offsets and allocates the context's small device scratch.  All t_c start at -1 (empty). */
+dt_status dt_create(dt_ctx **ctx_out, const dt_config *cfg);
+dt_status dt_destroy(dt_ctx *ctx);
+
+/* Closed-form size of the state cache: o_bytes = P*B*H*L*D*sizeof(state), lse_bytes = P*B*H*L*4.
+ * Per pair this is OUT (n_i*H*D) + LSE (n_i*H) against 2*n_j*H*D for the KV it replaces
+ * ("half of KV size", Section 2.2.4). */
+dt_status dt_cache_bytes(const dt_config *cfg, size_t *o_bytes, size_t *lse_bytes);
+
+/* Bind caller-owned device memory as the state cache (16-byte aligned, at least the sizes above).
+ * Contents are not touched; binding does not reset t_c. */
+dt_status dt_bind_cache(dt_ctx *ctx, void *o_state_dev, float *lse_state_dev, size_t o_bytes, size_t lse_bytes);
+
+/* Eq. 1 for every COMPUTE pair, every head and every query row; REUSE pairs cost nothing and
+ * their cache slots are not touched (Section 2.2.4, Fig. 6; Section 5.2 steps evict/compute/store).
+ *   q, k, v        device, bf16, logical shape [B, L, H, D]; strides_blhd in elements
+ *                  (stride of D must be 1, the others multiples of 8; bases 16-byte aligned)
+ *   mask_dev       device, uint8 [P*P] row-major (i = query partition, j = KV partition),
+ *                  non-zero = COMPUTE.  Read on the device: no host copy, no synchronisation.
+ *   step           denoising step index (>= 0), recorded as t_c of every COMPUTE pair
+ * A REUSE pair with t_c = -1 sets the device status to DT_ERR_STATE (see dt_poll); the COMPUTE
+ * pairs are still evaluated. */
+dt_status dt_attn_states(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
+                         const int64_t strides_blhd[4], const uint8_t *mask_dev, int32_t step, void *stream);
+
+/* Eq. 2 folded over all P cached states of each query row (fresh or reused alike):
+ *   LSE[r] = log sum_j exp(LSE_ij[r]),  OUT[r] = sum_j exp(LSE_ij[r] - LSE[r]) OUT_ij[r].
+ *   out_dev        device, bf16, logical [B, L, H, D] with out_strides_blhd (elements; D stride 1,
+ *                  others multiples of 8, base 16-byte aligned)
+ *   lse_out_dev    device, fp32 [B, H, L], or NULL */
+dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev,
+                         void *stream);
+
+/* Plan from the cached LSEs (call after a step that computed every pair -- an anchor step):
+ *   per row  w_j = exp(LSE_ij - logsumexp_k LSE_ik)                  (Eq. 8)
+ *   W[i][j]  = mean of w_j over batch, heads and the rows of partition i
+ *   target_fraction < 0 : mask[i][j] = (i == j) or (W[i][j] > eps)    (Eq. 13, strict)
+ *   target_fraction >= 0: K = round(f P^2) clipped to [P, P^2]; the diagonal plus the K - P
+ *                         off-diagonal pairs of largest W are COMPUTE (ties: smaller |i-j|, then
+ *                         smaller i*P+j); eps_out = midpoint between the last selected and the
+ *                         first unselected W (0 if all are selected; the largest off-diagonal W
+ *                         if none is)
+ *   mask_dev       device, uint8 [P*P], written
+ *   w_dev          device, double [P*P], written; or NULL
+ *   eps_out_dev    device, double [1], written (eps used or derived); or NULL */
+dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask_dev, double *w_dev,
+                  double *eps_out_dev, void *stream);
+
+/* One whole step from HOST buffers: copies q, k, v (bf16 [B,L,H,D] contiguous) and the mask to the
+ * device workspace, runs dt_attn_states and dt_state_merge, copies out (bf16 [B,L,H,D]) and lse
+ * (fp32 [B,H,L], may be NULL) back and synchronises `stream`.  workspace_dev must hold
+ * dt_step_host_workspace_bytes() bytes of device memory.  Host buffers should be pinned for
+ * full copy bandwidth. */
+dt_status dt_step_host_workspace_bytes(const dt_config *cfg, size_t *bytes);
+dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, const void *v_host,
+                       const uint8_t *mask_host, int32_t step, void *out_host, float *lse_out_host,
+                       void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/* Cache timesteps t_c[i][j] (-1 = empty), host int32 [P*P].  Both synchronise the device.
+ * Together with the cache contents they are everything needed to snapshot and resume. */
+dt_status dt_get_tc(dt_ctx *ctx, int32_t *tc_host);
+dt_status dt_set_tc(dt_ctx *ctx, const int32_t *tc_host);
+
+/* Number of kernels this library has launched through `ctx` since creation. */
+dt_status dt_launch_count(dt_ctx *ctx, uint64_t *count);
+
+/* Read (and clear) the device status word; synchronises the device.  Returns DT_OK,
+ * DT_ERR_STATE or DT_ERR_TIMEOUT. */
+dt_status dt_poll(dt_ctx *ctx);
+
+const char *dt_status_str(dt_status s);
+const char *dt_last_error(dt_ctx *ctx); /* text of the last error on this context ("" if none) */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DITANGO_H_ */

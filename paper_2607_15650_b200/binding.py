@@ -1,0 +1,207 @@
+"""ctypes binding of libditango's C ABI: same names, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  torch is used for device memory
+and streams.  If the shared library is missing this module raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libditango.so")
+
+DT_OK, DT_ERR_INVALID_ARG, DT_ERR_UNSUPPORTED, DT_ERR_STATE, DT_ERR_CUDA, DT_ERR_TIMEOUT = range(6)
+DT_STATE_FP32, DT_STATE_BF16 = 0, 1
+DT_MAX_P = 32
+
+EXPORTS = [
+    "dt_create", "dt_destroy", "dt_cache_bytes", "dt_bind_cache", "dt_attn_states", "dt_state_merge",
+    "dt_plan", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
+    "dt_launch_count", "dt_poll", "dt_status_str", "dt_last_error",
+]
+
+
+class dt_config(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("L", C.c_int32), ("P", C.c_int32),
+                ("part_offsets", C.POINTER(C.c_int32)), ("softmax_scale", C.c_float),
+                ("state_dtype", C.c_int32), ("device", C.c_int32)]
+
+
+class DitangoError(RuntimeError):
+    def __init__(self, status, name, detail=""):
+        self.status = status
+        super().__init__(f"{name}" + (f": {detail}" if detail else ""))
+
+
+_lib = None
+
+
+def lib():
+    """Load libditango.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2607_15650_b200.build` "
+                          "(there is no CPU or PyTorch fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i64p, u8p, f32p, f64p, i32p = (C.c_void_p, C.POINTER(C.c_int64), C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.POINTER(C.c_int32))
+    szp = C.POINTER(C.c_size_t)
+    sig = {
+        "dt_create": (C.c_int, [C.POINTER(vp), C.POINTER(dt_config)]),
+        "dt_destroy": (C.c_int, [vp]),
+        "dt_cache_bytes": (C.c_int, [C.POINTER(dt_config), szp, szp]),
+        "dt_bind_cache": (C.c_int, [vp, vp, f32p, C.c_size_t, C.c_size_t]),
+        "dt_attn_states": (C.c_int, [vp, vp, vp, vp, i64p, u8p, C.c_int32, vp]),
+        "dt_state_merge": (C.c_int, [vp, vp, i64p, f32p, vp]),
+        "dt_plan": (C.c_int, [vp, C.c_double, C.c_double, u8p, f64p, f64p, vp]),
+        "dt_step_host_workspace_bytes": (C.c_int, [C.POINTER(dt_config), szp]),
+        "dt_step_host": (C.c_int, [vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, C.c_size_t, vp]),
+        "dt_get_tc": (C.c_int, [vp, i32p]),
+        "dt_set_tc": (C.c_int, [vp, i32p]),
+        "dt_launch_count": (C.c_int, [vp, C.POINTER(C.c_uint64)]),
+        "dt_poll": (C.c_int, [vp]),
+        "dt_status_str": (C.c_char_p, [C.c_int]),
+        "dt_last_error": (C.c_char_p, [vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(L, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = L
+    return L
+
+
+def make_config(B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0):
+    off = np.ascontiguousarray(offsets, dtype=np.int32)
+    cfg = dt_config(B, H, D, L, off.size - 1, off.ctypes.data_as(C.POINTER(C.c_int32)), float(softmax_scale),
+                    int(state_dtype), int(device))
+    cfg._keepalive = off
+    return cfg
+
+
+def status_str(s: int) -> str:
+    return lib().dt_status_str(int(s)).decode()
+
+
+def dt_cache_bytes(cfg):
+    o, l = C.c_size_t(), C.c_size_t()
+    s = lib().dt_cache_bytes(C.byref(cfg), C.byref(o), C.byref(l))
+    if s != DT_OK:
+        raise DitangoError(s, status_str(s))
+    return o.value, l.value
+
+
+def dt_step_host_workspace_bytes(cfg):
+    n = C.c_size_t()
+    s = lib().dt_step_host_workspace_bytes(C.byref(cfg), C.byref(n))
+    if s != DT_OK:
+        raise DitangoError(s, status_str(s))
+    return n.value
+
+
+def _strides4(t: torch.Tensor):
+    return (C.c_int64 * 4)(*[int(x) for x in t.stride()])
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+class Context:
+    """Owns a dt_ctx and (optionally) the state-cache tensors bound to it."""
+
+    def __init__(self, B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0, alloc_cache=True):
+        self._h = C.c_void_p()
+        self.cfg = make_config(B, H, D, L, offsets, softmax_scale, state_dtype, device)
+        self.device = torch.device("cuda", device)
+        s = lib().dt_create(C.byref(self._h), C.byref(self.cfg))
+        if s != DT_OK:
+            self._h = C.c_void_p()
+            raise DitangoError(s, status_str(s), "dt_create")
+        self.o_state = self.lse_state = None
+        if alloc_cache:
+            P = self.cfg.P
+            sdt = torch.float32 if state_dtype == DT_STATE_FP32 else torch.bfloat16
+            o = torch.empty((P, B, H, L, D), dtype=sdt, device=self.device)
+            l = torch.empty((P, B, H, L), dtype=torch.float32, device=self.device)
+            self.dt_bind_cache(o, l)
+
+    def _check(self, s):
+        if s != DT_OK:
+            raise DitangoError(s, status_str(s), lib().dt_last_error(self._h).decode())
+
+    def dt_bind_cache(self, o_state: torch.Tensor, lse_state: torch.Tensor):
+        assert o_state.is_cuda and lse_state.is_cuda and o_state.is_contiguous() and lse_state.is_contiguous()
+        self._check(lib().dt_bind_cache(self._h, C.c_void_p(o_state.data_ptr()), C.c_void_p(lse_state.data_ptr()),
+                                        o_state.numel() * o_state.element_size(), lse_state.numel() * 4))
+        self.o_state, self.lse_state = o_state, lse_state
+
+    def dt_attn_states(self, q, k, v, mask_dev, step, stream=None):
+        assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and q.is_cuda
+        assert q.stride() == k.stride() == v.stride() and q.shape == k.shape == v.shape
+        assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()
+        self._check(lib().dt_attn_states(self._h, C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()),
+                                         C.c_void_p(v.data_ptr()), _strides4(q), C.c_void_p(mask_dev.data_ptr()),
+                                         int(step), _stream_ptr(stream)))
+
+    def dt_state_merge(self, out, lse_out=None, stream=None):
+        assert out.dtype == torch.bfloat16 and out.is_cuda
+        lp = C.c_void_p(lse_out.data_ptr()) if lse_out is not None else C.c_void_p()
+        if lse_out is not None:
+            assert lse_out.dtype == torch.float32 and lse_out.is_contiguous()
+        self._check(lib().dt_state_merge(self._h, C.c_void_p(out.data_ptr()), _strides4(out), lp, _stream_ptr(stream)))
+
+    def dt_plan(self, mask_dev, eps=0.0, target_fraction=-1.0, w_dev=None, eps_out_dev=None, stream=None):
+        assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()
+        wp = C.c_void_p(w_dev.data_ptr()) if w_dev is not None else C.c_void_p()
+        ep = C.c_void_p(eps_out_dev.data_ptr()) if eps_out_dev is not None else C.c_void_p()
+        if w_dev is not None:
+            assert w_dev.dtype == torch.float64 and w_dev.is_contiguous()
+        if eps_out_dev is not None:
+            assert eps_out_dev.dtype == torch.float64
+        self._check(lib().dt_plan(self._h, float(eps), float(target_fraction), C.c_void_p(mask_dev.data_ptr()), wp, ep,
+                                  _stream_ptr(stream)))
+
+    def dt_step_host(self, q_host, k_host, v_host, mask_host, step, out_host, lse_out_host, workspace, stream=None):
+        lp = C.c_void_p(lse_out_host.data_ptr()) if lse_out_host is not None else C.c_void_p()
+        self._check(lib().dt_step_host(self._h, C.c_void_p(q_host.data_ptr()), C.c_void_p(k_host.data_ptr()),
+                                       C.c_void_p(v_host.data_ptr()), C.c_void_p(mask_host.data_ptr()), int(step),
+                                       C.c_void_p(out_host.data_ptr()), lp, C.c_void_p(workspace.data_ptr()),
+                                       workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
+
+    def dt_get_tc(self):
+        P = self.cfg.P
+        tc = np.empty((P, P), dtype=np.int32)
+        self._check(lib().dt_get_tc(self._h, tc.ctypes.data_as(C.POINTER(C.c_int32))))
+        return tc
+
+    def dt_set_tc(self, tc):
+        tc = np.ascontiguousarray(tc, dtype=np.int32)
+        self._check(lib().dt_set_tc(self._h, tc.ctypes.data_as(C.POINTER(C.c_int32))))
+
+    def dt_launch_count(self) -> int:
+        n = C.c_uint64()
+        self._check(lib().dt_launch_count(self._h, C.byref(n)))
+        return int(n.value)
+
+    def dt_poll(self):
+        """Raises DitangoError if the device recorded a condition; returns None otherwise."""
+        self._check(lib().dt_poll(self._h))
+
+    def close(self):
+        if self._h:
+            lib().dt_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

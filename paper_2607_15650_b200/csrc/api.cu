@@ -1,0 +1,348 @@
+// C-ABI of libditango: argument checking, tensor-map encoding, launches.  No arithmetic of the
+// method lives here.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "dt_internal.h"
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+dt_status fail(dt_ctx *ctx, dt_status s, const char *what) {
+    if (ctx) ctx->err = what ? what : "";
+    return s;
+}
+
+dt_status fail_cuda(dt_ctx *ctx, cudaError_t e, const char *where) {
+    if (ctx) ctx->err = std::string(where) + ": " + cudaGetErrorString(e);
+    return DT_ERR_CUDA;
+}
+
+dt_status check_config(const dt_config *c, const char **why) {
+    *why = "";
+    if (!c || !c->part_offsets) { *why = "null config or part_offsets"; return DT_ERR_INVALID_ARG; }
+    if (c->B < 1 || c->H < 1 || c->L < 1 || c->P < 1) { *why = "B, H, L, P must be positive"; return DT_ERR_INVALID_ARG; }
+    if (c->D != 64 && c->D != 128) { *why = "head dim must be 64 or 128"; return DT_ERR_UNSUPPORTED; }
+    if (c->P > DT_MAX_P) { *why = "more than 32 partitions"; return DT_ERR_UNSUPPORTED; }
+    if (c->state_dtype != DT_STATE_FP32 && c->state_dtype != DT_STATE_BF16) { *why = "unknown state dtype"; return DT_ERR_UNSUPPORTED; }
+    if (!(c->softmax_scale > 0.f) || !std::isfinite(c->softmax_scale)) { *why = "softmax_scale must be finite and > 0"; return DT_ERR_INVALID_ARG; }
+    if (c->part_offsets[0] != 0 || c->part_offsets[c->P] != c->L) { *why = "offsets must start at 0 and end at L"; return DT_ERR_INVALID_ARG; }
+    for (int i = 0; i < c->P; ++i)
+        if (c->part_offsets[i + 1] <= c->part_offsets[i]) { *why = "offsets must be strictly increasing"; return DT_ERR_INVALID_ARG; }
+    if ((long long)c->B * c->H > 65535) { *why = "B*H exceeds 65535"; return DT_ERR_UNSUPPORTED; }
+    return DT_OK;
+}
+
+size_t state_elem_bytes(int dtype) { return dtype == DT_STATE_FP32 ? 4 : 2; }
+
+dt_status check_strides(const int64_t s[4], const void *base, const char **why) {
+    if (!s) { *why = "null strides"; return DT_ERR_INVALID_ARG; }
+    if (s[3] != 1) { *why = "stride of D must be 1"; return DT_ERR_INVALID_ARG; }
+    for (int d = 0; d < 3; ++d)
+        if (s[d] <= 0 || (s[d] % 8) != 0) { *why = "strides of B, L, H must be positive multiples of 8 elements"; return DT_ERR_INVALID_ARG; }
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0) { *why = "tensor base must be 16-byte aligned"; return DT_ERR_INVALID_ARG; }
+    return DT_OK;
+}
+
+// bf16 [B, L, H, D] viewed as a 4-D tensor map (d, h, l, b); box = 64 elements x 1 head x 128 tokens,
+// 128-byte swizzle, out-of-range rows read as zero.
+dt_status encode_qkv_map(dt_ctx *ctx, CUtensorMap *tm, const void *base, const int64_t s[4]) {
+    const dt_config &c = ctx->cfg;
+    cuuint64_t dims[4] = {(cuuint64_t)c.D, (cuuint64_t)c.H, (cuuint64_t)c.L, (cuuint64_t)c.B};
+    cuuint64_t strides[3] = {(cuuint64_t)s[2] * 2, (cuuint64_t)s[1] * 2, (cuuint64_t)s[0] * 2};
+    cuuint32_t box[4] = {64, 1, (cuuint32_t)dt::ATTN_TILE, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+        tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char buf[96];
+        snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        ctx->err = buf;
+        return DT_ERR_CUDA;
+    }
+    return DT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *dt_status_str(dt_status s) {
+    switch (s) {
+        case DT_OK: return "DT_OK";
+        case DT_ERR_INVALID_ARG: return "DT_ERR_INVALID_ARG";
+        case DT_ERR_UNSUPPORTED: return "DT_ERR_UNSUPPORTED";
+        case DT_ERR_STATE: return "DT_ERR_STATE";
+        case DT_ERR_CUDA: return "DT_ERR_CUDA";
+        case DT_ERR_TIMEOUT: return "DT_ERR_TIMEOUT";
+    }
+    return "DT_ERR_UNKNOWN";
+}
+
+const char *dt_last_error(dt_ctx *ctx) { return ctx ? ctx->err.c_str() : ""; }
+
+dt_status dt_cache_bytes(const dt_config *cfg, size_t *o_bytes, size_t *lse_bytes) {
+    const char *why;
+    dt_status s = check_config(cfg, &why);
+    if (s != DT_OK) return s;
+    if (!o_bytes || !lse_bytes) return DT_ERR_INVALID_ARG;
+    const size_t rows = (size_t)cfg->P * cfg->B * cfg->H * cfg->L;
+    *o_bytes = rows * cfg->D * state_elem_bytes(cfg->state_dtype);
+    *lse_bytes = rows * 4;
+    return DT_OK;
+}
+
+dt_status dt_create(dt_ctx **ctx_out, const dt_config *cfg) {
+    if (!ctx_out) return DT_ERR_INVALID_ARG;
+    *ctx_out = nullptr;
+    const char *why;
+    dt_status s = check_config(cfg, &why);
+    if (s != DT_OK) return s;
+    cudaError_t e = cudaSetDevice(cfg->device);
+    if (e != cudaSuccess) return DT_ERR_CUDA;
+    cudaDeviceProp prop;
+    if ((e = cudaGetDeviceProperties(&prop, cfg->device)) != cudaSuccess) return DT_ERR_CUDA;
+    if (prop.major != 10) return DT_ERR_UNSUPPORTED;  // the kernels are built for sm_100a only
+
+    dt_ctx *ctx = new (std::nothrow) dt_ctx();
+    if (!ctx) return DT_ERR_CUDA;
+    ctx->cfg = *cfg;
+    ctx->off.assign(cfg->part_offsets, cfg->part_offsets + cfg->P + 1);
+    ctx->cfg.part_offsets = ctx->off.data();
+    ctx->num_sms = prop.multiProcessorCount;
+    for (int i = 0; i < cfg->P; ++i) ctx->n_max = std::max(ctx->n_max, ctx->off[i + 1] - ctx->off[i]);
+    const int qblock = dt::ATTN_NQ * dt::ATTN_TILE;
+    ctx->qblocks_max = (ctx->n_max + qblock - 1) / qblock;
+    ctx->plan_chunks = (ctx->n_max + dt::PLAN_CHUNK_ROWS - 1) / dt::PLAN_CHUNK_ROWS;
+
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !ctx->encode_tiled) {
+        delete ctx;
+        return DT_ERR_CUDA;
+    }
+    const int P = cfg->P, BH = cfg->B * cfg->H;
+    bool ok = true;
+    ok = ok && cudaMalloc(&ctx->off_dev, (P + 1) * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->tc_dev, P * P * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->worklist_dev, (1 + P * P) * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->status_dev, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->plan_partials_dev, (size_t)BH * P * ctx->plan_chunks * P * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMemcpy(ctx->off_dev, ctx->off.data(), (P + 1) * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemset(ctx->tc_dev, 0xFF, P * P * sizeof(int32_t)) == cudaSuccess;  // -1 = empty
+    ok = ok && cudaMemset(ctx->worklist_dev, 0, (1 + P * P) * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(ctx->status_dev, 0, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && dt::attn_states_configure() == cudaSuccess;
+    if (!ok) {
+        dt_destroy(ctx);
+        return DT_ERR_CUDA;
+    }
+    *ctx_out = ctx;
+    return DT_OK;
+}
+
+dt_status dt_destroy(dt_ctx *ctx) {
+    if (!ctx) return DT_OK;
+    cudaSetDevice(ctx->cfg.device);
+    cudaFree(ctx->off_dev);
+    cudaFree(ctx->tc_dev);
+    cudaFree(ctx->worklist_dev);
+    cudaFree(ctx->status_dev);
+    cudaFree(ctx->plan_partials_dev);
+    delete ctx;
+    return DT_OK;
+}
+
+dt_status dt_bind_cache(dt_ctx *ctx, void *o_state_dev, float *lse_state_dev, size_t o_bytes, size_t lse_bytes) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!o_state_dev || !lse_state_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null cache pointer");
+    if ((reinterpret_cast<uintptr_t>(o_state_dev) & 15u) || (reinterpret_cast<uintptr_t>(lse_state_dev) & 15u))
+        return fail(ctx, DT_ERR_INVALID_ARG, "cache pointers must be 16-byte aligned");
+    size_t need_o, need_l;
+    dt_cache_bytes(&ctx->cfg, &need_o, &need_l);
+    if (o_bytes < need_o || lse_bytes < need_l) return fail(ctx, DT_ERR_STATE, "cache buffers smaller than dt_cache_bytes");
+    ctx->o_state = o_state_dev;
+    ctx->lse_state = lse_state_dev;
+    return DT_OK;
+}
+
+dt_status dt_attn_states(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
+                         const int64_t strides_blhd[4], const uint8_t *mask_dev, int32_t step, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!q_dev || !k_dev || !v_dev || !mask_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null tensor pointer");
+    if (step < 0) return fail(ctx, DT_ERR_INVALID_ARG, "step must be >= 0");
+    if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
+    const char *why;
+    for (const void *t : {q_dev, k_dev, v_dev}) {
+        dt_status s = check_strides(strides_blhd, t, &why);
+        if (s != DT_OK) return fail(ctx, s, why);
+    }
+    CUtensorMap tq, tk, tv;
+    dt_status s;
+    if ((s = encode_qkv_map(ctx, &tq, q_dev, strides_blhd)) != DT_OK) return s;
+    if ((s = encode_qkv_map(ctx, &tk, k_dev, strides_blhd)) != DT_OK) return s;
+    if ((s = encode_qkv_map(ctx, &tv, v_dev, strides_blhd)) != DT_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dt_config &c = ctx->cfg;
+    cudaError_t e = dt::launch_worklist(mask_dev, ctx->tc_dev, ctx->worklist_dev, ctx->status_dev, c.P, step, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "work-list launch");
+    dt::AttnParams p;
+    p.off = ctx->off_dev;
+    p.worklist = ctx->worklist_dev;
+    p.status = ctx->status_dev;
+    p.o_state = ctx->o_state;
+    p.lse_state = ctx->lse_state;
+    p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P;
+    p.qblocks_max = ctx->qblocks_max;
+    p.scale_log2 = c.softmax_scale * 1.44269504088896340736f;
+    e = dt::launch_attn_states(tq, tk, tv, p, c.D, c.state_dtype, ctx->num_sms, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "attention launch");
+    ctx->launches += 2;
+    return DT_OK;
+}
+
+dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev,
+                         void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!out_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null output pointer");
+    if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
+    const char *why;
+    dt_status s = check_strides(out_strides_blhd, out_dev, &why);
+    if (s != DT_OK) return fail(ctx, s, why);
+    const dt_config &c = ctx->cfg;
+    dt::MergeParams p;
+    p.o_state = ctx->o_state;
+    p.lse_state = ctx->lse_state;
+    p.out = out_dev;
+    p.lse_out = lse_out_dev;
+    p.P = c.P; p.H = c.H; p.L = c.L;
+    p.R = (long long)c.B * c.H * c.L;
+    p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
+    cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "merge launch");
+    ctx->launches += 1;
+    return DT_OK;
+}
+
+dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask_dev, double *w_dev,
+                  double *eps_out_dev, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!mask_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null mask pointer");
+    if (!ctx->lse_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
+    if (target_fraction < 0 && !std::isfinite(eps)) return fail(ctx, DT_ERR_INVALID_ARG, "eps must be finite");
+    if (target_fraction > 1.0 || std::isnan(target_fraction)) return fail(ctx, DT_ERR_INVALID_ARG, "target_fraction must be <= 1");
+    const dt_config &c = ctx->cfg;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    dt::PlanParams pp;
+    pp.lse_state = ctx->lse_state;
+    pp.off = ctx->off_dev;
+    pp.partials = ctx->plan_partials_dev;
+    pp.P = c.P; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
+    pp.R = (long long)c.B * c.H * c.L;
+    cudaError_t e = dt::launch_plan_partial(pp, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
+    dt::PlanFinalParams pf;
+    pf.partials = ctx->plan_partials_dev;
+    pf.off = ctx->off_dev;
+    pf.P = c.P; pf.BH = pp.BH; pf.chunks = pp.chunks;
+    pf.mode_target = target_fraction >= 0 ? 1 : 0;
+    const int total = c.P * c.P;
+    int K = (int)std::floor(target_fraction * total + 0.5);
+    K = std::min(std::max(K, c.P), total);
+    pf.K = K;
+    pf.eps = eps;
+    pf.mask = mask_dev;
+    pf.w_out = w_dev;
+    pf.eps_out = eps_out_dev;
+    e = dt::launch_plan_final(pf, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "plan finalise launch");
+    ctx->launches += 2;
+    return DT_OK;
+}
+
+dt_status dt_step_host_workspace_bytes(const dt_config *cfg, size_t *bytes) {
+    const char *why;
+    dt_status s = check_config(cfg, &why);
+    if (s != DT_OK) return s;
+    if (!bytes) return DT_ERR_INVALID_ARG;
+    const size_t elems = (size_t)cfg->B * cfg->L * cfg->H * cfg->D;
+    const size_t lse = (((size_t)cfg->B * cfg->H * cfg->L * 4) + 255) & ~(size_t)255;
+    *bytes = 4 * ((elems * 2 + 255) & ~(size_t)255) + lse + 1024 /* mask */;
+    return DT_OK;
+}
+
+dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, const void *v_host,
+                       const uint8_t *mask_host, int32_t step, void *out_host, float *lse_out_host,
+                       void *workspace_dev, size_t workspace_bytes, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!q_host || !k_host || !v_host || !mask_host || !out_host || !workspace_dev)
+        return fail(ctx, DT_ERR_INVALID_ARG, "null pointer");
+    size_t need;
+    dt_step_host_workspace_bytes(&ctx->cfg, &need);
+    if (workspace_bytes < need) return fail(ctx, DT_ERR_INVALID_ARG, "workspace smaller than dt_step_host_workspace_bytes");
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) return fail(ctx, DT_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    const dt_config &c = ctx->cfg;
+    const size_t elems = (size_t)c.B * c.L * c.H * c.D;
+    const size_t tb = (elems * 2 + 255) & ~(size_t)255;
+    const size_t lse_b = (size_t)c.B * c.H * c.L * 4;
+    uint8_t *w = static_cast<uint8_t *>(workspace_dev);
+    void *qd = w, *kd = w + tb, *vd = w + 2 * tb, *od = w + 3 * tb;
+    float *ld = reinterpret_cast<float *>(w + 4 * tb);
+    uint8_t *md = w + 4 * tb + ((lse_b + 255) & ~(size_t)255);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(qd, q_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy q");
+    if ((e = cudaMemcpyAsync(kd, k_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy k");
+    if ((e = cudaMemcpyAsync(vd, v_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy v");
+    if ((e = cudaMemcpyAsync(md, mask_host, (size_t)c.P * c.P, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy mask");
+    const int64_t strides[4] = {(int64_t)c.L * c.H * c.D, (int64_t)c.H * c.D, c.D, 1};
+    dt_status s;
+    if ((s = dt_attn_states(ctx, qd, kd, vd, strides, md, step, stream)) != DT_OK) return s;
+    if ((s = dt_state_merge(ctx, od, strides, ld, stream)) != DT_OK) return s;
+    if ((e = cudaMemcpyAsync(out_host, od, elems * 2, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy out");
+    if (lse_out_host && (e = cudaMemcpyAsync(lse_out_host, ld, lse_b, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return fail_cuda(ctx, e, "copy lse");
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(ctx, e, "synchronise");
+    return DT_OK;
+}
+
+dt_status dt_get_tc(dt_ctx *ctx, int32_t *tc_host) {
+    if (!ctx || !tc_host) return DT_ERR_INVALID_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(tc_host, ctx->tc_dev, ctx->cfg.P * ctx->cfg.P * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    return e == cudaSuccess ? DT_OK : fail_cuda(ctx, e, "dt_get_tc");
+}
+
+dt_status dt_set_tc(dt_ctx *ctx, const int32_t *tc_host) {
+    if (!ctx || !tc_host) return DT_ERR_INVALID_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->tc_dev, tc_host, ctx->cfg.P * ctx->cfg.P * sizeof(int32_t), cudaMemcpyHostToDevice);
+    return e == cudaSuccess ? DT_OK : fail_cuda(ctx, e, "dt_set_tc");
+}
+
+dt_status dt_launch_count(dt_ctx *ctx, uint64_t *count) {
+    if (!ctx || !count) return DT_ERR_INVALID_ARG;
+    *count = ctx->launches;
+    return DT_OK;
+}
+
+dt_status dt_poll(dt_ctx *ctx) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    int32_t word = 0;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&word, ctx->status_dev, sizeof word, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && word != 0) e = cudaMemset(ctx->status_dev, 0, sizeof word);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "dt_poll");
+    if (word & dt::STATUS_WAIT_TIMEOUT) return fail(ctx, DT_ERR_TIMEOUT, "a bounded device-side wait expired");
+    if (word & dt::STATUS_REUSE_EMPTY) return fail(ctx, DT_ERR_STATE, "REUSE of a pair that was never computed");
+    return DT_OK;
+}
+
+}  // extern "C"

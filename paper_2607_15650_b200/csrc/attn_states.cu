@@ -1,0 +1,445 @@
+// dt_attn_states: Eq. 1 for every COMPUTE pair -- flash attention of one query block of
+// partition i against the keys of partition j only, emitting the partition-normalised output
+// OUT_ij and LSE_ij straight into the state cache.  REUSE pairs never appear in the work list,
+// so they cost no instruction and no byte.
+//
+// One persistent CTA per SM walks the work list (b*h slowest, then COMPUTE pair, then query
+// block), so CTAs running at the same time share one head's K/V partition through L2.
+//
+// Per CTA (10 warps):
+//   warps 0-3 / 4-7  softmax warpgroups for query tile 0 / 1 (128 rows each, one row per thread)
+//   warp 8           TMA producer: Q tiles once per work item, K and V tiles through a ring
+//   warp 9           MMA issuer (one elected lane): tcgen05.mma into TMEM
+// TMEM (512 columns): S0 | S1 | O0 | O1.  S_t = Q K_t^T (fp32) lands in S; the softmax warpgroup
+// reads its row, writes P = exp2(s*scale*log2e - m) back over S as packed bf16, and the PV MMA
+// takes P from TMEM as its A operand and V from shared memory (MN-major) as B, accumulating in O.
+// While one query tile is in softmax the tensor core works on the other (ping-pong).
+// The running maximum is only moved (and O, l rescaled) when it grew by more than 2^8: stale
+// maxima cancel exactly in OUT = O / l and LSE = m + log l.
+//
+// Every wait on an mbarrier is bounded; on expiry the CTA records STATUS_WAIT_TIMEOUT, leaves
+// its loops, frees TMEM and returns.
+#include <cuda_bf16.h>
+
+#include "dt_internal.h"
+#include "ptx_sm100.cuh"
+
+namespace dt {
+namespace {
+
+constexpr int NUM_SOFTMAX_THREADS = ATTN_NQ * 128;
+constexpr int TMA_WARP = NUM_SOFTMAX_THREADS / 32;
+constexpr int MMA_WARP = TMA_WARP + 1;
+constexpr int ATTN_THREADS = NUM_SOFTMAX_THREADS + 64;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s
+constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
+
+template <int D>
+struct Cfg {
+    static constexpr int NHALF = D / 64;                      // 64-element (128-byte) swizzle atoms per row
+    static constexpr int HALF_BYTES = ATTN_TILE * 128;        // one [128 rows x 64 bf16] box
+    static constexpr int TILE_BYTES = NHALF * HALF_BYTES;     // one Q, K or V tile
+    static constexpr int STAGES = (D == 128) ? 5 : 10;        // K/V ring depth
+    static constexpr int Q_BYTES = ATTN_NQ * TILE_BYTES;
+    static constexpr int KV_BYTES = STAGES * TILE_BYTES;
+    static constexpr int NBARS = 2 + 2 * STAGES + 4 * ATTN_NQ;
+    static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + Q_BYTES + KV_BYTES + NBARS * 8 + 64;
+    // TMEM columns
+    static constexpr int S_COL = 0;                           // S tile q: S_COL + q*128
+    static constexpr int O_COL = ATTN_NQ * 128;               // O tile q: O_COL + q*D
+};
+
+struct Bars {
+    uint32_t q_full, q_empty;
+    uint32_t kv_full, kv_empty;   // + 8*stage
+    uint32_t s_full, p_full, o_full, o_free;  // + 8*q
+};
+
+struct WorkItem {
+    int bh, b, h, i, j;
+    int q_row0;     // first query row of the block (global token index)
+    int n_q;        // valid query rows in the block (<= NQ*128)
+    int kv_row0;    // first key of partition j
+    int n_kv;       // keys in partition j
+    int tiles;      // ceil(n_kv / 128)
+};
+
+// Work index -> item.  Returns false when the block lies beyond the end of partition i.
+__device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, long long w, WorkItem &it) {
+    const long long per_bh = (long long)npairs * p.qblocks_max;
+    it.bh = (int)(w / per_bh);
+    const int rem = (int)(w - (long long)it.bh * per_bh);
+    const int pair = rem / p.qblocks_max;
+    const int qb = rem - pair * p.qblocks_max;
+    const int code = p.worklist[1 + pair];
+    it.i = code & 0xFF;
+    it.j = code >> 8;
+    it.b = it.bh / p.H;
+    it.h = it.bh - it.b * p.H;
+    const int qs = p.off[it.i], qe = p.off[it.i + 1];
+    it.q_row0 = qs + qb * (ATTN_NQ * ATTN_TILE);
+    it.n_q = min(qe - it.q_row0, ATTN_NQ * ATTN_TILE);
+    it.kv_row0 = p.off[it.j];
+    it.n_kv = p.off[it.j + 1] - it.kv_row0;
+    it.tiles = (it.n_kv + ATTN_TILE - 1) / ATTN_TILE;
+    return it.n_q > 0;
+}
+
+template <typename StateT>
+__device__ __forceinline__ void store_state_chunk(StateT *dst, const uint32_t (&r)[32], float inv_l);
+
+template <>
+__device__ __forceinline__ void store_state_chunk<float>(float *dst, const uint32_t (&r)[32], float inv_l) {
+#pragma unroll
+    for (int c = 0; c < 32; c += 4) {
+        float4 v = make_float4(__uint_as_float(r[c]) * inv_l, __uint_as_float(r[c + 1]) * inv_l,
+                               __uint_as_float(r[c + 2]) * inv_l, __uint_as_float(r[c + 3]) * inv_l);
+        __stcs(reinterpret_cast<float4 *>(dst + c), v);
+    }
+}
+template <>
+__device__ __forceinline__ void store_state_chunk<__nv_bfloat16>(__nv_bfloat16 *dst, const uint32_t (&r)[32], float inv_l) {
+#pragma unroll
+    for (int c = 0; c < 32; c += 8) {
+        uint4 v;
+        v.x = pack_bf16x2(__uint_as_float(r[c]) * inv_l, __uint_as_float(r[c + 1]) * inv_l);
+        v.y = pack_bf16x2(__uint_as_float(r[c + 2]) * inv_l, __uint_as_float(r[c + 3]) * inv_l);
+        v.z = pack_bf16x2(__uint_as_float(r[c + 4]) * inv_l, __uint_as_float(r[c + 5]) * inv_l);
+        v.w = pack_bf16x2(__uint_as_float(r[c + 6]) * inv_l, __uint_as_float(r[c + 7]) * inv_l);
+        __stcs(reinterpret_cast<uint4 *>(dst + c), v);
+    }
+}
+
+template <int D, typename StateT>
+__global__ void __launch_bounds__(ATTN_THREADS, 1)
+attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                   const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
+    using C = Cfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    // 1024-byte aligned carve-up (the 128-byte swizzle pattern repeats every 1024 bytes)
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t q_smem = smem_base;
+    const uint32_t kv_smem = q_smem + C::Q_BYTES;
+    const uint32_t bar_base = kv_smem + C::KV_BYTES;
+    Bars bars;
+    bars.q_full = bar_base;
+    bars.q_empty = bar_base + 8;
+    bars.kv_full = bar_base + 16;
+    bars.kv_empty = bars.kv_full + 8 * C::STAGES;
+    bars.s_full = bars.kv_empty + 8 * C::STAGES;
+    bars.p_full = bars.s_full + 8 * ATTN_NQ;
+    bars.o_full = bars.p_full + 8 * ATTN_NQ;
+    bars.o_free = bars.o_full + 8 * ATTN_NQ;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_ptr = &abort_flag;
+
+    if (warp == TMA_WARP && lane == 0) {
+        abort_flag = 0;
+        mbar_init(bars.q_full, 1);
+        mbar_init(bars.q_empty, 1);
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(bars.kv_full + 8 * s, 1);
+            mbar_init(bars.kv_empty + 8 * s, 1);
+        }
+        for (int q = 0; q < ATTN_NQ; ++q) {
+            mbar_init(bars.s_full + 8 * q, 1);
+            mbar_init(bars.p_full + 8 * q, 128);
+            mbar_init(bars.o_full + 8 * q, 1);
+            mbar_init(bars.o_free + 8 * q, 128);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    const int npairs = p.worklist[0];
+    const long long total_work = (long long)npairs * p.qblocks_max * p.B * p.H;
+
+    if (warp == TMA_WARP) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&tmap_q);
+            prefetch_tensormap(&tmap_k);
+            prefetch_tensormap(&tmap_v);
+            uint32_t q_phase = 0, kv_it = 0;
+            bool ok = true;
+            for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+                WorkItem it;
+                if (!decode_work(p, npairs, w, it)) continue;
+                ok = mbar_wait_bounded(bars.q_empty, q_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                if (!ok) break;
+                mbar_arrive_expect_tx(bars.q_full, C::Q_BYTES);
+#pragma unroll
+                for (int q = 0; q < ATTN_NQ; ++q)
+#pragma unroll
+                    for (int hf = 0; hf < C::NHALF; ++hf)
+                        tma_load_4d(q_smem + q * C::TILE_BYTES + hf * C::HALF_BYTES, &tmap_q, bars.q_full, hf * 64, it.h,
+                                    it.q_row0 + q * ATTN_TILE, it.b);
+                q_phase ^= 1u;
+                for (int t = 0; t < it.tiles && ok; ++t) {
+#pragma unroll
+                    for (int kv = 0; kv < 2; ++kv) {
+                        const uint32_t st = kv_it % C::STAGES, ph = (kv_it / C::STAGES) & 1u;
+                        ok = mbar_wait_bounded(bars.kv_empty + 8 * st, ph ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(bars.kv_full + 8 * st, C::TILE_BYTES);
+#pragma unroll
+                        for (int hf = 0; hf < C::NHALF; ++hf)
+                            tma_load_4d(kv_smem + st * C::TILE_BYTES + hf * C::HALF_BYTES, kv == 0 ? &tmap_k : &tmap_v,
+                                        bars.kv_full + 8 * st, hf * 64, it.h, it.kv_row0 + t * ATTN_TILE, it.b);
+                        ++kv_it;
+                    }
+                }
+            }
+            if (!ok) {
+                if (!*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
+                *abort_ptr = 1;
+                // let loads that are still in flight land before the CTA's shared memory goes away
+                const uint64_t t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    } else if (warp == MMA_WARP) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t IDESC_QK = make_idesc_bf16_f32(128, ATTN_TILE, false);
+            constexpr uint32_t IDESC_PV = make_idesc_bf16_f32(128, D, true);
+            uint32_t q_phase = 0, kv_it = 0, p_phase = 0, of_phase = 0;
+            bool ok = true;
+
+            // S[q] = Q[q] K^T for the K tile in ring stage `st`
+            auto issue_qk = [&](int q, uint32_t st) {
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t koff = (kk / 4) * C::HALF_BYTES + (kk % 4) * 32;
+                    const uint64_t a = make_smem_desc_sw128(q_smem + q * C::TILE_BYTES + koff, 16, 1024);
+                    const uint64_t b = make_smem_desc_sw128(kv_smem + st * C::TILE_BYTES + koff, 16, 1024);
+                    mma_ss(tmem_base + C::S_COL + q * 128, a, b, IDESC_QK, kk > 0 ? 1u : 0u);
+                }
+            };
+            // O[q] (+)= P[q] V for the V tile in ring stage `st`
+            auto issue_pv = [&](int q, uint32_t st, bool accumulate) {
+#pragma unroll
+                for (int kk = 0; kk < ATTN_TILE / 16; ++kk) {
+                    const uint64_t b =
+                        make_smem_desc_sw128(kv_smem + st * C::TILE_BYTES + kk * 2048, C::HALF_BYTES, 1024);
+                    mma_ts(tmem_base + C::O_COL + q * D, tmem_base + C::S_COL + q * 128 + kk * 8, b, IDESC_PV,
+                           (accumulate || kk > 0) ? 1u : 0u);
+                }
+            };
+
+            for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+                WorkItem it;
+                if (!decode_work(p, npairs, w, it)) continue;
+                ok = mbar_wait_bounded(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
+                if (!ok) break;
+                q_phase ^= 1u;
+                // first K tile
+                {
+                    const uint32_t st = kv_it % C::STAGES, ph = (kv_it / C::STAGES) & 1u;
+                    ok = mbar_wait_bounded(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int q = 0; q < ATTN_NQ; ++q) {
+                        issue_qk(q, st);
+                        tc_commit(bars.s_full + 8 * q);
+                    }
+                    tc_commit(bars.kv_empty + 8 * st);
+                    if (it.tiles == 1) tc_commit(bars.q_empty);
+                    ++kv_it;
+                }
+                for (int t = 0; t < it.tiles && ok; ++t) {
+                    const uint32_t st_v = kv_it % C::STAGES, ph_v = (kv_it / C::STAGES) & 1u;
+                    const uint32_t st_k = (kv_it + 1) % C::STAGES, ph_k = ((kv_it + 1) / C::STAGES) & 1u;
+                    const bool more = (t + 1 < it.tiles);
+                    ok = mbar_wait_bounded(bars.kv_full + 8 * st_v, ph_v, abort_ptr, WAIT_LIMIT_NS);
+                    if (!ok) break;
+#pragma unroll
+                    for (int q = 0; q < ATTN_NQ; ++q) {
+                        ok = mbar_wait_bounded(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_NS);
+                        if (!ok) break;
+                        if (t == 0) {  // the previous item's epilogue must have drained O[q]
+                            ok = mbar_wait_bounded(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                        issue_pv(q, st_v, t > 0);
+                        if (!more) tc_commit(bars.o_full + 8 * q);
+                        if (more) {
+                            if (q == 0) {
+                                ok = mbar_wait_bounded(bars.kv_full + 8 * st_k, ph_k, abort_ptr, WAIT_LIMIT_NS);
+                                if (!ok) break;
+                                tc_fence_after();
+                            }
+                            issue_qk(q, st_k);
+                            tc_commit(bars.s_full + 8 * q);
+                        }
+                    }
+                    if (!ok) break;
+                    tc_commit(bars.kv_empty + 8 * st_v);
+                    ++kv_it;
+                    if (more) {
+                        tc_commit(bars.kv_empty + 8 * st_k);
+                        ++kv_it;
+                        if (t + 2 == it.tiles) tc_commit(bars.q_empty);
+                    }
+                    p_phase ^= 1u;
+                }
+                of_phase ^= 1u;
+            }
+            if (!ok) {
+                if (!*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
+                *abort_ptr = 1;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax warpgroups
+        const int q = warp / 4;                       // query tile handled by this warpgroup
+        const int row_in_tile = (warp % 4) * 32 + lane;
+        const uint32_t lane_addr = ((uint32_t)((warp % 4) * 32)) << 16;
+        const uint32_t s_tmem = tmem_base + lane_addr + C::S_COL + q * 128;
+        const uint32_t o_tmem = tmem_base + lane_addr + C::O_COL + q * D;
+        uint32_t s_phase = 0, o_phase = 0;
+        bool ok = true;
+        StateT *o_state = static_cast<StateT *>(p.o_state);
+
+        for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+            WorkItem it;
+            if (!decode_work(p, npairs, w, it)) continue;
+            float m_used = -INFINITY, l_sum = 0.f;
+            for (int t = 0; t < it.tiles; ++t) {
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.s_full + 8 * q, s_phase, abort_ptr, WAIT_LIMIT_NS));
+                if (!ok) break;
+                s_phase ^= 1u;
+                tc_fence_after();
+                uint32_t s[4][32];   // this thread's row of S: 128 fp32 logits (before scaling)
+                tmem_ld_x32(s_tmem + 0, s[0]);
+                tmem_ld_x32(s_tmem + 32, s[1]);
+                tmem_ld_x32(s_tmem + 64, s[2]);
+                tmem_ld_x32(s_tmem + 96, s[3]);
+                tmem_wait_ld();
+                const int valid = it.n_kv - t * ATTN_TILE;   // keys of this tile that belong to partition j
+                if (valid < ATTN_TILE) {
+#pragma unroll
+                    for (int c = 0; c < 128; ++c)
+                        if (c >= valid) s[c >> 5][c & 31] = 0xFF800000u;  // -inf
+                }
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(s[c >> 5][c & 31]));
+                const float m_new = fmaxf(m_used, mx * p.scale_log2);
+                // move the reference maximum only when it grew by more than 2^RESCALE_THRESHOLD
+                const bool need = (m_new - m_used > RESCALE_THRESHOLD);   // true on the first tile (m_used = -inf)
+                if (t == 0) {
+                    m_used = m_new;
+                } else if (__any_sync(0xFFFFFFFFu, need)) {
+                    const float alpha = need ? ex2_approx(m_used - m_new) : 1.0f;
+                    if (need) m_used = m_new;
+                    l_sum *= alpha;
+#pragma unroll
+                    for (int c0 = 0; c0 < D; c0 += 32) {
+                        uint32_t o[32];
+                        tmem_ld_x32(o_tmem + c0, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                        tmem_st_x32(o_tmem + c0, o);
+                    }
+                }
+                const float neg_m = -m_used;
+                float rs = 0.f;
+                uint32_t pk[2][32];  // P row as packed bf16 pairs (key 2c in the low half)
+#pragma unroll
+                for (int c = 0; c < 128; c += 2) {
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(s[c >> 5][c & 31]), p.scale_log2, neg_m));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(s[(c + 1) >> 5][(c + 1) & 31]), p.scale_log2, neg_m));
+                    rs += p0 + p1;
+                    pk[c >> 6][(c >> 1) & 31] = pack_bf16x2(p0, p1);
+                }
+                l_sum += rs;
+                tmem_st_x32(s_tmem + 0, pk[0]);
+                tmem_st_x32(s_tmem + 32, pk[1]);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bars.p_full + 8 * q);
+            }
+            if (!ok) break;
+            // epilogue: OUT_ij = O / l, LSE_ij = ln2 * (m + log2 l); rows beyond the partition are dropped
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.o_full + 8 * q, o_phase, abort_ptr, WAIT_LIMIT_NS));
+            if (!ok) break;
+            o_phase ^= 1u;
+            tc_fence_after();
+            const int row_in_block = q * ATTN_TILE + row_in_tile;
+            const bool row_valid = row_in_block < it.n_q;
+            const float inv_l = 1.0f / l_sum;
+            const long long srow = ((long long)it.j * p.B * p.H + it.bh) * p.L + it.q_row0 + row_in_block;
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t o[32];
+                tmem_ld_x32(o_tmem + c0, o);
+                tmem_wait_ld();
+                if (c0 + 32 >= D) {  // O[q] fully read: the next item's first PV may overwrite it
+                    tc_fence_before();
+                    mbar_arrive(bars.o_free + 8 * q);
+                }
+                if (row_valid) store_state_chunk<StateT>(o_state + srow * D + c0, o, inv_l);
+            }
+            if (row_valid) p.lse_state[srow] = 0.69314718055994530942f * (m_used + log2f(l_sum));
+        }
+        if (!ok && lane == 0) {
+            if (!*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
+            *abort_ptr = 1;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+template <int D, typename StateT>
+cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const AttnParams &p,
+                   int num_ctas, cudaStream_t stream) {
+    attn_states_kernel<D, StateT><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, p);
+    return cudaGetLastError();
+}
+
+template <int D, typename StateT>
+cudaError_t configure() {
+    return cudaFuncSetAttribute(attn_states_kernel<D, StateT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Cfg<D>::SMEM_BYTES);
+}
+
+}  // namespace
+
+cudaError_t attn_states_configure() {
+    cudaError_t e;
+    if ((e = configure<64, float>()) != cudaSuccess) return e;
+    if ((e = configure<128, float>()) != cudaSuccess) return e;
+    if ((e = configure<64, __nv_bfloat16>()) != cudaSuccess) return e;
+    return configure<128, __nv_bfloat16>();
+}
+
+cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
+                               const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream) {
+    if (state_dtype == DT_STATE_FP32) {
+        return D == 64 ? launch<64, float>(tq, tk, tv, p, num_ctas, stream)
+                       : launch<128, float>(tq, tk, tv, p, num_ctas, stream);
+    }
+    return D == 64 ? launch<64, __nv_bfloat16>(tq, tk, tv, p, num_ctas, stream)
+                   : launch<128, __nv_bfloat16>(tq, tk, tv, p, num_ctas, stream);
+}
+
+}  // namespace dt

@@ -1,0 +1,90 @@
+// Internal declarations shared by the translation units of libditango.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/ditango.h"
+
+namespace dt {
+
+// Device status word bits (read by dt_poll).
+enum : int { STATUS_REUSE_EMPTY = 1, STATUS_WAIT_TIMEOUT = 2 };
+
+constexpr int PLAN_CHUNK_ROWS = 1024;  // rows of one (b, h, partition) handled by one dt_plan block
+constexpr int ATTN_TILE = 128;         // query rows per TMEM accumulator / keys per KV tile
+constexpr int ATTN_NQ = 2;             // query tiles a CTA keeps in flight (ping-pong)
+
+struct AttnParams {
+    const int32_t *off;       // device, P+1
+    const int32_t *worklist;  // device: [0] = number of COMPUTE pairs, then i | (j << 8) per pair
+    int32_t *status;          // device status word
+    void *o_state;            // [P][B][H][L][D]
+    float *lse_state;         // [P][B][H][L]
+    int B, H, L, P;
+    int qblocks_max;          // ceil(max_i n_i / (ATTN_NQ * ATTN_TILE))
+    float scale_log2;         // softmax_scale * log2(e)
+};
+
+struct MergeParams {
+    const void *o_state;
+    const float *lse_state;
+    void *out;       // bf16
+    float *lse_out;  // may be null
+    int P, H, L;
+    long long R;     // B*H*L rows
+    long long sb, sl, sh;  // output strides in elements
+};
+
+struct PlanParams {
+    const float *lse_state;  // [P][R]
+    const int32_t *off;      // device, P+1
+    float *partials;         // [BH][P][chunks][P]
+    int P, BH, L, chunks;
+    long long R;
+};
+
+struct PlanFinalParams {
+    const float *partials;
+    const int32_t *off;
+    int P, BH, chunks;
+    int mode_target;   // 0: threshold with eps; 1: select K pairs by rank
+    int K;
+    double eps;
+    uint8_t *mask;
+    double *w_out;     // may be null
+    double *eps_out;   // may be null
+};
+
+cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, int P, int step,
+                            cudaStream_t stream);
+cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
+                               const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream);
+cudaError_t attn_states_configure();  // sets the dynamic shared-memory attribute once per process/device
+cudaError_t launch_state_merge(const MergeParams &p, int D, int state_dtype, cudaStream_t stream);
+cudaError_t launch_plan_partial(const PlanParams &p, cudaStream_t stream);
+cudaError_t launch_plan_final(const PlanFinalParams &p, cudaStream_t stream);
+
+}  // namespace dt
+
+struct dt_ctx {
+    dt_config cfg;
+    std::vector<int32_t> off;
+    int n_max = 0;
+    int qblocks_max = 0;
+    int plan_chunks = 0;
+    int num_sms = 0;
+    int32_t *off_dev = nullptr;
+    int32_t *tc_dev = nullptr;
+    int32_t *worklist_dev = nullptr;
+    int32_t *status_dev = nullptr;
+    float *plan_partials_dev = nullptr;
+    void *o_state = nullptr;
+    float *lse_state = nullptr;
+    uint64_t launches = 0;
+    std::string err;
+    void *encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
+};

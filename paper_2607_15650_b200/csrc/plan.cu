@@ -1,0 +1,167 @@
+// dt_plan: partition importance weights (Eq. 8) reduced to one contribution value per
+// (query partition, KV partition) pair and thresholded into the COMPUTE / REUSE mask (Eq. 13),
+// plus the work-list builder that turns a mask into the list of pairs dt_attn_states evaluates.
+//
+// Stage 1 (HBM-bound, P * 4 bytes per query row): one block handles up to PLAN_CHUNK_ROWS rows of
+// one (b, h, query partition i), so all its threads share i.  Each thread reads the P cached
+// LSE_ij of a row (coalesced across rows), forms w_j = exp(LSE_ij - logsumexp_k LSE_ik) in fp32
+// and keeps P running sums; a fixed-order block reduction writes P partial sums to scratch.
+// Stage 2 (one block): sums the partials in fp64 in a fixed order, divides by the row count,
+// and either thresholds (W > eps, strict) or ranks the off-diagonal pairs to hit a target count.
+// No atomics: the result is bit-reproducible from run to run.
+#include "dt_internal.h"
+
+namespace dt {
+namespace {
+
+constexpr int PLAN_THREADS = 256;
+
+template <int PMAX>
+__global__ void __launch_bounds__(PLAN_THREADS) plan_partial_kernel(PlanParams p) {
+    const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z;
+    const int P = p.P;
+    const int row0 = p.off[i] + c * PLAN_CHUNK_ROWS;
+    const int row1 = min(row0 + PLAN_CHUNK_ROWS, p.off[i + 1]);
+    float acc[PMAX];
+#pragma unroll
+    for (int j = 0; j < PMAX; ++j) acc[j] = 0.f;
+    const float *base = p.lse_state + (long long)bh * p.L;
+    for (int l = row0 + (int)threadIdx.x; l < row1; l += PLAN_THREADS) {
+        float x[PMAX];
+        float M = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < PMAX; ++j) {
+            x[j] = (j < P) ? __ldcs(base + (long long)j * p.R + l) : -INFINITY;
+            M = fmaxf(M, x[j]);
+        }
+        if (M == -INFINITY) continue;  // row without any mass: contributes nothing
+        float Z = 0.f;
+#pragma unroll
+        for (int j = 0; j < PMAX; ++j) {
+            x[j] = expf(x[j] - M);
+            Z += x[j];
+        }
+        const float inv = 1.f / Z;
+#pragma unroll
+        for (int j = 0; j < PMAX; ++j) acc[j] = fmaf(x[j], inv, acc[j]);
+    }
+    // block reduction in a fixed order: xor-shuffle tree inside a warp, then warp 0 adds the 8 warps
+    __shared__ float red[PLAN_THREADS / 32][PMAX];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int j = 0; j < PMAX; ++j) {
+        float v = acc[j];
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, s);
+        if (lane == 0) red[warp][j] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < P) {
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < PLAN_THREADS / 32; ++w) v += red[w][threadIdx.x];
+        p.partials[(((long long)bh * P + i) * p.chunks + c) * P + threadIdx.x] = v;
+    }
+}
+
+// Strict total order used to rank off-diagonal pairs: larger W first, then smaller |i-j|, then
+// smaller flat index.
+__device__ __forceinline__ bool ranks_before(double wa, int da, int fa, double wb, int db, int fb) {
+    if (wa != wb) return wa > wb;
+    if (da != db) return da < db;
+    return fa < fb;
+}
+
+__global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
+    __shared__ double W[DT_MAX_P * DT_MAX_P];
+    __shared__ double edge[2];
+    const int P = p.P, total = P * P;
+    const int e = threadIdx.x;
+    const int i = e / P, j = e - i * P;
+    if (e < total) {
+        double s = 0.0;
+        for (int bh = 0; bh < p.BH; ++bh)
+            for (int c = 0; c < p.chunks; ++c) s += (double)p.partials[(((long long)bh * P + i) * p.chunks + c) * P + j];
+        const double cnt = (double)p.BH * (double)(p.off[i + 1] - p.off[i]);
+        W[e] = s / cnt;
+        if (p.w_out) p.w_out[e] = W[e];
+    }
+    if (e < 2) edge[e] = 0.0;
+    __syncthreads();
+    if (!p.mode_target) {
+        if (e < total) p.mask[e] = (i == j || W[e] > p.eps) ? 1 : 0;
+        if (e == 0 && p.eps_out) *p.eps_out = p.eps;
+        return;
+    }
+    const int noff = total - P, sel = p.K - P;
+    int rank = -1;
+    if (e < total && i != j) {
+        rank = 0;
+        const double w = W[e];
+        const int d = i > j ? i - j : j - i;
+        for (int o = 0; o < total; ++o) {
+            const int oi = o / P, oj = o - oi * P;
+            if (oi == oj || o == e) continue;
+            const int od = oi > oj ? oi - oj : oj - oi;
+            if (ranks_before(W[o], od, o, w, d, e)) ++rank;
+        }
+        if (rank == sel - 1) edge[0] = w;
+        if (rank == sel) edge[1] = w;
+    }
+    if (e < total) p.mask[e] = (i == j || (rank >= 0 && rank < sel)) ? 1 : 0;
+    __syncthreads();
+    if (e == 0 && p.eps_out) {
+        double eps;
+        if (noff == 0 || sel == noff) eps = 0.0;
+        else if (sel == 0) eps = edge[1];
+        else eps = 0.5 * (edge[0] + edge[1]);
+        *p.eps_out = eps;
+    }
+}
+
+// mask -> compact list of COMPUTE pairs (ordered by i*P+j), t_c update, REUSE-of-empty detection.
+__global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int32_t *tc, int32_t *worklist,
+                                                        int32_t *status, int P, int step) {
+    __shared__ uint8_t flag[DT_MAX_P * DT_MAX_P];
+    const int total = P * P, e = threadIdx.x;
+    bool f = false;
+    if (e < total) {
+        f = mask[e] != 0;
+        flag[e] = f ? 1 : 0;
+        if (f) tc[e] = step;
+        else if (tc[e] < 0) atomicOr(status, STATUS_REUSE_EMPTY);
+    }
+    __syncthreads();
+    if (e < total) {
+        int pos = 0, cnt = 0;
+        for (int o = 0; o < total; ++o) {
+            cnt += flag[o];
+            if (o < e) pos += flag[o];
+        }
+        if (f) worklist[1 + pos] = (e / P) | ((e % P) << 8);
+        if (e == 0) worklist[0] = cnt;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_plan_partial(const PlanParams &p, cudaStream_t stream) {
+    dim3 grid((unsigned)p.chunks, (unsigned)p.P, (unsigned)p.BH);
+    if (p.P <= 8) plan_partial_kernel<8><<<grid, PLAN_THREADS, 0, stream>>>(p);
+    else if (p.P <= 16) plan_partial_kernel<16><<<grid, PLAN_THREADS, 0, stream>>>(p);
+    else plan_partial_kernel<32><<<grid, PLAN_THREADS, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_plan_final(const PlanFinalParams &p, cudaStream_t stream) {
+    plan_final_kernel<<<1, 1024, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, int P, int step,
+                            cudaStream_t stream) {
+    worklist_kernel<<<1, 1024, 0, stream>>>(mask, tc, worklist, status, P, step);
+    return cudaGetLastError();
+}
+
+}  // namespace dt

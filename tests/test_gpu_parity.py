@@ -1,0 +1,304 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded
+inputs.  Tolerances are the ones stated for bf16 inputs with fp32 accumulation:
+O max-abs <= 2e-2 and mean-abs <= 2e-3, LSE abs <= 5e-3, plan mask bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2607_15650_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+
+O_MAX, O_MEAN, LSE_ABS = 2e-2, 2e-3, 5e-3
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    binding.lib()
+
+
+def check_o(got, ref, what=""):
+    err = np.abs(np.asarray(got, dtype=np.float64) - ref)
+    assert err.max() <= O_MAX, f"{what}: O max abs err {err.max():.3e}"
+    assert err.mean() <= O_MEAN, f"{what}: O mean abs err {err.mean():.3e}"
+
+
+def check_lse(got, ref, what=""):
+    err = np.abs(np.asarray(got, dtype=np.float64) - ref)
+    assert err.max() <= LSE_ABS, f"{what}: LSE max abs err {err.max():.3e}"
+
+
+class Run:
+    """Drives one workload through the C ABI and the oracle side by side."""
+
+    def __init__(self, wl, rows_by_bh=None, state_dtype=binding.DT_STATE_FP32, seed=0, offsets=None):
+        self.wl = wl
+        self.off = wl.offsets() if offsets is None else np.asarray(offsets, dtype=np.int32)
+        self.P = self.off.size - 1
+        self.dev = torch.device("cuda", 0)
+        self.ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, self.off, wl.scale, state_dtype, 0)
+        self.gen = inputs.StepInputs(wl, seed=seed, device=self.dev)
+        if rows_by_bh is None:
+            rows_by_bh = {(b, h): np.arange(wl.L, dtype=np.int32) for b in range(wl.B) for h in range(wl.H)}
+        self.rows = rows_by_bh
+        self.ses = orc.OracleSession(wl.B, wl.L, wl.H, wl.D, self.off, wl.scale, rows_by_bh)
+        self.out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=self.dev)
+        self.lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=self.dev)
+        self.t = 0
+
+    def step(self, mask, check_states=False):
+        self.t += 1
+        q, k, v = self.gen.next()
+        mask = np.ascontiguousarray(mask, dtype=np.uint8).reshape(self.P, self.P)
+        mask_dev = torch.from_numpy(mask).to(self.dev)
+        self.ctx.dt_attn_states(q, k, v, mask_dev, self.t)
+        self.ctx.dt_state_merge(self.out, self.lse)
+        torch.cuda.synchronize()
+        self.ctx.dt_poll()
+        qb, kb, vb = (inputs.bf16_bits(x) for x in (q, k, v))
+        outs, lses = self.ses.step(qb, kb, vb, mask, self.t)
+        out_h = self.out.float().cpu().numpy()
+        lse_h = self.lse.cpu().numpy()
+        for (b, h), rows in self.rows.items():
+            check_o(out_h[b, rows, h, :], outs[(b, h)], f"step {self.t} head {h} merged")
+            check_lse(lse_h[b, h, rows], lses[(b, h)], f"step {self.t} head {h} merged")
+        if check_states:
+            o_st = self.ctx.o_state.float().cpu().numpy()     # [P, B, H, L, D]
+            l_st = self.ctx.lse_state.cpu().numpy()           # [P, B, H, L]
+            for (b, h), rows in self.rows.items():
+                for j in range(self.P):
+                    check_o(o_st[j, b, h, rows, :], self.ses.o[(b, h)][:, j, :], f"step {self.t} state j={j}")
+                    check_lse(l_st[j, b, h, rows], self.ses.lse[(b, h)][:, j], f"step {self.t} state j={j}")
+        assert (self.ctx.dt_get_tc() == self.ses.tc).all()
+        return q, k, v
+
+
+def test_config0_two_steps_full_then_banded():
+    """Correctness config: 1024 tokens, 2 heads, D = 64, P = 4; step 1 computes all 16 pairs, step 2
+    computes |i-j| <= 1 and reuses the rest from step 1.  Every pair state and the merged output are
+    compared element by element."""
+    wl = inputs.WORKLOADS["c0_correctness"]
+    run = Run(wl)
+    run.step(np.ones((4, 4), np.uint8), check_states=True)
+    run.step(inputs.banded_mask(4, 1), check_states=True)
+    assert run.ctx.dt_launch_count() == 6
+
+
+@pytest.mark.parametrize("D,grid,n_text,offsets", [
+    (64, (2, 6, 7), 0, [0, 30, 61, 84]),                 # partitions smaller than one tile
+    (128, (3, 9, 11), 5, [0, 100, 302]),                 # ragged tail inside a 128-row tile, text rows
+    (128, (4, 11, 13), 0, [0, 129, 385, 572]),           # 1 / 2 / 1.46 tiles
+    (64, (5, 12, 13), 3, [0, 300, 783]),                 # more than one 256-row query block per partition
+])
+def test_ragged_partitions_and_tails(D, grid, n_text, offsets):
+    wl = inputs.Workload("ragged", 1, 3, D, grid, n_text, len(offsets) - 1, 2, 0.05)
+    assert wl.L == offsets[-1]
+    P = len(offsets) - 1
+    run = Run(wl, offsets=offsets, seed=5)
+    run.step(np.ones((P, P), np.uint8), check_states=True)
+    run.step(np.eye(P, dtype=np.uint8), check_states=True)
+
+
+def test_batch_two_and_bf16_state_cache():
+    wl = inputs.Workload("b2", 2, 2, 128, (2, 10, 13), 0, 2, 2, 0.05)
+    run = Run(wl, state_dtype=binding.DT_STATE_BF16, seed=2)
+    run.step(np.ones((2, 2), np.uint8), check_states=True)
+    run.step(np.array([[1, 0], [1, 1]], np.uint8), check_states=True)
+
+
+def test_strided_inputs_and_output():
+    """Q, K, V packed as one [B, L, 3, H, D] buffer (strides are not the contiguous ones)."""
+    wl = inputs.Workload("strided", 1, 2, 64, (2, 8, 9), 0, 2, 1, 0.05)
+    dev = torch.device("cuda", 0)
+    q, k, v = inputs.StepInputs(wl, seed=7, device=dev).next()
+    packed = torch.stack([q, k, v], dim=2).contiguous()
+    qs, ks, vs = packed[:, :, 0], packed[:, :, 1], packed[:, :, 2]
+    assert not qs.is_contiguous()
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale)
+    ones = torch.ones(4, dtype=torch.uint8, device=dev)
+    out_wide = torch.zeros((wl.B, wl.L, 2, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
+    out = out_wide[:, :, 1]
+    ctx.dt_attn_states(qs, ks, vs, ones, 1)
+    ctx.dt_state_merge(out, None)
+    torch.cuda.synchronize()
+    ctx.dt_poll()
+    qb, kb, vb = (inputs.bf16_bits(x) for x in (q, k, v))
+    for h in range(wl.H):
+        ref, _ = orc.full_attention(qb, kb, vb, wl.scale, 0, h, np.arange(wl.L, dtype=np.int32))
+        check_o(out[0, :, h].float().cpu().numpy(), ref, "strided")
+    assert (out_wide[:, :, 0] == 0).all()
+
+
+def test_state_merge_alone_on_oracle_states():
+    """dt_state_merge fed with states produced by the oracle (uploaded), against the oracle's merge."""
+    rng = np.random.default_rng(3)
+    B, H, D, L, P = 1, 3, 128, 77, 5
+    off = orc.uniform_offsets(L, P)
+    o_st = rng.standard_normal((P, B, H, L, D))
+    l_st = rng.standard_normal((P, B, H, L)) * 4.0
+    l_st[2, 0, 1, 5] = -np.inf                       # a state without mass has weight zero
+    dev = torch.device("cuda", 0)
+    for sdt, tdt in ((binding.DT_STATE_FP32, torch.float32), (binding.DT_STATE_BF16, torch.bfloat16)):
+        ctx = binding.Context(B, H, D, L, off, 0.1, sdt, alloc_cache=False)
+        o_dev = torch.from_numpy(o_st).to(tdt).to(dev)
+        l_dev = torch.from_numpy(l_st).to(torch.float32).to(dev)
+        ctx.dt_bind_cache(o_dev, l_dev)
+        out = torch.empty((B, L, H, D), dtype=torch.bfloat16, device=dev)
+        lse = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+        ctx.dt_state_merge(out, lse)
+        torch.cuda.synchronize()
+        o_in = o_dev.double().cpu().numpy()              # what the kernel actually read
+        l_in = l_dev.double().cpu().numpy()
+        ref_o, ref_l = orc.merge(np.moveaxis(o_in, 0, 3).reshape(B * H * L, P, D),
+                                 np.moveaxis(l_in, 0, 3).reshape(B * H * L, P))
+        got = out.float().cpu().numpy().transpose(0, 2, 1, 3).reshape(B * H * L, D)
+        check_o(got, ref_o, "merge alone")
+        check_lse(lse.cpu().numpy().reshape(-1), ref_l, "merge alone")
+
+
+def _plan_case(wl, lse_host, off, fractions, eps_list):
+    """dt_plan on a given LSE cache (fp32 values) against the oracle fed the same values."""
+    dev = torch.device("cuda", 0)
+    P = off.size - 1
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, off, wl.scale, alloc_cache=False)
+    o_dummy = torch.empty((P, wl.B, wl.H, wl.L, wl.D), dtype=torch.float32, device=dev)
+    l_dev = torch.from_numpy(lse_host.astype(np.float32)).to(dev)
+    ctx.dt_bind_cache(o_dummy, l_dev)
+    W_ref = orc.contribution(lse_host.astype(np.float32).astype(np.float64), off)
+    mask = torch.empty(P * P, dtype=torch.uint8, device=dev)
+    W = torch.empty(P * P, dtype=torch.float64, device=dev)
+    eps_out = torch.empty(1, dtype=torch.float64, device=dev)
+    for f in fractions:
+        ctx.dt_plan(mask, target_fraction=f, w_dev=W, eps_out_dev=eps_out)
+        torch.cuda.synchronize()
+        Wg = W.cpu().numpy().reshape(P, P)
+        np.testing.assert_allclose(Wg, W_ref, rtol=2e-5, atol=1e-9)
+        np.testing.assert_allclose(Wg.sum(1), 1.0, atol=1e-5)
+        ref_mask, ref_eps, K = orc.target_fraction(W_ref, f)
+        # the decision itself, taken on the GPU's own W in the same precision, must be reproduced exactly
+        own_mask, own_eps, _ = orc.target_fraction(Wg, f)
+        got = mask.cpu().numpy().reshape(P, P)
+        assert (got == own_mask).all() and eps_out.item() == own_eps
+        assert got.sum() == K
+        # and it equals the oracle's plan whenever the oracle's own margin is resolvable in fp32
+        offd = ~np.eye(P, dtype=bool)
+        gap = np.abs(W_ref[offd] - ref_eps).min() / max(ref_eps, 1e-300)
+        if gap > 1e-4:
+            assert (got == ref_mask).all()
+            assert eps_out.item() == pytest.approx(ref_eps, rel=1e-4)
+    for eps in eps_list:
+        ctx.dt_plan(mask, eps=eps, w_dev=W, eps_out_dev=eps_out)
+        torch.cuda.synchronize()
+        Wg = W.cpu().numpy().reshape(P, P)
+        got = mask.cpu().numpy().reshape(P, P)
+        assert (got == orc.threshold(Wg, eps)).all() and eps_out.item() == eps
+        if (np.abs(W_ref - eps)[~np.eye(P, dtype=bool)].min() / eps) > 1e-4:
+            assert (got == orc.threshold(W_ref, eps)).all()
+    # run-to-run bit reproducibility (no atomics in the reduction)
+    W2 = torch.empty_like(W)
+    ctx.dt_plan(mask, eps=0.1, w_dev=W2)
+    torch.cuda.synchronize()
+    assert torch.equal(W, W2)
+
+
+def test_plan_on_synthetic_lse_uneven_partitions():
+    rng = np.random.default_rng(4)
+    wl = inputs.Workload("plan", 2, 3, 64, (1, 1, 2500), 0, 5, 1, 0.05)
+    off = np.array([0, 100, 1300, 1301, 2400, 2500], np.int32)
+    P = 5
+    dist = np.abs(np.subtract.outer(np.arange(P), np.arange(P)))
+    part = np.searchsorted(off, np.arange(wl.L), side="right") - 1
+    lse = rng.standard_normal((P, wl.B, wl.H, wl.L)) * 0.5
+    for j in range(P):
+        lse[j] += -1.1 * dist[part, j]
+    _plan_case(wl, lse, off, [0.0, 0.2, 0.4, 0.52, 0.8, 1.0], [0.05, 0.2, 0.5])
+
+
+def test_plan_threshold_equality_is_reuse():
+    """W exactly equal to eps must give REUSE (strict '>'): constant LSEs give W = 1/P exactly."""
+    wl = inputs.Workload("eq", 1, 1, 64, (1, 1, 64), 0, 4, 1, 0.05)
+    off = wl.offsets()
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, off, wl.scale, alloc_cache=False)
+    ctx.dt_bind_cache(torch.empty((4, 1, 1, 64, 64), device=dev), torch.zeros((4, 1, 1, 64), device=dev))
+    mask = torch.empty(16, dtype=torch.uint8, device=dev)
+    ctx.dt_plan(mask, eps=0.25)
+    assert (mask.cpu().numpy().reshape(4, 4) == np.eye(4)).all()
+    ctx.dt_plan(mask, eps=0.2499999)
+    assert mask.cpu().numpy().all()
+
+
+def test_plan_from_gpu_states_of_config0_matches_oracle_plan():
+    """End of an anchor step: dt_plan on the cache dt_attn_states just filled, against the oracle's
+    plan from the oracle's own LSEs (f = 0.5), and the plan then drives the next step."""
+    wl = inputs.WORKLOADS["c0_correctness"]
+    run = Run(wl)
+    run.step(np.ones((4, 4), np.uint8))
+    dev = run.dev
+    mask = torch.empty(16, dtype=torch.uint8, device=dev)
+    W = torch.empty(16, dtype=torch.float64, device=dev)
+    run.ctx.dt_plan(mask, target_fraction=0.5, w_dev=W)
+    torch.cuda.synchronize()
+    lse_ref = np.empty((4, wl.B, wl.H, wl.L))
+    for (b, h), rows in run.rows.items():
+        lse_ref[:, b, h, :] = run.ses.lse[(b, h)].T
+    W_ref = orc.contribution(lse_ref, run.off)
+    np.testing.assert_allclose(W.cpu().numpy().reshape(4, 4), W_ref, rtol=1e-3, atol=1e-6)
+    ref_mask, ref_eps, K = orc.target_fraction(W_ref, 0.5)
+    got = mask.cpu().numpy().reshape(4, 4)
+    assert K == 8 and got.sum() == 8
+    assert (got == ref_mask).all()
+    run.step(got, check_states=True)
+
+
+def test_reuse_of_never_computed_pair_is_reported():
+    wl = inputs.tiny_workload(grid=(2, 6, 7), P=3)
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale)
+    q, k, v = inputs.StepInputs(wl, device=dev).next()
+    ctx.dt_attn_states(q, k, v, torch.eye(3, dtype=torch.uint8, device=dev).reshape(-1).contiguous(), 0)
+    with pytest.raises(binding.DitangoError) as ei:
+        ctx.dt_poll()
+    assert ei.value.status == binding.DT_ERR_STATE
+    ctx.dt_poll()                                            # cleared by the first poll
+    tc = ctx.dt_get_tc()
+    assert (tc.diagonal() == 0).all() and tc[0, 1] == -1
+    # snapshot / resume of t_c
+    tc2 = tc.copy(); tc2[0, 1] = 5
+    ctx.dt_set_tc(tc2)
+    assert (ctx.dt_get_tc() == tc2).all()
+
+
+def test_argument_errors_do_not_launch():
+    wl = inputs.tiny_workload()
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale, alloc_cache=False)
+    q, k, v = inputs.StepInputs(wl, device=dev).next()
+    mask = torch.ones(9, dtype=torch.uint8, device=dev)
+    with pytest.raises(binding.DitangoError) as ei:
+        ctx.dt_attn_states(q, k, v, mask, 1)                 # cache not bound
+    assert ei.value.status == binding.DT_ERR_STATE
+    with pytest.raises(binding.DitangoError) as ei:
+        ctx.dt_bind_cache(torch.empty(16, device=dev), torch.empty(16, device=dev))   # too small
+    assert ei.value.status == binding.DT_ERR_STATE
+    assert ctx.dt_launch_count() == 0
+
+
+def test_step_from_host_buffers():
+    wl = inputs.Workload("host", 1, 2, 64, (2, 9, 10), 0, 2, 1, 0.05)
+    q, k, v = inputs.StepInputs(wl, seed=9, device="cpu").next()
+    qp, kp, vp = (x.contiguous().pin_memory() for x in (q, k, v))
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale)
+    ws = torch.empty(binding.dt_step_host_workspace_bytes(ctx.cfg), dtype=torch.uint8, device="cuda:0")
+    out = torch.empty_like(q).pin_memory()
+    lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32).pin_memory()
+    mask = torch.ones(4, dtype=torch.uint8)
+    ctx.dt_step_host(qp, kp, vp, mask, 1, out, lse, ws)
+    ctx.dt_poll()
+    qb, kb, vb = (inputs.bf16_bits(x) for x in (q, k, v))
+    for h in range(wl.H):
+        ref, ref_l = orc.full_attention(qb, kb, vb, wl.scale, 0, h, np.arange(wl.L, dtype=np.int32))
+        check_o(out[0, :, h].float().numpy(), ref, "host step")
+        check_lse(lse[0, h].numpy(), ref_l, "host step")
