@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the selective attention-state path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One timed "step" is one selective denoising step of the whole hot path on one attention layer:
+dt_attn_states (COMPUTE pairs of the current plan) + dt_state_merge (all P states per row) +
+dt_plan (contribution measure of the refreshed cache -> plan of the next step).  Before the timed
+region an anchor step computes every pair and the first plan is derived from it.  Inputs (bf16
+Q, K, V of every denoising step of the workload) are resident in HBM; they and the state cache
+are far larger than L2, so no explicit flush is needed.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead, on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_15650_b200 import inputs  # noqa: E402
+
+METRIC = "effective_attn_tflops"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "c3_wan720p"
+
+
+# ------------------------------------------------------------------------------------------ helpers
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.idx = device_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.idx)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as fh:
+            for line in fh:
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def full_flops(wl) -> float:
+    return 4.0 * wl.L * wl.L * wl.D * wl.H * wl.B
+
+
+def computed_flops(wl, mask: np.ndarray) -> float:
+    n = np.diff(wl.offsets()).astype(np.float64)
+    return 4.0 * wl.D * wl.H * wl.B * float((np.outer(n, n) * (mask.reshape(wl.P, wl.P) != 0)).sum())
+
+
+def merge_bytes(wl, state_bytes: int) -> float:
+    return float(wl.L) * wl.H * wl.B * (wl.P * (wl.D * state_bytes + 4) + 2 * wl.D + 4)
+
+
+def plan_bytes(wl) -> float:
+    return float(wl.L) * wl.H * wl.B * wl.P * 4
+
+
+def dist_info():
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return world, rank, local
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Max of a per-rank scalar (the multi-rank timing rule); identity for one rank."""
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(units_per_rank: float, seconds_max: float, world: int) -> float:
+    """Whole-job throughput of `world` independent replicas: all ranks' units over the slowest rank's time."""
+    return units_per_rank * world / seconds_max
+
+
+# ------------------------------------------------------------------------------------------ oracle legs
+def oracle_sample(wl, q, k, v, mask, budget_s: float, seed: int = 0):
+    """Time the oracle, as it stands, on a bounded sample: one head, a seeded subset of query rows;
+    per row the COMPUTE pair states of its partition (Eq. 1) and the P-way merge (Eq. 2) -- REUSE
+    states are taken as already cached (zeros stand in; the arithmetic cost is the same).
+    Returns effective TFLOP/s (full-attention flops of the sampled rows / time), seconds, description."""
+    from oracle import oracle as orc
+    off = wl.offsets()
+    rng = np.random.default_rng(seed)
+    mask = mask.reshape(wl.P, wl.P)
+    qb, kb, vb = (inputs.bf16_bits(x[:, :, :1].contiguous()) for x in (q, k, v))   # head 0 only
+
+    def run(rows):
+        t0 = time.perf_counter()
+        part = np.searchsorted(off, rows, side="right") - 1
+        o_st = np.zeros((rows.size, wl.P, wl.D)); l_st = np.full((rows.size, wl.P), -30.0)
+        for i in range(wl.P):
+            sel = np.nonzero(part == i)[0]
+            if sel.size == 0:
+                continue
+            for j in range(wl.P):
+                if mask[i, j]:
+                    o, l = orc.pair_state(qb, kb, vb, wl.scale, 0, 0, rows[sel], int(off[j]), int(off[j + 1]))
+                    o_st[sel, j], l_st[sel, j] = o, l
+        orc.merge(o_st, l_st)
+        return time.perf_counter() - t0
+
+    n, t = min(256, wl.L), 0.0
+    while True:                                   # grow the sample until it costs about budget_s
+        rows = np.sort(rng.choice(wl.L, size=n, replace=False)).astype(np.int32)
+        t = run(rows)
+        if t >= 0.5 * budget_s or n == wl.L:
+            break
+        n = int(min(wl.L, max(2 * n, 0.9 * budget_s / max(t / n, 1e-9))))
+    eff = 4.0 * n * wl.L * wl.D / t / 1e12
+    desc = (f"fp64 oracle, head 0 of {wl.H}, {n} of {wl.L} query rows (seeded), COMPUTE pairs of the plan "
+            f"({int(mask.sum())}/{wl.P * wl.P}) + {wl.P}-way merge; value = 4*rows*L*D/time")
+    return eff, t, desc, orc.num_threads()
+
+
+def run_reference(args, wl):
+    world, rank, _ = dist_info()
+    if rank != 0:
+        return
+    gen = inputs.StepInputs(wl, seed=0, device="cpu")
+    q, k, v = gen.next()
+    f = wl.fractions[-1]
+    K = min(max(int(np.floor(f * wl.P * wl.P + 0.5)), wl.P), wl.P * wl.P)
+    # banded plan with the target pair count (the oracle leg needs no GPU-derived plan)
+    d = np.abs(np.subtract.outer(np.arange(wl.P), np.arange(wl.P)))
+    order = np.argsort(d.reshape(-1), kind="stable")
+    mask = np.zeros(wl.P * wl.P, np.uint8); mask[order[:K]] = 1
+    budget = 8.0
+    vals, secs = [], []
+    for s in range(args.warmup + args.steps):
+        eff, t, desc, cores = oracle_sample(wl, q, k, v, mask, budget, seed=s)
+        if s >= args.warmup:
+            vals.append(eff); secs.append(t)
+    value = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(secs)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "D": wl.D, "L": wl.L, "P": wl.P,
+                   "computed_pair_fraction": K / (wl.P * wl.P)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+def run_cuda(args, wl):
+    from paper_2607_15650_b200 import binding, build
+    world, rank, local = dist_info()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    build.build()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks = load_peaks()
+    state_dtype = binding.DT_STATE_BF16 if args.state_dtype == "bf16" else binding.DT_STATE_FP32
+    sbytes = 2 if args.state_dtype == "bf16" else 4
+
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale, state_dtype, local)
+    gen = inputs.StepInputs(wl, seed=0, device=dev)
+    steps_in = [gen.next() for _ in range(wl.steps)]          # resident bf16 inputs of every denoising step
+    del gen
+    torch.cuda.empty_cache()
+    out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    PP = wl.P * wl.P
+    masks = [torch.ones(PP, dtype=torch.uint8, device=dev), torch.ones(PP, dtype=torch.uint8, device=dev)]
+    ones = torch.ones(PP, dtype=torch.uint8, device=dev)
+    W = torch.empty(PP, dtype=torch.float64, device=dev)
+    frac = args.fraction if args.fraction is not None else wl.fractions[-1]
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def one_step(t, cur, timers=None):
+        """dt_attn_states with plan `cur` -> dt_state_merge -> dt_plan into the other mask buffer."""
+        q, k, v = steps_in[1 + (t % (wl.steps - 1))] if wl.steps > 1 else steps_in[0]
+        if timers is not None:
+            e = [ev() for _ in range(4)]
+            e[0].record(stream)
+        ctx.dt_attn_states(q, k, v, masks[cur], t)
+        if timers is not None:
+            e[1].record(stream)
+        ctx.dt_state_merge(out, lse)
+        if timers is not None:
+            e[2].record(stream)
+        ctx.dt_plan(masks[cur ^ 1], target_fraction=frac, w_dev=W)
+        if timers is not None:
+            e[3].record(stream)
+            timers.append(e)
+        return cur ^ 1
+
+    # anchor step: every pair computed, first plan derived from it
+    q, k, v = steps_in[0]
+    ctx.dt_attn_states(q, k, v, ones, 0)
+    ctx.dt_state_merge(out, lse)
+    ctx.dt_plan(masks[0], target_fraction=frac, w_dev=W)
+    torch.cuda.synchronize()
+    ctx.dt_poll()
+    cur = 0
+    t = 1
+    for _ in range(args.warmup):
+        cur = one_step(t, cur); t += 1
+    torch.cuda.synchronize()
+
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.dt_launch_count()
+    timers = []
+    torch.cuda.synchronize()
+    e0, e1 = ev(), ev()
+    e0.record(stream)
+    for _ in range(args.steps):
+        cur = one_step(t, cur, timers); t += 1
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    launches = ctx.dt_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ctx.dt_poll()
+    total_ms = e0.elapsed_time(e1)
+    total_ms = max_over_ranks(total_ms, world, dev)
+    ms_per_step = total_ms / args.steps
+    attn_ms = [e[0].elapsed_time(e[1]) for e in timers]
+    merge_ms = [e[1].elapsed_time(e[2]) for e in timers]
+    plan_ms = [e[2].elapsed_time(e[3]) for e in timers]
+    mask_np = masks[cur].cpu().numpy()
+    comp_fl = computed_flops(wl, mask_np)           # pair count is fixed by the target fraction
+    n_comp = int((mask_np != 0).sum())
+    value = aggregate_throughput(full_flops(wl) / 1e12, ms_per_step / 1e3, world)
+
+    if rank != 0:
+        return
+
+    # ---- all-compute plan on the same kernel (context for "ms/step vs full attention")
+    full_ms = []
+    for i in range(3 + 1):
+        a, b, c = ev(), ev(), ev()
+        q, k, v = steps_in[i % wl.steps]
+        a.record(stream)
+        ctx.dt_attn_states(q, k, v, ones, t)
+        b.record(stream)
+        ctx.dt_state_merge(out, lse)
+        c.record(stream)
+        torch.cuda.synchronize()
+        t += 1
+        if i > 0:
+            full_ms.append((a.elapsed_time(b), b.elapsed_time(c)))
+    full_attn_ms = float(np.mean([x[0] for x in full_ms]))
+    full_step_ms = float(np.mean([x[0] + x[1] for x in full_ms]))
+
+    # ---- end to end through the C ABI with host buffers (pinned): H2D of q, k, v, mask; D2H of out, lse
+    e2e = None
+    if not args.no_e2e:
+        cfg = ctx.cfg
+        ws = torch.empty(binding.dt_step_host_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+        qh, kh, vh = (x.cpu().pin_memory() for x in steps_in[1 % wl.steps])
+        oh = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+        lh = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+        mh = masks[cur].cpu()
+        times = []
+        for i in range(1 + 3):
+            t0 = time.perf_counter()
+            ctx.dt_step_host(qh, kh, vh, mh, t, oh, lh, ws)
+            times.append(time.perf_counter() - t0)
+            t += 1
+        e2e_s = float(np.mean(times[1:]))
+        h2d = 3 * qh.numel() * 2 + PP
+        d2h = oh.numel() * 2 + lh.numel() * 4
+        e2e = {"value": full_flops(wl) / 1e12 / e2e_s, "unit": UNIT, "ms_per_step": 1e3 * e2e_s,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "includes": "dt_step_host: H2D q,k,v,mask + dt_attn_states + dt_state_merge + D2H out,lse"}
+        del ws
+
+    # ---- CPU oracle on a bounded sample of the same workload
+    cpu = None
+    if not args.no_cpu_baseline:
+        eff, secs, desc, cores = oracle_sample(wl, *steps_in[1 % wl.steps], mask_np, budget_s=15.0)
+        cpu = {"value": eff, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds": secs}
+
+    attn_avg_ms = float(np.mean(attn_ms))
+    achieved = comp_fl / 1e12 / (attn_avg_ms / 1e3)
+    peak = peaks["bf16_tflops_sustained"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "D": wl.D, "L": wl.L, "P": wl.P,
+                   "computed_pairs": n_comp, "computed_pair_fraction": n_comp / PP, "state_dtype": args.state_dtype,
+                   "step": "dt_attn_states + dt_state_merge + dt_plan", "multi_gpu": "independent replicas",
+                   "l2": "inputs (%.1f GB) and state cache larger than L2; no flush" %
+                         ((3 * wl.L * wl.H * wl.D * 2) / 1e9)},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": launches,
+        "roofline": {"kernel": "attn_states_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
+                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                     "peak_source": f"{peaks['source']} bf16 sustained", "frac_of_burst": achieved / peaks["bf16_tflops"],
+                     "frac_of_nominal_2250": achieved / 2250.0, "launch_ms": attn_avg_ms,
+                     "algorithmic_flops_per_launch": comp_fl},
+        "cpu_baseline": cpu,
+        "kernels": {
+            "attn_ms": attn_avg_ms, "merge_ms": float(np.mean(merge_ms)), "plan_ms": float(np.mean(plan_ms)),
+            "merge_gbs": merge_bytes(wl, sbytes) / 1e9 / (float(np.mean(merge_ms)) / 1e3),
+            "merge_frac_of_hbm": merge_bytes(wl, sbytes) / 1e9 / (float(np.mean(merge_ms)) / 1e3) / peaks["hbm_gbs"],
+            "plan_gbs": plan_bytes(wl) / 1e9 / (float(np.mean(plan_ms)) / 1e3),
+            "hbm_peak_gbs": peaks["hbm_gbs"],
+        },
+        "vs_all_compute": {"all_compute_attn_ms": full_attn_ms, "all_compute_step_ms": full_step_ms,
+                           "all_compute_tflops": full_flops(wl) / 1e12 / (full_attn_ms / 1e3),
+                           "all_compute_frac_of_peak": full_flops(wl) / 1e12 / (full_attn_ms / 1e3) / peak,
+                           "step_time_ratio": ms_per_step / full_step_ms},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--fraction", type=float, default=None, help="target computed-pair fraction of the plan")
+    ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    wl = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_cuda(args, wl)
+
+
+if __name__ == "__main__":
+    main()
