@@ -400,11 +400,16 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--fraction", type=float, default=None, help="target computed-pair fraction of the plan")
     ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
+    ap.add_argument("--heads", type=int, default=None,
+                    help="override the head count (smaller captures under a profiler; not a bench configuration)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     wl = inputs.WORKLOADS[args.workload]
+    if args.heads is not None:
+        import dataclasses
+        wl = dataclasses.replace(wl, H=args.heads, name=f"{wl.name}_h{args.heads}")
     if args.impl == "reference":
         run_reference(args, wl)
     else:
