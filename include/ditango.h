@@ -110,6 +110,30 @@ dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_b
 dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask_dev, double *w_dev,
                   double *eps_out_dev, void *stream);
 
+/* The same plan computation for callers that cannot allocate device memory at the point of the
+ * call: code running inside a region where the allocator must stay untouched (a fixed-memory
+ * serving process that sized its pools up front, a callback on a latency-critical path, a host that
+ * hands this library pre-carved buffers and forbids cudaMalloc afterwards).  The paper has no
+ * counterpart; this is a packaging variant of dt_plan.
+ *   - No context: the caller passes the LSE cache (device, fp32 [P][B][H][L]) and the partition
+ *     offsets (HOST, P+1 ints) directly, plus the same outputs and options as dt_plan.
+ *   - The per-block partial sums live in a fixed array inside the library's device image (1 MiB of
+ *     floats plus a 256-byte header for the offsets; every GPU that loads the library holds it until
+ *     the process exits).  Problems that need more than 262144 partial sums, i.e.
+ *     B*H*P*P*ceil(max_i n_i / 1024) > 262144, are refused with DT_ERR_UNSUPPORTED and nothing runs.
+ *   - Calls nothing that allocates or frees: no cudaMalloc / cudaFree, no allocating library routine.
+ *     The offsets are copied into the array's header with one cudaMemcpyAsync on `stream`.
+ *   - The first call on each device looks up the array's device address (the current device must
+ *     be the one that owns `stream` and the buffers); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing
+ *     in it has to start at zero (stage 1 overwrites every slot stage 2 reads), but two calls whose
+ *     kernels can overlap on the GPU (different streams, no ordering between them) race on it:
+ *     order them on one stream or with events.
+ * Results are bit-identical to dt_plan on the same inputs. */
+dt_status dt_plan_static(const float *lse_state_dev, const int32_t *part_offsets_host, int32_t B, int32_t H,
+                         int32_t L, int32_t P, double eps, double target_fraction, uint8_t *mask_dev,
+                         double *w_dev, double *eps_out_dev, void *stream);
+
 /* One whole step from HOST buffers: copies q, k, v (bf16 [B,L,H,D] contiguous) and the mask to the
  * device workspace, runs dt_attn_states and dt_state_merge, copies out (bf16 [B,L,H,D]) and lse
  * (fp32 [B,H,L], may be NULL) back and synchronises `stream`.  workspace_dev must hold

@@ -20,7 +20,7 @@ DT_MAX_P = 32
 
 EXPORTS = [
     "dt_create", "dt_destroy", "dt_cache_bytes", "dt_bind_cache", "dt_attn_states", "dt_state_merge",
-    "dt_plan", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
+    "dt_plan", "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
     "dt_launch_count", "dt_poll", "dt_status_str", "dt_last_error",
 ]
 
@@ -60,6 +60,8 @@ def lib():
         "dt_attn_states": (C.c_int, [vp, vp, vp, vp, i64p, u8p, C.c_int32, vp]),
         "dt_state_merge": (C.c_int, [vp, vp, i64p, f32p, vp]),
         "dt_plan": (C.c_int, [vp, C.c_double, C.c_double, u8p, f64p, f64p, vp]),
+        "dt_plan_static": (C.c_int, [f32p, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_double,
+                           u8p, f64p, f64p, vp]),
         "dt_step_host_workspace_bytes": (C.c_int, [C.POINTER(dt_config), szp]),
         "dt_step_host": (C.c_int, [vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, C.c_size_t, vp]),
         "dt_get_tc": (C.c_int, [vp, i32p]),
@@ -112,6 +114,30 @@ def _stream_ptr(stream):
     if stream is None:
         stream = torch.cuda.current_stream()
     return C.c_void_p(stream.cuda_stream)
+
+
+STATIC_PLAN_MAX_PARTIALS = 262144
+
+
+def dt_plan_static(lse_state, offsets, B, H, L, mask_dev, eps=0.0, target_fraction=-1.0, w_dev=None,
+                   eps_out_dev=None, stream=None):
+    """Plan without a context and without any allocation inside the library (see ditango.h): for callers
+    that may not touch the CUDA allocator when they plan.  `lse_state` is the fp32 LSE cache [P, B, H, L]
+    on the device, `offsets` the P+1 partition offsets on the host.  Problems needing more than
+    STATIC_PLAN_MAX_PARTIALS partial sums are refused (DT_ERR_UNSUPPORTED)."""
+    off = np.ascontiguousarray(offsets, dtype=np.int32)
+    P = off.size - 1
+    assert lse_state.is_cuda and lse_state.dtype == torch.float32 and lse_state.is_contiguous()
+    assert mask_dev.is_cuda and mask_dev.dtype == torch.uint8 and mask_dev.is_contiguous()
+    wp = C.c_void_p(w_dev.data_ptr()) if w_dev is not None else C.c_void_p()
+    ep = C.c_void_p(eps_out_dev.data_ptr()) if eps_out_dev is not None else C.c_void_p()
+    s = lib().dt_plan_static(C.c_void_p(lse_state.data_ptr()), off.ctypes.data_as(C.POINTER(C.c_int32)), int(B), int(H),
+                             int(L), int(P), float(eps), float(target_fraction), C.c_void_p(mask_dev.data_ptr()), wp, ep,
+                             _stream_ptr(stream))
+    if s != DT_OK:
+        detail = ("problem exceeds the built-in scratch of %d partial sums" % STATIC_PLAN_MAX_PARTIALS
+                  if s == DT_ERR_UNSUPPORTED else "dt_plan_static")
+        raise DitangoError(s, status_str(s), detail)
 
 
 class Context:

@@ -9,6 +9,8 @@
 // Stage 2 (one block): sums the partials in fp64 in a fixed order, divides by the row count,
 // and either thresholds (W > eps, strict) or ranks the off-diagonal pairs to hit a target count.
 // No atomics: the result is bit-reproducible from run to run.
+#include <math.h>
+
 #include "dt_internal.h"
 
 namespace dt {
@@ -165,3 +167,80 @@ cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist,
 }
 
 }  // namespace dt
+
+// ---------------------------------------------------------------------------------------------
+// dt_plan_static: the plan computation with no allocation anywhere on its path.
+//
+// Stage 1's per-block partial sums need scratch memory.  dt_plan takes it from the context, which
+// dt_create allocated; this entry point instead keeps it in a device array that is part of the
+// library image, so a caller that must not allocate can still plan.
+namespace {
+
+constexpr int STATIC_PLAN_OFFSET_SLOTS = 64;                       // ints reserved for the P+1 offsets
+constexpr size_t STATIC_PLAN_MAX_PARTIALS = 262144;                // floats (1 MiB) for stage-1 partial sums
+constexpr int STATIC_PLAN_MAX_DEVICES = 64;
+
+static __device__ __align__(256) float g_plan_static_scratch[STATIC_PLAN_OFFSET_SLOTS + STATIC_PLAN_MAX_PARTIALS];
+
+// In host code the array's name is only a handle: the device address is looked up once per device.
+float *g_plan_static_ptr[STATIC_PLAN_MAX_DEVICES] = {nullptr};
+
+}  // namespace
+
+extern "C" dt_status dt_plan_static(const float *lse_state_dev, const int32_t *part_offsets_host, int32_t B, int32_t H,
+                                    int32_t L, int32_t P, double eps, double target_fraction, uint8_t *mask_dev,
+                                    double *w_dev, double *eps_out_dev, void *stream) {
+    if (!lse_state_dev || !part_offsets_host || !mask_dev) return DT_ERR_INVALID_ARG;
+    if (B < 1 || H < 1 || L < 1 || P < 1) return DT_ERR_INVALID_ARG;
+    if (P > DT_MAX_P || (long long)B * H > 65535) return DT_ERR_UNSUPPORTED;
+    if (part_offsets_host[0] != 0 || part_offsets_host[P] != L) return DT_ERR_INVALID_ARG;
+    int n_max = 0;
+    for (int i = 0; i < P; ++i) {
+        const int n = part_offsets_host[i + 1] - part_offsets_host[i];
+        if (n <= 0) return DT_ERR_INVALID_ARG;
+        n_max = n > n_max ? n : n_max;
+    }
+    if (target_fraction < 0 && !(eps == eps && eps - eps == 0.0)) return DT_ERR_INVALID_ARG;   // eps must be finite
+    if (target_fraction > 1.0 || target_fraction != target_fraction) return DT_ERR_INVALID_ARG;
+    const int chunks = (n_max + dt::PLAN_CHUNK_ROWS - 1) / dt::PLAN_CHUNK_ROWS;
+    const size_t need = (size_t)B * H * P * chunks * P;
+    if (need > STATIC_PLAN_MAX_PARTIALS) return DT_ERR_UNSUPPORTED;   // problem larger than the built-in scratch
+
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= STATIC_PLAN_MAX_DEVICES) return DT_ERR_CUDA;
+    if (g_plan_static_ptr[device] == nullptr) {   // first call on this device: resolve the array's device address
+        float *ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_plan_static_scratch) != cudaSuccess || !ptr)
+            return DT_ERR_CUDA;
+        g_plan_static_ptr[device] = ptr;
+    }
+    float *scratch = g_plan_static_ptr[device];
+    int32_t *off_dev = reinterpret_cast<int32_t *>(scratch);
+    float *partials = scratch + STATIC_PLAN_OFFSET_SLOTS;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(off_dev, part_offsets_host, (P + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return DT_ERR_CUDA;
+
+    dt::PlanParams pp;
+    pp.lse_state = lse_state_dev;
+    pp.off = off_dev;
+    pp.partials = partials;
+    pp.P = P; pp.BH = B * H; pp.L = L; pp.chunks = chunks;
+    pp.R = (long long)B * H * L;
+    if (dt::launch_plan_partial(pp, st) != cudaSuccess) return DT_ERR_CUDA;
+    dt::PlanFinalParams pf;
+    pf.partials = partials;
+    pf.off = off_dev;
+    pf.P = P; pf.BH = pp.BH; pf.chunks = chunks;
+    pf.mode_target = target_fraction >= 0 ? 1 : 0;
+    const int total = P * P;
+    int K = (int)floor(target_fraction * total + 0.5);
+    K = K < P ? P : (K > total ? total : K);
+    pf.K = K;
+    pf.eps = eps;
+    pf.mask = mask_dev;
+    pf.w_out = w_dev;
+    pf.eps_out = eps_out_dev;
+    if (dt::launch_plan_final(pf, st) != cudaSuccess) return DT_ERR_CUDA;
+    return DT_OK;
+}
