@@ -6,10 +6,11 @@
 // One persistent CTA per SM walks the work list (b*h slowest, then COMPUTE pair, then query
 // block), so CTAs running at the same time share one head's K/V partition through L2.
 //
-// Per CTA (10 warps):
+// Per CTA (12 warps; the producer warpgroup gives registers to the softmax warpgroups):
 //   warps 0-3 / 4-7  softmax warpgroups for query tile 0 / 1 (128 rows each, one row per thread)
 //   warp 8           TMA producer: Q tiles once per work item, K and V tiles through a ring
 //   warp 9           MMA issuer (one elected lane): tcgen05.mma into TMEM
+//   warps 10-11      idle (they complete the producer warpgroup for the register hand-over)
 // TMEM (512 columns): S0 | S1 | O0 | O1.  S_t = Q K_t^T (fp32) lands in S; the softmax warpgroup
 // reads its row, writes P = exp2(s*scale*log2e - m) back over S as packed bf16, and the PV MMA
 // takes P from TMEM as its A operand and V from shared memory (MN-major) as B, accumulating in O.
@@ -30,7 +31,8 @@ namespace {
 constexpr int NUM_SOFTMAX_THREADS = ATTN_NQ * 128;
 constexpr int TMA_WARP = NUM_SOFTMAX_THREADS / 32;
 constexpr int MMA_WARP = TMA_WARP + 1;
-constexpr int ATTN_THREADS = NUM_SOFTMAX_THREADS + 64;
+constexpr int ATTN_THREADS = NUM_SOFTMAX_THREADS + 128;  // producer warpgroup: TMA, MMA and two idle warps
+constexpr int REGS_SOFTMAX = 224, REGS_PRODUCER = 56;   // per-thread register budgets after the role split
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
 
@@ -165,7 +167,9 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     const int npairs = p.worklist[0];
     const long long total_work = (long long)npairs * p.qblocks_max * p.B * p.H;
 
-    if (warp == TMA_WARP) {
+    if (warp >= TMA_WARP) {
+      reg_dealloc<REGS_PRODUCER>();
+      if (warp == TMA_WARP) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&tmap_q);
@@ -209,7 +213,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         }
-    } else if (warp == MMA_WARP) {
+      } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t IDESC_QK = make_idesc_bf16_f32(128, ATTN_TILE, false);
@@ -303,7 +307,9 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 *abort_ptr = 1;
             }
         }
+      }
     } else {
+        reg_alloc<REGS_SOFTMAX>();
         // ------------------------------------------------------------ softmax warpgroups
         const int q = warp / 4;                       // query tile handled by this warpgroup
         const int row_in_tile = (warp % 4) * 32 + lane;
@@ -335,9 +341,16 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     for (int c = 0; c < 128; ++c)
                         if (c >= valid) s[c >> 5][c & 31] = 0xFF800000u;  // -inf
                 }
-                float mx = -INFINITY;
+                // row maximum: four independent chains of three-input max
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(s[c >> 5][c & 31]));
+                for (int c = 0; c < 128; c += 8) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        mx4[u] = fmax3(mx4[u], __uint_as_float(s[(c + 2 * u) >> 5][(c + 2 * u) & 31]),
+                                       __uint_as_float(s[(c + 2 * u + 1) >> 5][(c + 2 * u + 1) & 31]));
+                }
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 const float m_new = fmaxf(m_used, mx * p.scale_log2);
                 // move the reference maximum only when it grew by more than 2^RESCALE_THRESHOLD
                 const bool need = (m_new - m_used > RESCALE_THRESHOLD);   // true on the first tile (m_used = -inf)
@@ -357,19 +370,25 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         tmem_st_x32(o_tmem + c0, o);
                     }
                 }
-                const float neg_m = -m_used;
-                float rs = 0.f;
+                // P = exp2(s * scale_log2 - m): packed two-wide FMA and add, four independent sum chains
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+                const float2 nm2 = make_float2(-m_used, -m_used);
+                float2 rs4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 uint32_t pk[2][32];  // P row as packed bf16 pairs (key 2c in the low half)
 #pragma unroll
-                for (int c = 0; c < 128; c += 2) {
-                    const float p0 = ex2_approx(fmaf(__uint_as_float(s[c >> 5][c & 31]), p.scale_log2, neg_m));
-                    const float p1 = ex2_approx(fmaf(__uint_as_float(s[(c + 1) >> 5][(c + 1) & 31]), p.scale_log2, neg_m));
-                    rs += p0 + p1;
-                    pk[c >> 6][(c >> 1) & 31] = pack_bf16x2(p0, p1);
+                for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                    for (int c = half * 64; c < half * 64 + 64; c += 2) {
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[c >> 5][c & 31]),
+                                                                __uint_as_float(s[(c + 1) >> 5][(c + 1) & 31])), sc2, nm2);
+                        const float2 pp = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                        rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
+                        pk[half][(c >> 1) & 31] = pack_bf16x2(pp.x, pp.y);
+                    }
+                    tmem_st_x32(s_tmem + 32 * half, pk[half]);
                 }
-                l_sum += rs;
-                tmem_st_x32(s_tmem + 0, pk[0]);
-                tmem_st_x32(s_tmem + 32, pk[1]);
+                const float2 rs2 = __fadd2_rn(__fadd2_rn(rs4[0], rs4[1]), __fadd2_rn(rs4[2], rs4[3]));
+                l_sum += rs2.x + rs2.y;
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bars.p_full + 8 * q);
