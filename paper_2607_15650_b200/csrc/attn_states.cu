@@ -32,8 +32,12 @@ constexpr int NUM_SOFTMAX_THREADS = ATTN_NQ * 128;
 constexpr int TMA_WARP = NUM_SOFTMAX_THREADS / 32;
 constexpr int MMA_WARP = TMA_WARP + 1;
 constexpr int ATTN_THREADS = NUM_SOFTMAX_THREADS + 128;  // producer warpgroup: TMA, MMA and two idle warps
-constexpr int REGS_SOFTMAX = 224, REGS_PRODUCER = 56;   // per-thread register budgets after the role split
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s
+// Per-thread register budgets after the role split.  Each SM sub-partition holds 16384 registers and
+// three of this kernel's warps (two softmax, one producer); (2 * 208 + 88) * 32 = 16128 leaves 256
+// spare.  A split that needs every register never gets them: setmaxnreg.inc then blocks forever.
+constexpr int REGS_SOFTMAX = 208, REGS_PRODUCER = 88;
+static_assert((2 * REGS_SOFTMAX + REGS_PRODUCER) * 32 <= 16384 - 256, "register split leaves no slack");
+constexpr long long WAIT_LIMIT_NS = 4000000000ll;   // SM clock cycles: about 2 s
 constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
 
 template <int D>
@@ -55,6 +59,20 @@ struct Bars {
     uint32_t q_full, q_empty;
     uint32_t kv_full, kv_empty;   // + 8*stage
     uint32_t s_full, p_full, o_full, o_free;  // + 8*q
+};
+
+// Position in the K/V ring: stage index and the parity of its current use.
+template <int STAGES>
+struct RingPos {
+    uint32_t st = 0, ph = 0;
+    __device__ __forceinline__ void advance() {
+        if (++st == STAGES) { st = 0; ph ^= 1u; }
+    }
+    __device__ __forceinline__ RingPos next() const {
+        RingPos r = *this;
+        r.advance();
+        return r;
+    }
 };
 
 struct WorkItem {
@@ -175,7 +193,8 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             prefetch_tensormap(&tmap_q);
             prefetch_tensormap(&tmap_k);
             prefetch_tensormap(&tmap_v);
-            uint32_t q_phase = 0, kv_it = 0;
+            uint32_t q_phase = 0;
+            RingPos<C::STAGES> ring;
             bool ok = true;
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
@@ -193,7 +212,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 for (int t = 0; t < it.tiles && ok; ++t) {
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
-                        const uint32_t st = kv_it % C::STAGES, ph = (kv_it / C::STAGES) & 1u;
+                        const uint32_t st = ring.st, ph = ring.ph;
                         ok = mbar_wait_bounded(bars.kv_empty + 8 * st, ph ^ 1u, abort_ptr, WAIT_LIMIT_NS);
                         if (!ok) break;
                         mbar_arrive_expect_tx(bars.kv_full + 8 * st, C::TILE_BYTES);
@@ -201,7 +220,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         for (int hf = 0; hf < C::NHALF; ++hf)
                             tma_load_4d(kv_smem + st * C::TILE_BYTES + hf * C::HALF_BYTES, kv == 0 ? &tmap_k : &tmap_v,
                                         bars.kv_full + 8 * st, hf * 64, it.h, it.kv_row0 + t * ATTN_TILE, it.b);
-                        ++kv_it;
+                        ring.advance();
                     }
                 }
             }
@@ -218,28 +237,33 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         if (lane == 0) {
             constexpr uint32_t IDESC_QK = make_idesc_bf16_f32(128, ATTN_TILE, false);
             constexpr uint32_t IDESC_PV = make_idesc_bf16_f32(128, D, true);
-            uint32_t q_phase = 0, kv_it = 0, p_phase = 0, of_phase = 0;
+            uint32_t q_phase = 0, p_phase = 0, of_phase = 0;
+            RingPos<C::STAGES> ring;
             bool ok = true;
 
+            // Descriptors differ only in their 14-bit start-address field (units of 16 bytes), so each
+            // operand's descriptor is its base plus a small constant.
+            const uint64_t qdesc0 = make_smem_desc_sw128(q_smem, 16, 1024);
+            const uint64_t kdesc0 = make_smem_desc_sw128(kv_smem, 16, 1024);
+            const uint64_t vdesc0 = make_smem_desc_sw128(kv_smem, C::HALF_BYTES, 1024);
             // S[q] = Q[q] K^T for the K tile in ring stage `st`
             auto issue_qk = [&](int q, uint32_t st) {
+                const uint64_t a0 = qdesc0 + (uint64_t)((q * C::TILE_BYTES) >> 4);
+                const uint64_t b0 = kdesc0 + (uint64_t)((st * C::TILE_BYTES) >> 4);
+                const uint32_t d = tmem_base + C::S_COL + q * 128;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t koff = (kk / 4) * C::HALF_BYTES + (kk % 4) * 32;
-                    const uint64_t a = make_smem_desc_sw128(q_smem + q * C::TILE_BYTES + koff, 16, 1024);
-                    const uint64_t b = make_smem_desc_sw128(kv_smem + st * C::TILE_BYTES + koff, 16, 1024);
-                    mma_ss(tmem_base + C::S_COL + q * 128, a, b, IDESC_QK, kk > 0 ? 1u : 0u);
+                    const uint32_t koff = ((kk / 4) * C::HALF_BYTES + (kk % 4) * 32) >> 4;
+                    mma_ss(d, a0 + koff, b0 + koff, IDESC_QK, kk > 0 ? 1u : 0u);
                 }
             };
             // O[q] (+)= P[q] V for the V tile in ring stage `st`
             auto issue_pv = [&](int q, uint32_t st, bool accumulate) {
+                const uint64_t b0 = vdesc0 + (uint64_t)((st * C::TILE_BYTES) >> 4);
+                const uint32_t d = tmem_base + C::O_COL + q * D, a = tmem_base + C::S_COL + q * 128;
 #pragma unroll
-                for (int kk = 0; kk < ATTN_TILE / 16; ++kk) {
-                    const uint64_t b =
-                        make_smem_desc_sw128(kv_smem + st * C::TILE_BYTES + kk * 2048, C::HALF_BYTES, 1024);
-                    mma_ts(tmem_base + C::O_COL + q * D, tmem_base + C::S_COL + q * 128 + kk * 8, b, IDESC_PV,
-                           (accumulate || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < ATTN_TILE / 16; ++kk)
+                    mma_ts(d, a + kk * 8, b0 + (uint64_t)((kk * 2048) >> 4), IDESC_PV, (accumulate || kk > 0) ? 1u : 0u);
             };
 
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
@@ -250,7 +274,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 q_phase ^= 1u;
                 // first K tile
                 {
-                    const uint32_t st = kv_it % C::STAGES, ph = (kv_it / C::STAGES) & 1u;
+                    const uint32_t st = ring.st, ph = ring.ph;
                     ok = mbar_wait_bounded(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
                     if (!ok) break;
                     tc_fence_after();
@@ -261,14 +285,16 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     }
                     tc_commit(bars.kv_empty + 8 * st);
                     if (it.tiles == 1) tc_commit(bars.q_empty);
-                    ++kv_it;
+                    ring.advance();
                 }
+                // Steady state.  This thread only waits on p_full: softmax warp 0 checks that V_t and
+                // K_{t+1} have landed before it arrives there, so one wait covers both (every wait here
+                // drains the queue of issued MMAs, and the tensor pipe idles until new ones arrive).
                 for (int t = 0; t < it.tiles && ok; ++t) {
-                    const uint32_t st_v = kv_it % C::STAGES, ph_v = (kv_it / C::STAGES) & 1u;
-                    const uint32_t st_k = (kv_it + 1) % C::STAGES, ph_k = ((kv_it + 1) / C::STAGES) & 1u;
+                    const uint32_t st_v = ring.st;
+                    ring.advance();
+                    const uint32_t st_k = ring.st;
                     const bool more = (t + 1 < it.tiles);
-                    ok = mbar_wait_bounded(bars.kv_full + 8 * st_v, ph_v, abort_ptr, WAIT_LIMIT_NS);
-                    if (!ok) break;
 #pragma unroll
                     for (int q = 0; q < ATTN_NQ; ++q) {
                         ok = mbar_wait_bounded(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_NS);
@@ -279,23 +305,18 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         }
                         tc_fence_after();
                         issue_pv(q, st_v, t > 0);
-                        if (!more) tc_commit(bars.o_full + 8 * q);
                         if (more) {
-                            if (q == 0) {
-                                ok = mbar_wait_bounded(bars.kv_full + 8 * st_k, ph_k, abort_ptr, WAIT_LIMIT_NS);
-                                if (!ok) break;
-                                tc_fence_after();
-                            }
                             issue_qk(q, st_k);
                             tc_commit(bars.s_full + 8 * q);
+                        } else {
+                            tc_commit(bars.o_full + 8 * q);
                         }
                     }
                     if (!ok) break;
                     tc_commit(bars.kv_empty + 8 * st_v);
-                    ++kv_it;
                     if (more) {
                         tc_commit(bars.kv_empty + 8 * st_k);
-                        ++kv_it;
+                        ring.advance();
                         if (t + 2 == it.tiles) tc_commit(bars.q_empty);
                     }
                     p_phase ^= 1u;
@@ -318,12 +339,14 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const uint32_t o_tmem = tmem_base + lane_addr + C::O_COL + q * D;
         uint32_t s_phase = 0, o_phase = 0;
         bool ok = true;
+        RingPos<C::STAGES> ring;   // used by warp 0 only: it vouches for K/V arrival on behalf of the MMA thread
         StateT *o_state = static_cast<StateT *>(p.o_state);
 
         for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             WorkItem it;
             if (!decode_work(p, npairs, w, it)) continue;
             float m_used = -INFINITY, l_sum = 0.f;
+            ring.advance();   // K_0 of the item: the MMA thread waits for that one itself
             for (int t = 0; t < it.tiles; ++t) {
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.s_full + 8 * q, s_phase, abort_ptr, WAIT_LIMIT_NS));
                 if (!ok) break;
@@ -390,6 +413,16 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 const float2 rs2 = __fadd2_rn(__fadd2_rn(rs4[0], rs4[1]), __fadd2_rn(rs4[2], rs4[3]));
                 l_sum += rs2.x + rs2.y;
                 tmem_wait_st();
+                if (warp == 0) {   // V_t and K_{t+1} must be in shared memory before P_t is announced
+                    ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
+                    ring.advance();
+                    if (ok && t + 1 < it.tiles) {
+                        ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
+                        ring.advance();
+                    }
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                }
                 tc_fence_before();
                 mbar_arrive(bars.p_full + 8 * q);
             }

@@ -47,19 +47,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: gives up after `limit_ns` of wall time or as soon as *abort_flag is set.
+// Bounded wait: gives up after `limit_cycles` SM clock cycles or as soon as *abort_flag is set.
 // Returns false on give-up (the caller records the status and leaves its loop normally).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                                  uint64_t limit_ns) {
+                                                  long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
-    uint64_t t0 = global_timer_ns();
-    uint32_t n = 0;
-    while (true) {
+    const long long t0 = clock64();
+#pragma unroll 1
+    for (uint32_t n = 1;; ++n) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (((++n) & 0xFFu) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > limit_ns) return false;
-        }
+        if ((n & 0xFFu) == 0u && (*abort_flag || clock64() - t0 > limit_cycles)) return false;
     }
 }
 
