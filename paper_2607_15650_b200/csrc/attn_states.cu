@@ -10,7 +10,8 @@
 //   warps 0-3 / 4-7  softmax warpgroups for query tile 0 / 1 (128 rows each, one row per thread)
 //   warp 8           TMA producer: Q tiles once per work item, K and V tiles through a ring
 //   warp 9           MMA issuer (one elected lane): tcgen05.mma into TMEM
-//   warps 10-11      idle (they complete the producer warpgroup for the register hand-over)
+//   warp 10          K/V watcher: adds its arrival to p_full[0] once V_t and K_{t+1} have landed
+//   warp 11          idle (completes the producer warpgroup for the register hand-over)
 // TMEM (512 columns): S0 | S1 | O0 | O1.  S_t = Q K_t^T (fp32) lands in S; the softmax warpgroup
 // reads its row, writes P = exp2(s*scale*log2e - m) back over S as packed bf16, and the PV MMA
 // takes P from TMEM as its A operand and V from shared memory (MN-major) as B, accumulating in O.
@@ -31,12 +32,17 @@ namespace {
 constexpr int NUM_SOFTMAX_THREADS = ATTN_NQ * 128;
 constexpr int TMA_WARP = NUM_SOFTMAX_THREADS / 32;
 constexpr int MMA_WARP = TMA_WARP + 1;
+constexpr int WATCH_WARP = TMA_WARP + 2;   // vouches for K/V arrival on behalf of the MMA thread
 constexpr int ATTN_THREADS = NUM_SOFTMAX_THREADS + 128;  // producer warpgroup: TMA, MMA and two idle warps
-// Per-thread register budgets after the role split.  Each SM sub-partition holds 16384 registers and
-// three of this kernel's warps (two softmax, one producer); (2 * 208 + 88) * 32 = 16128 leaves 256
-// spare.  A split that needs every register never gets them: setmaxnreg.inc then blocks forever.
-constexpr int REGS_SOFTMAX = 208, REGS_PRODUCER = 88;
-static_assert((2 * REGS_SOFTMAX + REGS_PRODUCER) * 32 <= 16384 - 256, "register split leaves no slack");
+// Per-thread register budgets after the role split.  setmaxnreg.inc can only take registers that a
+// setmaxnreg.dec of the same CTA has released (registers the launch left unallocated do not count);
+// a request beyond that blocks forever.  So with LAUNCH_REGS registers per thread at launch:
+//   (REGS_SOFTMAX - LAUNCH_REGS) * softmax threads  <=  (LAUNCH_REGS - REGS_PRODUCER) * 128.
+// LAUNCH_REGS is what ptxas assigns under __launch_bounds__(384, 1); attn_states_configure() checks it
+// against the compiled kernels and refuses to run on a mismatch.
+constexpr int LAUNCH_REGS = 168, REGS_SOFTMAX = 208, REGS_PRODUCER = 88;
+static_assert((REGS_SOFTMAX - LAUNCH_REGS) * NUM_SOFTMAX_THREADS <= (LAUNCH_REGS - REGS_PRODUCER) * 128,
+              "softmax warps would wait forever for registers nobody releases");
 constexpr long long WAIT_LIMIT_NS = 4000000000ll;   // SM clock cycles: about 2 s
 constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
 
@@ -167,7 +173,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         }
         for (int q = 0; q < ATTN_NQ; ++q) {
             mbar_init(bars.s_full + 8 * q, 1);
-            mbar_init(bars.p_full + 8 * q, 128);
+            mbar_init(bars.p_full + 8 * q, 128 + (q == 0 ? 1 : 0));   // tile 0: + the K/V watcher
             mbar_init(bars.o_full + 8 * q, 1);
             mbar_init(bars.o_free + 8 * q, 128);
         }
@@ -328,6 +334,37 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 *abort_ptr = 1;
             }
         }
+      } else if (warp == WATCH_WARP) {
+        // ------------------------------------------------------------ K/V watcher
+        // One more arrival on p_full[0] per tile, made once V_t and K_{t+1} are in shared memory: the
+        // MMA thread's single wait then covers P_t and both tiles without a poll of its own.
+        if (lane == 0) {
+            RingPos<C::STAGES> ring;
+            uint32_t p_phase = 0;
+            bool ok = true;
+            for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+                WorkItem it;
+                if (!decode_work(p, npairs, w, it)) continue;
+                ring.advance();   // K_0 of the item: the MMA thread waits for that one itself
+                for (int t = 0; t < it.tiles && ok; ++t) {
+                    ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
+                    ring.advance();
+                    if (ok && t + 1 < it.tiles) {
+                        ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
+                        ring.advance();
+                    }
+                    if (ok) {   // one arrival per phase: wait for the phase to close before the next one
+                        mbar_arrive(bars.p_full);
+                        ok = mbar_wait_bounded(bars.p_full, p_phase, abort_ptr, WAIT_LIMIT_NS);
+                        p_phase ^= 1u;
+                    }
+                }
+            }
+            if (!ok) {
+                if (!*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
+                *abort_ptr = 1;
+            }
+        }
       }
     } else {
         reg_alloc<REGS_SOFTMAX>();
@@ -339,14 +376,12 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const uint32_t o_tmem = tmem_base + lane_addr + C::O_COL + q * D;
         uint32_t s_phase = 0, o_phase = 0;
         bool ok = true;
-        RingPos<C::STAGES> ring;   // used by warp 0 only: it vouches for K/V arrival on behalf of the MMA thread
         StateT *o_state = static_cast<StateT *>(p.o_state);
 
         for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             WorkItem it;
             if (!decode_work(p, npairs, w, it)) continue;
             float m_used = -INFINITY, l_sum = 0.f;
-            ring.advance();   // K_0 of the item: the MMA thread waits for that one itself
             for (int t = 0; t < it.tiles; ++t) {
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.s_full + 8 * q, s_phase, abort_ptr, WAIT_LIMIT_NS));
                 if (!ok) break;
@@ -413,16 +448,6 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 const float2 rs2 = __fadd2_rn(__fadd2_rn(rs4[0], rs4[1]), __fadd2_rn(rs4[2], rs4[3]));
                 l_sum += rs2.x + rs2.y;
                 tmem_wait_st();
-                if (warp == 0) {   // V_t and K_{t+1} must be in shared memory before P_t is announced
-                    ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
-                    ring.advance();
-                    if (ok && t + 1 < it.tiles) {
-                        ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
-                        ring.advance();
-                    }
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
-                }
                 tc_fence_before();
                 mbar_arrive(bars.p_full + 8 * q);
             }
@@ -470,6 +495,10 @@ cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorM
 
 template <int D, typename StateT>
 cudaError_t configure() {
+    cudaFuncAttributes attr;
+    cudaError_t e = cudaFuncGetAttributes(&attr, attn_states_kernel<D, StateT>);
+    if (e != cudaSuccess) return e;
+    if (attr.numRegs != LAUNCH_REGS) return cudaErrorInvalidConfiguration;   // the register hand-over would not balance
     return cudaFuncSetAttribute(attn_states_kernel<D, StateT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 Cfg<D>::SMEM_BYTES);
 }
