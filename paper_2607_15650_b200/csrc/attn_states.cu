@@ -45,6 +45,10 @@ static_assert((REGS_SOFTMAX - LAUNCH_REGS) * NUM_SOFTMAX_THREADS <= (LAUNCH_REGS
               "softmax warps would wait forever for registers nobody releases");
 constexpr long long WAIT_LIMIT_NS = 4000000000ll;   // SM clock cycles: about 2 s
 constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
+#ifndef DT_POLY_PER_8
+#define DT_POLY_PER_8 0
+#endif
+constexpr int POLY_PER_8 = DT_POLY_PER_8;           // key pairs (of every 8) whose exp2 runs on the FMA pipe
 
 template <int D>
 struct Cfg {
@@ -399,54 +403,70 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     for (int c = 0; c < 128; ++c)
                         if (c >= valid) s[c >> 5][c & 31] = 0xFF800000u;  // -inf
                 }
-                // row maximum: four independent chains of three-input max
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                if (t == 0) {   // first tile of the item: there is no earlier maximum to lean on
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int c = 0; c < 128; c += 8) {
+                    for (int c = 0; c < 128; c += 8) {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        mx4[u] = fmax3(mx4[u], __uint_as_float(s[(c + 2 * u) >> 5][(c + 2 * u) & 31]),
-                                       __uint_as_float(s[(c + 2 * u + 1) >> 5][(c + 2 * u + 1) & 31]));
-                }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                const float m_new = fmaxf(m_used, mx * p.scale_log2);
-                // move the reference maximum only when it grew by more than 2^RESCALE_THRESHOLD
-                const bool need = (m_new - m_used > RESCALE_THRESHOLD);   // true on the first tile (m_used = -inf)
-                if (t == 0) {
-                    m_used = m_new;
-                } else if (__any_sync(0xFFFFFFFFu, need)) {
-                    const float alpha = need ? ex2_approx(m_used - m_new) : 1.0f;
-                    if (need) m_used = m_new;
-                    l_sum *= alpha;
-#pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += 32) {
-                        uint32_t o[32];
-                        tmem_ld_x32(o_tmem + c0, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                        tmem_st_x32(o_tmem + c0, o);
+                        for (int u = 0; u < 4; ++u)
+                            mx4[u] = fmax3(mx4[u], __uint_as_float(s[(c + 2 * u) >> 5][(c + 2 * u) & 31]),
+                                           __uint_as_float(s[(c + 2 * u + 1) >> 5][(c + 2 * u + 1) & 31]));
                     }
+                    m_used = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
                 }
-                // P = exp2(s * scale_log2 - m): packed two-wide FMA and add, four independent sum chains
+                // P = exp2(s * scale_log2 - m_used) with the reference maximum of the earlier tiles; this
+                // tile's own maximum is gathered in the shadow of the exponentials (the MUFU is the busy
+                // unit here).  Only if it exceeds m_used by more than 2^RESCALE_THRESHOLD are m_used, O and
+                // l moved and P computed again -- rare after the first tiles; the result does not depend
+                // on which reference is used, since it cancels in OUT = O / l and LSE = m + log l.
                 const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-                const float2 nm2 = make_float2(-m_used, -m_used);
-                float2 rs4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                uint32_t pk[2][32];  // P row as packed bf16 pairs (key 2c in the low half)
+                // one pass over the row: P to TMEM, returns the row sum; optionally the raw row maximum
+                auto exp_pass = [&](float m_ref, float &mx_out) -> float {
+                    const float2 nm2 = make_float2(-m_ref, -m_ref);
+                    float2 rs4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t pk[32];  // 64 keys as packed bf16 pairs (even key in the low half)
 #pragma unroll
-                    for (int c = half * 64; c < half * 64 + 64; c += 2) {
-                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[c >> 5][c & 31]),
-                                                                __uint_as_float(s[(c + 1) >> 5][(c + 1) & 31])), sc2, nm2);
-                        const float2 pp = make_float2(ex2_approx(x.x), ex2_approx(x.y));
-                        rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
-                        pk[half][(c >> 1) & 31] = pack_bf16x2(pp.x, pp.y);
+                        for (int c = half * 64; c < half * 64 + 64; c += 2) {
+                            const float s0 = __uint_as_float(s[c >> 5][c & 31]), s1 = __uint_as_float(s[(c + 1) >> 5][(c + 1) & 31]);
+                            const float2 x = __ffma2_rn(make_float2(s0, s1), sc2, nm2);
+                            const float2 pp = (((c >> 1) & 7) < POLY_PER_8) ? exp2_poly2(x)
+                                                                            : make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                            mx4[(c >> 1) & 3] = fmax3(mx4[(c >> 1) & 3], s0, s1);
+                            rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
+                            pk[(c >> 1) & 31] = pack_bf16x2(pp.x, pp.y);
+                        }
+                        tmem_st_x32(s_tmem + 32 * half, pk);
                     }
-                    tmem_st_x32(s_tmem + 32 * half, pk[half]);
+                    mx_out = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    const float2 r = __fadd2_rn(__fadd2_rn(rs4[0], rs4[1]), __fadd2_rn(rs4[2], rs4[3]));
+                    return r.x + r.y;
+                };
+                float mx_raw;
+                float rs = exp_pass(m_used, mx_raw);
+                if (t > 0) {
+                    const float m_tile = mx_raw * p.scale_log2;
+                    const bool need = (m_tile - m_used > RESCALE_THRESHOLD);
+                    if (__any_sync(0xFFFFFFFFu, need)) {   // rare: move the reference, rescale O and l, redo P
+                        const float alpha = need ? ex2_approx(m_used - m_tile) : 1.0f;
+                        if (need) m_used = m_tile;
+                        l_sum *= alpha;
+                        tmem_wait_st();
+#pragma unroll
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t o[32];
+                            tmem_ld_x32(o_tmem + c0, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            tmem_st_x32(o_tmem + c0, o);
+                        }
+                        rs = exp_pass(m_used, mx_raw);
+                    }
                 }
-                const float2 rs2 = __fadd2_rn(__fadd2_rn(rs4[0], rs4[1]), __fadd2_rn(rs4[2], rs4[3]));
-                l_sum += rs2.x + rs2.y;
+                l_sum += rs;
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bars.p_full + 8 * q);
