@@ -222,6 +222,7 @@ dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_b
     p.lse_state = ctx->lse_state;
     p.out = out_dev;
     p.lse_out = lse_out_dev;
+    p.status = ctx->status_dev;
     p.P = c.P; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];

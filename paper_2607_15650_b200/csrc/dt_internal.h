@@ -34,6 +34,7 @@ struct MergeParams {
     const float *lse_state;
     void *out;       // bf16
     float *lse_out;  // may be null
+    int32_t *status; // device status word
     int P, H, L;
     long long R;     // B*H*L rows
     long long sb, sl, sh;  // output strides in elements

@@ -1,16 +1,20 @@
 // dt_state_merge: Eq. 2 folded over the P cached states of every query row.
 //
-// HBM-bound streaming kernel.  One query row (b, h, l) is handled by D / VEC consecutive
-// threads, each owning VEC = 16 bytes / sizeof(state) head-dim elements; for every KV
-// partition j the row's slice of OUT_ij is one 128-bit load, so a warp reads 512 contiguous
-// bytes per j.  The P log-sum-exps of the row are read once per thread (same address across
-// the row's threads: one broadcast transaction) and turned into weights
-// exp(LSE_ij - max_j LSE_ij) / Z in fp32; the weighted sum is accumulated in fp32 and stored
-// as bf16 in the [B, L, H, D] output.  Algorithmic bytes per row:
-// P * (D * sizeof(state) + 4) read + 2 D + 4 written.
+// HBM-bound streaming kernel.  A block owns ROWS consecutive rows (b, h, l) of the cache.  For each
+// KV partition j those rows are one contiguous run of ROWS * D state elements, which one thread
+// fetches with a bulk asynchronous copy (cp.async.bulk, completion counted on an mbarrier) into
+// shared memory: P copies of a few KB each are in flight per block without costing a register,
+// and several blocks per SM keep the memory system saturated while others compute.  Meanwhile the
+// block's threads read the rows' P log-sum-exps, and each (row, 16-byte column group) thread forms
+// the weights exp(LSE_ij - max_j LSE_ij) / Z in fp32.  After the copies land, the weighted sum is
+// accumulated in fp32 from shared memory and stored as bf16 in the [B, L, H, D] output.
+// Algorithmic bytes per row: P * (D * sizeof(state) + 4) read + 2 D + 4 written.
+//
+// The wait for the copies is bounded; on expiry the block records STATUS_WAIT_TIMEOUT and returns.
 #include <cuda_bf16.h>
 
 #include "dt_internal.h"
+#include "ptx_sm100.cuh"
 
 namespace dt {
 namespace {
@@ -21,7 +25,7 @@ template <>
 struct StateVec<float> {
     static constexpr int VEC = 4;
     __device__ static __forceinline__ void load(const float *p, float (&v)[4]) {
-        float4 x = __ldcs(reinterpret_cast<const float4 *>(p));
+        const float4 x = *reinterpret_cast<const float4 *>(p);
         v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
     }
 };
@@ -29,7 +33,7 @@ template <>
 struct StateVec<__nv_bfloat16> {
     static constexpr int VEC = 8;
     __device__ static __forceinline__ void load(const __nv_bfloat16 *p, float (&v)[8]) {
-        uint4 x = __ldcs(reinterpret_cast<const uint4 *>(p));
+        const uint4 x = *reinterpret_cast<const uint4 *>(p);
         const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -55,62 +59,101 @@ __device__ __forceinline__ void store_bf16(__nv_bfloat16 *p, const float (&v)[VE
 }
 
 constexpr int MERGE_THREADS = 256;
-constexpr int JB = 8;  // states fetched per batch of independent loads
+constexpr int MERGE_STAGE_BYTES = 64 * 1024;          // state bytes one block keeps in flight
+constexpr long long MERGE_WAIT_LIMIT = 4000000000ll;  // SM clock cycles: about 2 s
 
 template <typename StateT, int D>
-__global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(MergeParams p) {
-    constexpr int VEC = StateVec<StateT>::VEC;
-    constexpr int TPR = D / VEC;                 // threads per row
-    constexpr int RPB = MERGE_THREADS / TPR;     // rows per block
-    const long long row = (long long)blockIdx.x * RPB + threadIdx.x / TPR;
-    const int lane = threadIdx.x % TPR;
-    if (row >= p.R) return;
-    const int P = p.P;
-    const StateT *o_state = static_cast<const StateT *>(p.o_state);
-
-    // weights: LSE_ij - M, then exp; P <= 32 values kept in registers
-    float ls[DT_MAX_P];
-    float M = -INFINITY;
-#pragma unroll
-    for (int j = 0; j < DT_MAX_P; ++j) {
-        ls[j] = (j < P) ? __ldg(p.lse_state + (long long)j * p.R + row) : -INFINITY;
-        M = fmaxf(M, ls[j]);
+struct MergeCfg {
+    static constexpr int VEC = StateVec<StateT>::VEC;
+    static constexpr int TPR = D / VEC;                       // threads per row
+    static constexpr int MAX_ROWS = MERGE_THREADS / TPR;      // rows the block's threads can cover
+    static constexpr int ROW_BYTES = D * (int)sizeof(StateT);
+    static int rows(int P) {
+        int r = MERGE_STAGE_BYTES / (P * ROW_BYTES);
+        r = r < 1 ? 1 : r;
+        return r > MAX_ROWS ? MAX_ROWS : r;
     }
-    float Z = 0.f;
+    static size_t smem_bytes(int P) {
+        return (size_t)P * rows(P) * ROW_BYTES + (size_t)rows(P) * DT_MAX_P * sizeof(float) + 32;
+    }
+};
+
+template <typename StateT, int D>
+__global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(MergeParams p, int ROWS) {
+    using Cf = MergeCfg<StateT, D>;
+    constexpr int VEC = Cf::VEC, TPR = Cf::TPR;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int P = p.P;
+    StateT *tile = reinterpret_cast<StateT *>(smem);                                   // [P][ROWS][D]
+    float *lse_s = reinterpret_cast<float *>(smem + (size_t)P * ROWS * Cf::ROW_BYTES); // [ROWS][DT_MAX_P]
+    uint64_t *bar_ptr = reinterpret_cast<uint64_t *>(lse_s + ROWS * DT_MAX_P);
+    int *abort_flag = reinterpret_cast<int *>(bar_ptr + 1);
+    const uint32_t bar = smem_u32(bar_ptr);
+
+    const long long row0 = (long long)blockIdx.x * ROWS;
+    const int valid = (int)min((long long)ROWS, p.R - row0);   // rows of this block that exist
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        mbar_init(bar, 1);
+        fence_mbar_init();
+        // one bulk copy per KV partition: `valid` consecutive rows of slot j
+        const uint32_t bytes = (uint32_t)valid * Cf::ROW_BYTES;
+        mbar_arrive_expect_tx(bar, bytes * (uint32_t)P);
+        const StateT *src = static_cast<const StateT *>(p.o_state) + row0 * D;
+        for (int j = 0; j < P; ++j)
+            bulk_load(smem_u32(tile + (size_t)j * ROWS * D), src + (long long)j * p.R * D, bytes, bar);
+    }
+    // the rows' log-sum-exps, through shared memory so that every thread of a row sees all P of them
+    for (int e = threadIdx.x; e < valid * P; e += MERGE_THREADS) {
+        const int r = e / P, j = e - r * P;
+        lse_s[r * DT_MAX_P + j] = __ldg(p.lse_state + (long long)j * p.R + row0 + r);
+    }
+    __syncthreads();   // also publishes the mbarrier initialisation to the waiting threads
+
+    const int r = threadIdx.x / TPR, lane = threadIdx.x % TPR;
+    const bool active = r < valid;
+    float w[DT_MAX_P];
+    float M = -INFINITY, Z = 0.f;
+    if (active) {
+#pragma unroll
+        for (int j = 0; j < DT_MAX_P; ++j) {
+            w[j] = (j < P) ? lse_s[r * DT_MAX_P + j] : -INFINITY;
+            M = fmaxf(M, w[j]);
+        }
+    }
     const bool empty = (M == -INFINITY);   // no partition has any mass: output 0, LSE = -inf
 #pragma unroll
     for (int j = 0; j < DT_MAX_P; ++j) {
-        ls[j] = (j < P && !empty) ? __expf(ls[j] - M) : 0.f;
-        Z += ls[j];
+        w[j] = (active && j < P && !empty) ? __expf(w[j] - M) : 0.f;
+        Z += w[j];
     }
+
+    if (!mbar_wait_bounded(bar, 0, abort_flag, MERGE_WAIT_LIMIT)) {
+        if (p.status) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
+        *abort_flag = 1;
+        return;
+    }
+    if (!active) return;
 
     float acc[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
-    const StateT *base = o_state + row * D + lane * VEC;
-    const long long slab = p.R * D;
+    const StateT *mine = tile + (size_t)r * D + lane * VEC;
 #pragma unroll
-    for (int j0 = 0; j0 < DT_MAX_P; j0 += JB) {
-        if (j0 < P) {
-            float v[JB][VEC];
+    for (int j = 0; j < DT_MAX_P; ++j) {
+        if (j < P) {
+            float v[VEC];
+            StateVec<StateT>::load(mine + (size_t)j * ROWS * D, v);
 #pragma unroll
-            for (int jj = 0; jj < JB; ++jj) {
-                if (j0 + jj < P) StateVec<StateT>::load(base + (long long)(j0 + jj) * slab, v[jj]);
-            }
-#pragma unroll
-            for (int jj = 0; jj < JB; ++jj) {
-                if (j0 + jj < P) {
-                    const float w = ls[j0 + jj];
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) acc[e] = fmaf(w, v[jj][e], acc[e]);
-                }
-            }
+            for (int e = 0; e < VEC; ++e) acc[e] = fmaf(w[j], v[e], acc[e]);
         }
     }
     const float inv = empty ? 0.f : 1.f / Z;
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] *= inv;
 
+    const long long row = row0 + r;
     const long long bh = row / p.L;
     const int l = (int)(row - bh * p.L);
     const int b = (int)(bh / p.H), h = (int)(bh - (long long)b * p.H);
@@ -121,10 +164,15 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(MergeParams 
 
 template <typename StateT, int D>
 cudaError_t launch(const MergeParams &p, cudaStream_t stream) {
-    constexpr int RPB = MERGE_THREADS / (D / StateVec<StateT>::VEC);
-    const long long blocks = (p.R + RPB - 1) / RPB;
+    using Cf = MergeCfg<StateT, D>;
+    const int rows = Cf::rows(p.P);
+    const size_t smem = Cf::smem_bytes(p.P);
+    const long long blocks = (p.R + rows - 1) / rows;
     if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
-    state_merge_kernel<StateT, D><<<(unsigned)blocks, MERGE_THREADS, 0, stream>>>(p);
+    cudaError_t e = cudaFuncSetAttribute(state_merge_kernel<StateT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         MERGE_STAGE_BYTES + MERGE_THREADS * DT_MAX_P * (int)sizeof(float) + 32);
+    if (e != cudaSuccess) return e;
+    state_merge_kernel<StateT, D><<<(unsigned)blocks, MERGE_THREADS, smem, stream>>>(p, rows);
     return cudaGetLastError();
 }
 
