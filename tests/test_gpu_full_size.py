@@ -1,0 +1,101 @@
+"""Parity at the full sizes of the named workloads, in the launch configuration bench.py times:
+anchor step (all pairs) -> dt_plan -> selective steps driven by that plan.
+
+The fp64 oracle cannot afford whole tensors here (1e14 flops at the headline size), so:
+  * the plan is checked in isolation: the oracle's contribution / target-fraction rule is fed the
+    GPU's own LSE cache (copied to the host) and must reproduce the GPU mask bit for bit, and
+    W to 2e-5 relative;
+  * the attention path is checked on a seeded sample of (head, row) pairs -- including the first
+    and last rows and the rows on both sides of every partition boundary -- whose pair states and
+    merged outputs the oracle computes one by one from the same bf16 inputs, following the same
+    masks over the steps (cached states included).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2607_15650_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+O_MAX, O_MEAN, LSE_ABS = 2e-2, 2e-3, 5e-3
+
+
+def _run_full_size(name, fraction, n_samples, n_selective, state_dtype=binding.DT_STATE_FP32):
+    build.build()
+    wl = inputs.WORKLOADS[name]
+    dev = torch.device("cuda", 0)
+    off = wl.offsets()
+    P = wl.P
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, off, wl.scale, state_dtype)
+    gen = inputs.StepInputs(wl, seed=0, device=dev)
+    rows = inputs.sample_rows(wl, n_samples, seed=11)
+    ses = orc.OracleSession(wl.B, wl.L, wl.H, wl.D, off, wl.scale, rows)
+    out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    mask = torch.ones(P * P, dtype=torch.uint8, device=dev)
+    W = torch.empty(P * P, dtype=torch.float64, device=dev)
+    eps = torch.empty(1, dtype=torch.float64, device=dev)
+    errs = []
+    for t in range(1 + n_selective):
+        q, k, v = gen.next()
+        mask_h = mask.cpu().numpy().reshape(P, P).copy()
+        ctx.dt_attn_states(q, k, v, mask, t)
+        ctx.dt_state_merge(out, lse)
+        torch.cuda.synchronize()
+        ctx.dt_poll()
+        # sampled rows against the oracle under the same plan
+        ref_o, ref_l = ses.step(*(inputs.bf16_bits(x) for x in (q, k, v)), mask_h, t)
+        for (b, h), r in rows.items():
+            ridx = torch.from_numpy(r.astype(np.int64)).to(dev)
+            got_o = out[b, ridx, h].float().cpu().numpy()
+            got_l = lse[b, h, ridx].cpu().numpy()
+            eo = np.abs(got_o - ref_o[(b, h)])
+            el = np.abs(got_l - ref_l[(b, h)])
+            errs.append((eo.max(), eo.mean(), el.max()))
+            assert eo.max() <= O_MAX and el.max() <= LSE_ABS, (name, t, b, h, eo.max(), el.max())
+            # the cached pair states of those rows, fresh or reused
+            st_o = ctx.o_state[:, b, h][:, ridx].float().cpu().numpy()          # [P, n, D]
+            st_l = ctx.lse_state[:, b, h][:, ridx].cpu().numpy()                # [P, n]
+            assert np.abs(st_o.transpose(1, 0, 2) - ses.o[(b, h)]).max() <= O_MAX
+            assert np.abs(st_l.T - ses.lse[(b, h)]).max() <= LSE_ABS
+        assert np.mean([e[1] for e in errs]) <= O_MEAN
+        assert (ctx.dt_get_tc() == ses.tc).all()
+        if t == 0:
+            # plan from the anchor step's LSE cache; the oracle gets the very same fp32 values
+            ctx.dt_plan(mask, target_fraction=fraction, w_dev=W, eps_out_dev=eps)
+            torch.cuda.synchronize()
+            lse_cache = ctx.lse_state.cpu().numpy().astype(np.float64)           # [P, B, H, L]
+            W_ref = orc.contribution(lse_cache, off)
+            Wg = W.cpu().numpy().reshape(P, P)
+            np.testing.assert_allclose(Wg, W_ref, rtol=2e-5, atol=1e-10)
+            got_mask = mask.cpu().numpy().reshape(P, P)
+            own_mask, own_eps, K = orc.target_fraction(Wg, fraction)
+            assert (got_mask == own_mask).all() and eps.item() == own_eps and got_mask.sum() == K
+            ref_mask, ref_eps, _ = orc.target_fraction(W_ref, fraction)
+            offd = ~np.eye(P, dtype=bool)
+            margin = np.abs(W_ref[offd] - ref_eps).min() / ref_eps
+            if margin > 1e-4:           # otherwise the oracle's own plan is not resolvable in fp32
+                assert (got_mask == ref_mask).all()
+            # locality of the synthetic workload: contribution falls with partition distance
+            d = np.abs(np.subtract.outer(np.arange(P), np.arange(P)))
+            assert W_ref[d == 0].mean() > W_ref[d == 1].mean() > W_ref[d >= 3].mean()
+    return errs
+
+
+def test_full_size_c3_wan720p_headline():
+    """The configuration bench.py times: 75 600 tokens, 40 heads, D 128, P 16, f = 0.40."""
+    _run_full_size("c3_wan720p", 0.40, n_samples=48, n_selective=2)
+
+
+def test_full_size_c1_cogvideox_d64_with_text_tokens():
+    _run_full_size("c1_cogvideox", 0.5, n_samples=64, n_selective=2)
+
+
+def test_full_size_c2_wan480p_uneven_partitions():
+    _run_full_size("c2_wan480p", 0.25, n_samples=48, n_selective=1)
+
+
+def test_full_size_c4_hunyuan_p32_bf16_state_cache():
+    """Largest footprint: 118 800 tokens, P = 32 (3712/3713-row partitions), states cached in bf16."""
+    _run_full_size("c4_hunyuan720p", 0.125, n_samples=32, n_selective=1, state_dtype=binding.DT_STATE_BF16)
