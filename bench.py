@@ -99,6 +99,12 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# DRAM traffic of attn_states_kernel per (head, COMPUTE pair) of the c3-shaped tiles, from the ncu capture
+# summarised in profiles/attn_states_kernel_c3_wan720p_h4.md: (243.5 MB read + 943.0 MB written) / (4 heads x 102 pairs).
+# Traffic grows in proportion to heads x pairs (the pair states written dominate it).
+NCU_ATTN_TRAFFIC_PER_HEAD_PAIR = {"c3_wan720p": (243.5e6 + 943.0e6) / (4 * 102)}
+
+
 def full_flops(wl) -> float:
     return 4.0 * wl.L * wl.L * wl.D * wl.H * wl.B
 
@@ -190,7 +196,7 @@ def run_reference(args, wl):
     d = np.abs(np.subtract.outer(np.arange(wl.P), np.arange(wl.P)))
     order = np.argsort(d.reshape(-1), kind="stable")
     mask = np.zeros(wl.P * wl.P, np.uint8); mask[order[:K]] = 1
-    budget = 8.0
+    budget = 5.0
     vals, secs = [], []
     for s in range(args.warmup + args.steps):
         eff, t, desc, cores = oracle_sample(wl, q, k, v, mask, budget, seed=s)
@@ -371,7 +377,10 @@ def run_cuda(args, wl):
         "e2e": e2e,
         "gpu_launches": launches,
         "roofline": {"kernel": "attn_states_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
-                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                     "unit": "TFLOP/s", "frac": achieved / peak,
+                     "traffic": (NCU_ATTN_TRAFFIC_PER_HEAD_PAIR[args.workload] * wl.H * n_comp
+                                 if args.workload in NCU_ATTN_TRAFFIC_PER_HEAD_PAIR and args.state_dtype == "fp32" else None),
+                     "traffic_note": "bytes per launch, ncu dram read+write of a 4-head capture scaled by heads x pairs",
                      "peak_source": f"{peaks['source']} bf16 sustained", "frac_of_burst": achieved / peaks["bf16_tflops"],
                      "frac_of_nominal_2250": achieved / 2250.0, "launch_ms": attn_avg_ms,
                      "algorithmic_flops_per_launch": comp_fl},
