@@ -44,7 +44,8 @@ constexpr int LAUNCH_REGS = 168, REGS_SOFTMAX = 208, REGS_PRODUCER = 88;
 static_assert((REGS_SOFTMAX - LAUNCH_REGS) * NUM_SOFTMAX_THREADS <= (LAUNCH_REGS - REGS_PRODUCER) * 128,
               "softmax warps would wait forever for registers nobody releases");
 constexpr long long WAIT_LIMIT_NS = 4000000000ll;   // SM clock cycles: about 2 s
-constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
+constexpr float ROWSUM_TRIGGER = 512.0f;   // a row sum of P at or above this sends the tile through the slow path
+constexpr float RESCALE_THRESHOLD = 1.0f;  // log2 units: in the slow path the reference moves if the maximum grew by more
 #ifndef DT_POLY_PER_8
 #define DT_POLY_PER_8 0
 #endif
@@ -403,7 +404,15 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     for (int c = 0; c < 128; ++c)
                         if (c >= valid) s[c >> 5][c & 31] = 0xFF800000u;  // -inf
                 }
-                if (t == 0) {   // first tile of the item: there is no earlier maximum to lean on
+                // P = exp2(s * scale_log2 - m_used) with the reference maximum of the earlier tiles.  While
+                // the row sum of P stays below ROWSUM_TRIGGER no element can have exceeded it, so the tile's
+                // own maximum is not needed.  Only when a sum reaches it (rare after the first tiles) is the
+                // maximum taken and, if it lies more than 2^RESCALE_THRESHOLD above the reference, the
+                // reference moved, O and l rescaled and P computed again; afterwards every P <= 2 and the
+                // row sum is at most 256, so the slow path does not fire again until the maximum grows.
+                // The result does not depend on the reference: it cancels in OUT = O / l and LSE = m + log l.
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+                auto row_max = [&]() -> float {   // raw maximum of the row: four chains of three-input max
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                     for (int c = 0; c < 128; c += 8) {
@@ -412,19 +421,12 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             mx4[u] = fmax3(mx4[u], __uint_as_float(s[(c + 2 * u) >> 5][(c + 2 * u) & 31]),
                                            __uint_as_float(s[(c + 2 * u + 1) >> 5][(c + 2 * u + 1) & 31]));
                     }
-                    m_used = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
-                }
-                // P = exp2(s * scale_log2 - m_used) with the reference maximum of the earlier tiles; this
-                // tile's own maximum is gathered in the shadow of the exponentials (the MUFU is the busy
-                // unit here).  Only if it exceeds m_used by more than 2^RESCALE_THRESHOLD are m_used, O and
-                // l moved and P computed again -- rare after the first tiles; the result does not depend
-                // on which reference is used, since it cancels in OUT = O / l and LSE = m + log l.
-                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-                // one pass over the row: P to TMEM, returns the row sum; optionally the raw row maximum
-                auto exp_pass = [&](float m_ref, float &mx_out) -> float {
+                    return fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                };
+                // one pass over the row: P to TMEM, returns the row sum
+                auto exp_pass = [&](float m_ref) -> float {
                     const float2 nm2 = make_float2(-m_ref, -m_ref);
                     float2 rs4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         uint32_t pk[32];  // 64 keys as packed bf16 pairs (even key in the low half)
@@ -434,22 +436,21 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             const float2 x = __ffma2_rn(make_float2(s0, s1), sc2, nm2);
                             const float2 pp = (((c >> 1) & 7) < POLY_PER_8) ? exp2_poly2(x)
                                                                             : make_float2(ex2_approx(x.x), ex2_approx(x.y));
-                            mx4[(c >> 1) & 3] = fmax3(mx4[(c >> 1) & 3], s0, s1);
                             rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
                             pk[(c >> 1) & 31] = pack_bf16x2(pp.x, pp.y);
                         }
                         tmem_st_x32(s_tmem + 32 * half, pk);
                     }
-                    mx_out = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                     const float2 r = __fadd2_rn(__fadd2_rn(rs4[0], rs4[1]), __fadd2_rn(rs4[2], rs4[3]));
                     return r.x + r.y;
                 };
-                float mx_raw;
-                float rs = exp_pass(m_used, mx_raw);
-                if (t > 0) {
-                    const float m_tile = mx_raw * p.scale_log2;
+                if (t == 0) m_used = row_max() * p.scale_log2;   // first tile: no earlier maximum to lean on
+                float rs = exp_pass(m_used);
+                // (the negated comparison also catches inf / NaN after an overflow)
+                if (t > 0 && __any_sync(0xFFFFFFFFu, !(rs < ROWSUM_TRIGGER))) {
+                    const float m_tile = row_max() * p.scale_log2;
                     const bool need = (m_tile - m_used > RESCALE_THRESHOLD);
-                    if (__any_sync(0xFFFFFFFFu, need)) {   // rare: move the reference, rescale O and l, redo P
+                    if (__any_sync(0xFFFFFFFFu, need)) {
                         const float alpha = need ? ex2_approx(m_used - m_tile) : 1.0f;
                         if (need) m_used = m_tile;
                         l_sum *= alpha;
@@ -463,7 +464,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
                             tmem_st_x32(o_tmem + c0, o);
                         }
-                        rs = exp_pass(m_used, mx_raw);
+                        rs = exp_pass(m_used);
                     }
                 }
                 l_sum += rs;
