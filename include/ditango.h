@@ -152,6 +152,12 @@ dt_status dt_set_tc(dt_ctx *ctx, const int32_t *tc_host);
 /* Number of kernels this library has launched through `ctx` since creation. */
 dt_status dt_launch_count(dt_ctx *ctx, uint64_t *count);
 
+/* Self-test of the failure path (the paper has no counterpart): launches a one-thread kernel that waits,
+ * with the library's bounded wait, on a barrier nothing will ever signal; after `limit_us` microseconds
+ * (1..100000) the wait gives up and records the condition, so the next dt_poll returns DT_ERR_TIMEOUT
+ * and the context stays usable.  No fault, trap or unbounded loop is involved. */
+dt_status dt_selftest_wait_timeout(dt_ctx *ctx, uint32_t limit_us, void *stream);
+
 /* Read (and clear) the device status word; synchronises the device.  Returns DT_OK,
  * DT_ERR_STATE or DT_ERR_TIMEOUT. */
 dt_status dt_poll(dt_ctx *ctx);

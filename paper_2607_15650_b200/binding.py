@@ -21,7 +21,7 @@ DT_MAX_P = 32
 EXPORTS = [
     "dt_create", "dt_destroy", "dt_cache_bytes", "dt_bind_cache", "dt_attn_states", "dt_state_merge",
     "dt_plan", "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
-    "dt_launch_count", "dt_poll", "dt_status_str", "dt_last_error",
+    "dt_launch_count", "dt_selftest_wait_timeout", "dt_poll", "dt_status_str", "dt_last_error",
 ]
 
 
@@ -67,6 +67,7 @@ def lib():
         "dt_get_tc": (C.c_int, [vp, i32p]),
         "dt_set_tc": (C.c_int, [vp, i32p]),
         "dt_launch_count": (C.c_int, [vp, C.POINTER(C.c_uint64)]),
+        "dt_selftest_wait_timeout": (C.c_int, [vp, C.c_uint32, vp]),
         "dt_poll": (C.c_int, [vp]),
         "dt_status_str": (C.c_char_p, [C.c_int]),
         "dt_last_error": (C.c_char_p, [vp]),
@@ -216,6 +217,9 @@ class Context:
         n = C.c_uint64()
         self._check(lib().dt_launch_count(self._h, C.byref(n)))
         return int(n.value)
+
+    def dt_selftest_wait_timeout(self, limit_us=1000, stream=None):
+        self._check(lib().dt_selftest_wait_timeout(self._h, int(limit_us), _stream_ptr(stream)))
 
     def dt_poll(self):
         """Raises DitangoError if the device recorded a condition; returns None otherwise."""

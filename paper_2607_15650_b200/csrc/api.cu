@@ -334,6 +334,16 @@ dt_status dt_launch_count(dt_ctx *ctx, uint64_t *count) {
     return DT_OK;
 }
 
+dt_status dt_selftest_wait_timeout(dt_ctx *ctx, uint32_t limit_us, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (limit_us == 0 || limit_us > 100000) return fail(ctx, DT_ERR_INVALID_ARG, "limit_us must be in [1, 100000]");
+    const long long cycles = (long long)limit_us * 2000;   // about 2 GHz
+    cudaError_t e = dt::launch_wait_timeout_selftest(ctx->status_dev, cycles, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "self-test launch");
+    ctx->launches += 1;
+    return DT_OK;
+}
+
 dt_status dt_poll(dt_ctx *ctx) {
     if (!ctx) return DT_ERR_INVALID_ARG;
     int32_t word = 0;

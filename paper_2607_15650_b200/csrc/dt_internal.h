@@ -68,6 +68,7 @@ cudaError_t attn_states_configure();  // sets the dynamic shared-memory attribut
 cudaError_t launch_state_merge(const MergeParams &p, int D, int state_dtype, cudaStream_t stream);
 cudaError_t launch_plan_partial(const PlanParams &p, cudaStream_t stream);
 cudaError_t launch_plan_final(const PlanFinalParams &p, cudaStream_t stream);
+cudaError_t launch_wait_timeout_selftest(int32_t *status, long long limit_cycles, cudaStream_t stream);
 
 }  // namespace dt
 

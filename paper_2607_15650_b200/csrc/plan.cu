@@ -12,6 +12,7 @@
 #include <math.h>
 
 #include "dt_internal.h"
+#include "ptx_sm100.cuh"
 
 namespace dt {
 namespace {
@@ -145,6 +146,27 @@ __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int
     }
 }
 
+// Self-test of the bounded-wait machinery: one thread waits on an mbarrier that nobody will ever
+// arrive at, with a short limit; the wait must give up, record STATUS_WAIT_TIMEOUT and return.
+__global__ void wait_timeout_selftest_kernel(int32_t *status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+        if (!mbar_wait_bounded(smem_u32(&bar), 0, &abort_flag, limit_cycles)) atomicOr(status, STATUS_WAIT_TIMEOUT);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_wait_timeout_selftest(int32_t *status, long long limit_cycles, cudaStream_t stream) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_cycles);
+    return cudaGetLastError();
+}
+
+namespace {
 }  // namespace
 
 cudaError_t launch_plan_partial(const PlanParams &p, cudaStream_t stream) {

@@ -271,6 +271,28 @@ def test_reuse_of_never_computed_pair_is_reported():
     assert (ctx.dt_get_tc() == tc2).all()
 
 
+def test_bounded_wait_gives_up_and_the_context_stays_usable():
+    """A wait that nothing will ever satisfy runs out after its limit, is reported by dt_poll as
+    DT_ERR_TIMEOUT, and the same context then runs a normal step."""
+    wl = inputs.tiny_workload(grid=(2, 6, 7), P=3)
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale)
+    ctx.dt_selftest_wait_timeout(limit_us=500)
+    with pytest.raises(binding.DitangoError) as ei:
+        ctx.dt_poll()
+    assert ei.value.status == binding.DT_ERR_TIMEOUT
+    ctx.dt_poll()                                            # cleared
+    q, k, v = inputs.StepInputs(wl, device=dev).next()
+    out = torch.empty_like(q)
+    ctx.dt_attn_states(q, k, v, torch.ones(9, dtype=torch.uint8, device=dev), 0)
+    ctx.dt_state_merge(out, None)
+    torch.cuda.synchronize()
+    ctx.dt_poll()
+    qb, kb, vb = (inputs.bf16_bits(x) for x in (q, k, v))
+    ref, _ = orc.full_attention(qb, kb, vb, wl.scale, 0, 1, np.arange(wl.L, dtype=np.int32))
+    check_o(out[0, :, 1].float().cpu().numpy(), ref, "after self-test")
+
+
 def test_argument_errors_do_not_launch():
     wl = inputs.tiny_workload()
     dev = torch.device("cuda", 0)
