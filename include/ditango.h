@@ -95,6 +95,23 @@ dt_status dt_attn_states(dt_ctx *ctx, const void *q_dev, const void *k_dev, cons
 dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev,
                          void *stream);
 
+/* Composed reuse state (Section 2.2.4, Fig. 6: "compose states from remote partitions and cache the
+ * result"; Eq. 15 is the same composition applied to groups).  While a plan holds, the REUSE states of
+ * a query row do not change, so they can be composed once (Eq. 2) into a single state per row:
+ *   dt_compose_reuse        comp = (+) over { j : mask[i][j] == 0 } of the cached state (i, j), for every
+ *                           row of every query partition i; rows without any REUSE slot get OUT = 0,
+ *                           LSE = -inf (weight zero).
+ *   dt_state_merge_planned  out = (+) over { j : mask[i][j] != 0 } of the cached states, (+) comp.
+ * With comp built from the same mask and an unchanged cache in the REUSE slots, the result equals
+ * dt_state_merge up to rounding, while reading (computed + 1) states per row instead of P.
+ *   mask_dev       device, uint8 [P*P], as in dt_attn_states
+ *   comp_o_dev     device, [B][H][L][D] in the cache's state dtype, 16-byte aligned (caller-owned)
+ *   comp_lse_dev   device, fp32 [B][H][L]
+ * Recompose whenever the plan changes or a REUSE slot is recomputed. */
+dt_status dt_compose_reuse(dt_ctx *ctx, const uint8_t *mask_dev, void *comp_o_dev, float *comp_lse_dev, void *stream);
+dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const void *comp_o_dev, const float *comp_lse_dev,
+                                 void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev, void *stream);
+
 /* Plan from the cached LSEs (call after a step that computed every pair -- an anchor step):
  *   per row  w_j = exp(LSE_ij - logsumexp_k LSE_ik)                  (Eq. 8)
  *   W[i][j]  = mean of w_j over batch, heads and the rows of partition i

@@ -20,7 +20,7 @@ DT_MAX_P = 32
 
 EXPORTS = [
     "dt_create", "dt_destroy", "dt_cache_bytes", "dt_bind_cache", "dt_attn_states", "dt_state_merge",
-    "dt_plan", "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
+    "dt_compose_reuse", "dt_state_merge_planned", "dt_plan", "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
     "dt_launch_count", "dt_selftest_wait_timeout", "dt_poll", "dt_status_str", "dt_last_error",
 ]
 
@@ -59,6 +59,8 @@ def lib():
         "dt_bind_cache": (C.c_int, [vp, vp, f32p, C.c_size_t, C.c_size_t]),
         "dt_attn_states": (C.c_int, [vp, vp, vp, vp, i64p, u8p, C.c_int32, vp]),
         "dt_state_merge": (C.c_int, [vp, vp, i64p, f32p, vp]),
+        "dt_compose_reuse": (C.c_int, [vp, u8p, vp, f32p, vp]),
+        "dt_state_merge_planned": (C.c_int, [vp, u8p, vp, f32p, vp, i64p, f32p, vp]),
         "dt_plan": (C.c_int, [vp, C.c_double, C.c_double, u8p, f64p, f64p, vp]),
         "dt_plan_static": (C.c_int, [f32p, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_double,
                            u8p, f64p, f64p, vp]),
@@ -184,6 +186,19 @@ class Context:
         if lse_out is not None:
             assert lse_out.dtype == torch.float32 and lse_out.is_contiguous()
         self._check(lib().dt_state_merge(self._h, C.c_void_p(out.data_ptr()), _strides4(out), lp, _stream_ptr(stream)))
+
+    def dt_compose_reuse(self, mask_dev, comp_o, comp_lse, stream=None):
+        assert comp_o.is_cuda and comp_o.is_contiguous() and comp_o.dtype == self.o_state.dtype
+        assert comp_lse.is_cuda and comp_lse.is_contiguous() and comp_lse.dtype == torch.float32
+        self._check(lib().dt_compose_reuse(self._h, C.c_void_p(mask_dev.data_ptr()), C.c_void_p(comp_o.data_ptr()),
+                                           C.c_void_p(comp_lse.data_ptr()), _stream_ptr(stream)))
+
+    def dt_state_merge_planned(self, mask_dev, comp_o, comp_lse, out, lse_out=None, stream=None):
+        assert out.dtype == torch.bfloat16 and out.is_cuda
+        lp = C.c_void_p(lse_out.data_ptr()) if lse_out is not None else C.c_void_p()
+        self._check(lib().dt_state_merge_planned(self._h, C.c_void_p(mask_dev.data_ptr()), C.c_void_p(comp_o.data_ptr()),
+                                                 C.c_void_p(comp_lse.data_ptr()), C.c_void_p(out.data_ptr()),
+                                                 _strides4(out), lp, _stream_ptr(stream)))
 
     def dt_plan(self, mask_dev, eps=0.0, target_fraction=-1.0, w_dev=None, eps_out_dev=None, stream=None):
         assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()

@@ -217,7 +217,8 @@ dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_b
     dt_status s = check_strides(out_strides_blhd, out_dev, &why);
     if (s != DT_OK) return fail(ctx, s, why);
     const dt_config &c = ctx->cfg;
-    dt::MergeParams p;
+    dt::MergeParams p = {};
+    p.mode = dt::MERGE_ALL;
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
     p.out = out_dev;
@@ -228,6 +229,59 @@ dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_b
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "merge launch");
+    ctx->launches += 1;
+    return DT_OK;
+}
+
+dt_status dt_compose_reuse(dt_ctx *ctx, const uint8_t *mask_dev, void *comp_o_dev, float *comp_lse_dev, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!mask_dev || !comp_o_dev || !comp_lse_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null pointer");
+    if ((reinterpret_cast<uintptr_t>(comp_o_dev) & 15u) != 0) return fail(ctx, DT_ERR_INVALID_ARG, "composed state must be 16-byte aligned");
+    if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
+    const dt_config &c = ctx->cfg;
+    dt::MergeParams p = {};
+    p.mode = dt::MERGE_COMPOSE;
+    p.mask = mask_dev;
+    p.off = ctx->off_dev;
+    p.o_state = ctx->o_state;
+    p.lse_state = ctx->lse_state;
+    p.comp_o_out = comp_o_dev;
+    p.comp_lse_out = comp_lse_dev;
+    p.status = ctx->status_dev;
+    p.P = c.P; p.H = c.H; p.L = c.L;
+    p.R = (long long)c.B * c.H * c.L;
+    cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "compose launch");
+    ctx->launches += 1;
+    return DT_OK;
+}
+
+dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const void *comp_o_dev, const float *comp_lse_dev,
+                                 void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!mask_dev || !comp_o_dev || !comp_lse_dev || !out_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null pointer");
+    if ((reinterpret_cast<uintptr_t>(comp_o_dev) & 15u) != 0) return fail(ctx, DT_ERR_INVALID_ARG, "composed state must be 16-byte aligned");
+    if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
+    const char *why;
+    dt_status s = check_strides(out_strides_blhd, out_dev, &why);
+    if (s != DT_OK) return fail(ctx, s, why);
+    const dt_config &c = ctx->cfg;
+    dt::MergeParams p = {};
+    p.mode = dt::MERGE_PLANNED;
+    p.mask = mask_dev;
+    p.off = ctx->off_dev;
+    p.o_state = ctx->o_state;
+    p.lse_state = ctx->lse_state;
+    p.comp_o = comp_o_dev;
+    p.comp_lse = comp_lse_dev;
+    p.out = out_dev;
+    p.lse_out = lse_out_dev;
+    p.status = ctx->status_dev;
+    p.P = c.P; p.H = c.H; p.L = c.L;
+    p.R = (long long)c.B * c.H * c.L;
+    p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
+    cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "planned merge launch");
     ctx->launches += 1;
     return DT_OK;
 }

@@ -29,7 +29,16 @@ struct AttnParams {
     float scale_log2;         // softmax_scale * log2(e)
 };
 
+enum : int { MERGE_ALL = 0, MERGE_COMPOSE = 1, MERGE_PLANNED = 2 };
+
 struct MergeParams {
+    int mode;                 // MERGE_ALL / MERGE_COMPOSE / MERGE_PLANNED
+    const uint8_t *mask;      // device, P*P (modes COMPOSE, PLANNED)
+    const int32_t *off;       // device, P+1 (modes COMPOSE, PLANNED)
+    const void *comp_o;       // composed state read by PLANNED: [B][H][L][D] in the cache's dtype
+    const float *comp_lse;    // [B][H][L]
+    void *comp_o_out;         // composed state written by COMPOSE
+    float *comp_lse_out;
     const void *o_state;
     const float *lse_state;
     void *out;       // bf16

@@ -158,6 +158,58 @@ def test_state_merge_alone_on_oracle_states():
         check_lse(lse.cpu().numpy().reshape(-1), ref_l, "merge alone")
 
 
+@pytest.mark.parametrize("state_dtype", [binding.DT_STATE_FP32, binding.DT_STATE_BF16])
+def test_composed_reuse_state_and_planned_merge(state_dtype):
+    """Fig. 6 / Eq. 15: the REUSE states of a plan are composed once into one cached state per row; a
+    selective step then merges its COMPUTE states with that composed state.  The composed state is
+    compared with the oracle's composition of the same slots, the planned merge with the oracle's
+    step output (which composes all P slots), over uneven partitions and a block that straddles them."""
+    offsets = [0, 100, 257, 300, 521, 700]
+    wl = inputs.Workload("compose", 1, 2, 128, (4, 7, 25), 0, 5, 2, 0.05)
+    P = 5
+    run = Run(wl, offsets=offsets, seed=13, state_dtype=state_dtype)
+    run.step(np.ones((P, P), np.uint8))
+    mask = inputs.banded_mask(P, 1)
+    mask[4, 0] = 1                                        # a non-banded COMPUTE pair
+    mask[2, :] = 1                                        # a query partition without any REUSE slot
+    dev = run.dev
+    mask_dev = torch.from_numpy(mask.reshape(-1).copy()).to(dev)
+    sdt = torch.float32 if state_dtype == binding.DT_STATE_FP32 else torch.bfloat16
+    comp_o = torch.empty((wl.B, wl.H, wl.L, wl.D), dtype=sdt, device=dev)
+    comp_l = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    run.ctx.dt_compose_reuse(mask_dev, comp_o, comp_l)
+    torch.cuda.synchronize()
+    run.ctx.dt_poll()
+    part = np.searchsorted(np.asarray(offsets), np.arange(wl.L), side="right") - 1
+    for (b, h), rows in run.rows.items():
+        o_ref = np.zeros((wl.L, wl.D)); l_ref = np.full(wl.L, -np.inf)
+        for i in range(P):
+            sel = np.nonzero(part == i)[0]
+            reuse = [j for j in range(P) if mask[i, j] == 0]
+            if reuse:
+                o_ref[sel], l_ref[sel] = orc.merge(run.ses.o[(b, h)][sel][:, reuse, :], run.ses.lse[(b, h)][sel][:, reuse])
+        got_l = comp_l[b, h].cpu().numpy()
+        fin = np.isfinite(l_ref)
+        assert (np.isneginf(got_l) == ~fin).all()
+        check_lse(got_l[fin], l_ref[fin], "composed state")
+        check_o(comp_o[b, h].float().cpu().numpy(), o_ref, "composed state")
+    # selective step: fresh COMPUTE states, then COMPUTE slots (+) composed state
+    run.t += 1
+    q, k, v = run.gen.next()
+    run.ctx.dt_attn_states(q, k, v, mask_dev, run.t)
+    out2 = torch.empty_like(run.out); lse2 = torch.empty_like(run.lse)
+    run.ctx.dt_state_merge_planned(mask_dev, comp_o, comp_l, out2, lse2)
+    run.ctx.dt_state_merge(run.out, run.lse)
+    torch.cuda.synchronize()
+    run.ctx.dt_poll()
+    outs, lses = run.ses.step(*(inputs.bf16_bits(x) for x in (q, k, v)), mask, run.t)
+    for (b, h), rows in run.rows.items():
+        check_o(out2[b, :, h].float().cpu().numpy(), outs[(b, h)], "planned merge")
+        check_lse(lse2[b, h].cpu().numpy(), lses[(b, h)], "planned merge")
+    assert (out2.float() - run.out.float()).abs().max().item() <= 2e-2
+    assert (lse2 - run.lse).abs().max().item() <= 5e-3
+
+
 def _plan_case(wl, lse_host, off, fractions, eps_list):
     """dt_plan on a given LSE cache (fp32 values) against the oracle fed the same values."""
     dev = torch.device("cuda", 0)
