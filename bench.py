@@ -258,20 +258,34 @@ def run_cuda(args, wl):
         ctx.dt_attn_states(q, k, v, masks[cur], t)
         if timers is not None:
             e[1].record(stream)
-        ctx.dt_state_merge(out, lse)
+        if args.composed:
+            ctx.dt_state_merge_planned(masks[cur], comp_o, comp_l, out, lse)
+        else:
+            ctx.dt_state_merge(out, lse)
         if timers is not None:
             e[2].record(stream)
         ctx.dt_plan(masks[cur ^ 1], target_fraction=frac, w_dev=W)
         if timers is not None:
             e[3].record(stream)
             timers.append(e)
-        return cur ^ 1
+        return cur if args.composed else cur ^ 1   # composed mode: the anchor's plan holds until the next anchor
 
     # anchor step: every pair computed, first plan derived from it
     q, k, v = steps_in[0]
     ctx.dt_attn_states(q, k, v, ones, 0)
     ctx.dt_state_merge(out, lse)
     ctx.dt_plan(masks[0], target_fraction=frac, w_dev=W)
+    comp_o = comp_l = None
+    compose_ms = None
+    if args.composed:
+        comp_o = torch.empty((wl.B, wl.H, wl.L, wl.D), dtype=ctx.o_state.dtype, device=dev)
+        comp_l = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+        c0, c1 = ev(), ev()
+        c0.record(stream)
+        ctx.dt_compose_reuse(masks[0], comp_o, comp_l)
+        c1.record(stream)
+        torch.cuda.synchronize()
+        compose_ms = c0.elapsed_time(c1)
     torch.cuda.synchronize()
     ctx.dt_poll()
     cur = 0
@@ -370,7 +384,8 @@ def run_cuda(args, wl):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "D": wl.D, "L": wl.L, "P": wl.P,
                    "computed_pairs": n_comp, "computed_pair_fraction": n_comp / PP, "state_dtype": args.state_dtype,
-                   "step": "dt_attn_states + dt_state_merge + dt_plan", "multi_gpu": "independent replicas",
+                   "step": ("dt_attn_states + dt_state_merge_planned + dt_plan" if args.composed
+                            else "dt_attn_states + dt_state_merge + dt_plan"), "multi_gpu": "independent replicas",
                    "l2": "inputs (%.1f GB) and state cache larger than L2; no flush" %
                          ((3 * wl.L * wl.H * wl.D * 2) / 1e9)},
         "clocks": clocks,
@@ -390,7 +405,7 @@ def run_cuda(args, wl):
             "merge_gbs": merge_bytes(wl, sbytes) / 1e9 / (float(np.mean(merge_ms)) / 1e3),
             "merge_frac_of_hbm": merge_bytes(wl, sbytes) / 1e9 / (float(np.mean(merge_ms)) / 1e3) / peaks["hbm_gbs"],
             "plan_gbs": plan_bytes(wl) / 1e9 / (float(np.mean(plan_ms)) / 1e3),
-            "hbm_peak_gbs": peaks["hbm_gbs"],
+            "hbm_peak_gbs": peaks["hbm_gbs"], "compose_once_ms": compose_ms,
         },
         "vs_all_compute": {"all_compute_attn_ms": full_attn_ms, "all_compute_step_ms": full_step_ms,
                            "all_compute_tflops": full_flops(wl) / 1e12 / (full_attn_ms / 1e3),
@@ -411,6 +426,9 @@ def main():
     ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
     ap.add_argument("--heads", type=int, default=None,
                     help="override the head count (smaller captures under a profiler; not a bench configuration)")
+    ap.add_argument("--composed", action="store_true",
+                    help="compose the plan's REUSE states once after the anchor step and merge COMPUTE states + that "
+                         "composed state in the selective steps (the plan then stays fixed between anchors)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

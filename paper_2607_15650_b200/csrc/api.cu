@@ -134,6 +134,7 @@ dt_status dt_create(dt_ctx **ctx_out, const dt_config *cfg) {
     ok = ok && cudaMalloc(&ctx->tc_dev, P * P * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->worklist_dev, (1 + P * P) * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->status_dev, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->sel_bits_dev, 2 * DT_MAX_P * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->plan_partials_dev, (size_t)BH * P * ctx->plan_chunks * P * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMemcpy(ctx->off_dev, ctx->off.data(), (P + 1) * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemset(ctx->tc_dev, 0xFF, P * P * sizeof(int32_t)) == cudaSuccess;  // -1 = empty
@@ -156,6 +157,7 @@ dt_status dt_destroy(dt_ctx *ctx) {
     cudaFree(ctx->worklist_dev);
     cudaFree(ctx->status_dev);
     cudaFree(ctx->plan_partials_dev);
+    cudaFree(ctx->sel_bits_dev);
     delete ctx;
     return DT_OK;
 }
@@ -241,8 +243,10 @@ dt_status dt_compose_reuse(dt_ctx *ctx, const uint8_t *mask_dev, void *comp_o_de
     const dt_config &c = ctx->cfg;
     dt::MergeParams p = {};
     p.mode = dt::MERGE_COMPOSE;
-    p.mask = mask_dev;
-    p.off = ctx->off_dev;
+    p.sel_bits = ctx->sel_bits_dev;
+    for (int i = 0; i <= c.P; ++i) p.off_val[i] = ctx->off[i];
+    cudaError_t es = dt::launch_merge_select(mask_dev, c.P, 0, ctx->sel_bits_dev, static_cast<cudaStream_t>(stream));
+    if (es != cudaSuccess) return fail_cuda(ctx, es, "selection launch");
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
     p.comp_o_out = comp_o_dev;
@@ -252,7 +256,7 @@ dt_status dt_compose_reuse(dt_ctx *ctx, const uint8_t *mask_dev, void *comp_o_de
     p.R = (long long)c.B * c.H * c.L;
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "compose launch");
-    ctx->launches += 1;
+    ctx->launches += 2;
     return DT_OK;
 }
 
@@ -268,8 +272,10 @@ dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const voi
     const dt_config &c = ctx->cfg;
     dt::MergeParams p = {};
     p.mode = dt::MERGE_PLANNED;
-    p.mask = mask_dev;
-    p.off = ctx->off_dev;
+    p.sel_bits = ctx->sel_bits_dev + DT_MAX_P;
+    for (int i = 0; i <= c.P; ++i) p.off_val[i] = ctx->off[i];
+    cudaError_t es = dt::launch_merge_select(mask_dev, c.P, 1, ctx->sel_bits_dev + DT_MAX_P, static_cast<cudaStream_t>(stream));
+    if (es != cudaSuccess) return fail_cuda(ctx, es, "selection launch");
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
     p.comp_o = comp_o_dev;
@@ -282,7 +288,7 @@ dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const voi
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "planned merge launch");
-    ctx->launches += 1;
+    ctx->launches += 2;
     return DT_OK;
 }
 

@@ -33,8 +33,8 @@ enum : int { MERGE_ALL = 0, MERGE_COMPOSE = 1, MERGE_PLANNED = 2 };
 
 struct MergeParams {
     int mode;                 // MERGE_ALL / MERGE_COMPOSE / MERGE_PLANNED
-    const uint8_t *mask;      // device, P*P (modes COMPOSE, PLANNED)
-    const int32_t *off;       // device, P+1 (modes COMPOSE, PLANNED)
+    const uint32_t *sel_bits; // device, P words from launch_merge_select (modes COMPOSE, PLANNED)
+    int32_t off_val[DT_MAX_P + 1];   // partition offsets by value (modes COMPOSE, PLANNED)
     const void *comp_o;       // composed state read by PLANNED: [B][H][L][D] in the cache's dtype
     const float *comp_lse;    // [B][H][L]
     void *comp_o_out;         // composed state written by COMPOSE
@@ -75,6 +75,7 @@ cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, con
                                const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream);
 cudaError_t attn_states_configure();  // sets the dynamic shared-memory attribute once per process/device
 cudaError_t launch_state_merge(const MergeParams &p, int D, int state_dtype, cudaStream_t stream);
+cudaError_t launch_merge_select(const uint8_t *mask, int P, int want_compute, uint32_t *sel_bits, cudaStream_t stream);
 cudaError_t launch_plan_partial(const PlanParams &p, cudaStream_t stream);
 cudaError_t launch_plan_final(const PlanFinalParams &p, cudaStream_t stream);
 cudaError_t launch_wait_timeout_selftest(int32_t *status, long long limit_cycles, cudaStream_t stream);
@@ -93,6 +94,7 @@ struct dt_ctx {
     int32_t *worklist_dev = nullptr;
     int32_t *status_dev = nullptr;
     float *plan_partials_dev = nullptr;
+    uint32_t *sel_bits_dev = nullptr;   // 2 * DT_MAX_P words: composition, planned merge
     void *o_state = nullptr;
     float *lse_state = nullptr;
     uint64_t launches = 0;

@@ -67,19 +67,26 @@ constexpr int MERGE_THREADS = 256;
 constexpr int MERGE_STAGE_BYTES = 64 * 1024;          // state bytes one block keeps in flight
 constexpr long long MERGE_WAIT_LIMIT = 4000000000ll;  // SM clock cycles: about 2 s
 
+constexpr int MERGE_CHUNK = 8;   // sources staged at a time by the subset modes
+
 template <typename StateT, int D>
 struct MergeCfg {
     static constexpr int VEC = StateVec<StateT>::VEC;
     static constexpr int TPR = D / VEC;                       // threads per row
     static constexpr int MAX_ROWS = MERGE_THREADS / TPR;      // rows the block's threads can cover
     static constexpr int ROW_BYTES = D * (int)sizeof(StateT);
-    static int rows(int nslots) {
-        int r = MERGE_STAGE_BYTES / (nslots * ROW_BYTES);
+    // MERGE_ALL stages all P slots at once (64 KB per block, three blocks per SM); the subset modes stage
+    // MERGE_CHUNK sources at a time for the full MAX_ROWS rows (32 KB per block, six blocks per SM), so
+    // that a step which needs few sources per row still keeps many bytes in flight per SM.
+    static int rows(int mode, int P) {
+        if (mode != MERGE_ALL) return MAX_ROWS;
+        int r = MERGE_STAGE_BYTES / (P * ROW_BYTES);
         r = r < 1 ? 1 : r;
         return r > MAX_ROWS ? MAX_ROWS : r;
     }
-    static size_t smem_bytes(int nslots) {
-        return (size_t)nslots * rows(nslots) * ROW_BYTES + (size_t)rows(nslots) * (DT_MAX_P + 1) * sizeof(float) + 32;
+    static int staged(int mode, int P) { return mode == MERGE_ALL ? P : MERGE_CHUNK; }
+    static size_t smem_bytes(int mode, int P) {
+        return (size_t)staged(mode, P) * rows(mode, P) * ROW_BYTES + (size_t)rows(mode, P) * (DT_MAX_P + 1) * sizeof(float) + 40 + 64;
     }
 };
 
@@ -97,129 +104,133 @@ __device__ __forceinline__ void store_state(__nv_bfloat16 *p, const float (&v)[V
 //   MERGE_COMPOSE  the REUSE slots of the row's query partition (mask == 0); the result is itself a
 //                  state (OUT in the cache's dtype, LSE) written to the composed-state buffers
 //   MERGE_PLANNED  the COMPUTE slots (mask != 0) plus the composed state as one more source
-template <typename StateT, int D>
-__global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(MergeParams p, int ROWS) {
+template <typename StateT, int D, int MODE>
+__global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid_constant__ MergeParams p, int ROWS) {
     using Cf = MergeCfg<StateT, D>;
     constexpr int VEC = Cf::VEC, TPR = Cf::TPR;
     constexpr int NS = DT_MAX_P + 1;   // sources per row at most: P slots + the composed state
     extern __shared__ __align__(128) uint8_t smem[];
-    __shared__ int32_t off_s[DT_MAX_P + 1];
-    __shared__ uint32_t sel_s[DT_MAX_P];   // per query partition: bit j set = slot j takes part
     const int P = p.P;
-    const int nslots = P + (p.mode == MERGE_PLANNED ? 1 : 0);
-    StateT *tile = reinterpret_cast<StateT *>(smem);                                        // [nslots][ROWS][D]
-    float *lse_s = reinterpret_cast<float *>(smem + (size_t)nslots * ROWS * Cf::ROW_BYTES);  // [ROWS][NS]
-    uint64_t *bar_ptr = reinterpret_cast<uint64_t *>(lse_s + ROWS * NS);
+    constexpr int EXTRA = (MODE == MERGE_PLANNED) ? 1 : 0;
+    const int nslots = P + EXTRA;
+    const int staged = (MODE == MERGE_ALL) ? P : MERGE_CHUNK;
+    StateT *tile = reinterpret_cast<StateT *>(smem);                                         // [staged][ROWS][D]
+    float *lse_s = reinterpret_cast<float *>(smem + (size_t)staged * ROWS * Cf::ROW_BYTES);   // [ROWS][NS]
+    uint64_t *bar_ptr = reinterpret_cast<uint64_t *>(lse_s + ((ROWS * NS + 1) & ~1));        // 8-byte aligned
     int *abort_flag = reinterpret_cast<int *>(bar_ptr + 1);
+    int *nsrc_s = abort_flag + 1;
+    uint8_t *src_s = reinterpret_cast<uint8_t *>(abort_flag + 2);                             // [NS] source ids in staging order
     const uint32_t bar = smem_u32(bar_ptr);
 
     const long long row0 = (long long)blockIdx.x * ROWS;
     const int valid = (int)min((long long)ROWS, p.R - row0);   // rows of this block that exist
+    const uint32_t bytes = (uint32_t)valid * Cf::ROW_BYTES;
 
-    if (p.mode != MERGE_ALL) {
-        if (threadIdx.x <= P) off_s[threadIdx.x] = p.off[threadIdx.x];
-        if (threadIdx.x < P) {
-            uint32_t bits = 0;
-            for (int j = 0; j < P; ++j) {
-                const bool compute = p.mask[threadIdx.x * P + j] != 0;
-                if (compute == (p.mode == MERGE_PLANNED)) bits |= 1u << j;
-            }
-            sel_s[threadIdx.x] = bits;
-        }
-        __syncthreads();
-    }
-    // query partition of a cache row (token index l = row mod L)
+    // query partition of a cache row (token index l = row mod L); the offsets travel as kernel
+    // parameters, so this needs no memory access
     auto partition_of = [&](long long row) -> int {
         const int l = (int)(row % p.L);
         int i = 0;
-        while (i + 1 < P && off_s[i + 1] <= l) ++i;
+#pragma unroll 1
+        while (i + 1 < P && p.off_val[i + 1] <= l) ++i;
         return i;
     };
+    // per query partition, bit j set = slot j takes part (prepared on the device from the mask)
+    auto sel_of = [&](long long row) -> uint32_t { return __ldg(p.sel_bits + partition_of(row)); };
     const uint32_t all_bits = (P == 32) ? 0xFFFFFFFFu : ((1u << P) - 1u);
+    // copies for the sources [first, first + count) of the staging order into tile slots 0..count-1
+    auto stage = [&](int first, int count) {
+        mbar_arrive_expect_tx(bar, bytes * (uint32_t)count);
+        for (int k = 0; k < count; ++k) {
+            const int src = (MODE == MERGE_ALL) ? first + k : (int)src_s[first + k];
+            const StateT *g = (src < P) ? static_cast<const StateT *>(p.o_state) + ((long long)src * p.R + row0) * D
+                                        : static_cast<const StateT *>(p.comp_o) + row0 * D;
+            bulk_load(smem_u32(tile + (size_t)k * ROWS * D), g, bytes, bar);
+        }
+    };
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         mbar_init(bar, 1);
         fence_mbar_init();
-        // slots any row of the block needs: one bulk copy each (`valid` consecutive rows of slot j)
-        uint32_t need = all_bits;
-        if (p.mode != MERGE_ALL) {
-            need = 0;
-            for (int r = 0; r < valid; ++r) need |= sel_s[partition_of(row0 + r)];
+        int nsrc = P;
+        if (MODE != MERGE_ALL) {
+            // sources any row of the block needs; its rows are consecutive, so only the partitions of its
+            // two ends and those between them matter
+            uint32_t need = 0;
+            const int i0 = partition_of(row0), i1 = partition_of(row0 + valid - 1);
+            if (valid >= p.L) { for (int i = 0; i < P; ++i) need |= __ldg(p.sel_bits + i); }   // a block longer than the sequence
+            else if (i0 <= i1 && (row0 % p.L) + valid <= p.L) { for (int i = i0; i <= i1; ++i) need |= __ldg(p.sel_bits + i); }
+            else { for (int i = 0; i < P; ++i) if (i >= i0 || i <= i1) need |= __ldg(p.sel_bits + i); }   // wraps into the next (b, h)
+            nsrc = 0;
+            for (int j = 0; j < P; ++j) if (need >> j & 1u) src_s[nsrc++] = (uint8_t)j;
+            if (MODE == MERGE_PLANNED) src_s[nsrc++] = (uint8_t)P;
         }
-        const uint32_t bytes = (uint32_t)valid * Cf::ROW_BYTES;
-        const uint32_t copies = (uint32_t)__popc(need) + (p.mode == MERGE_PLANNED ? 1u : 0u);
-        if (copies > 0) {
-            mbar_arrive_expect_tx(bar, bytes * copies);
-            const StateT *src = static_cast<const StateT *>(p.o_state) + row0 * D;
-            for (int j = 0; j < P; ++j)
-                if (need >> j & 1u) bulk_load(smem_u32(tile + (size_t)j * ROWS * D), src + (long long)j * p.R * D, bytes, bar);
-            if (p.mode == MERGE_PLANNED)
-                bulk_load(smem_u32(tile + (size_t)P * ROWS * D), static_cast<const StateT *>(p.comp_o) + row0 * D, bytes, bar);
-        } else {
-            mbar_arrive(bar);
-        }
+        *nsrc_s = nsrc;
+        if (nsrc > 0) stage(0, min(nsrc, staged));
     }
     // the rows' log-sum-exps, through shared memory so that every thread of a row sees all of them;
     // sources that do not take part get -inf, i.e. weight zero
-    for (int e = threadIdx.x; e < valid * NS; e += MERGE_THREADS) {
-        const int r = e / NS, j = e - r * NS;
+    for (int e = threadIdx.x; e < valid * nslots; e += MERGE_THREADS) {
+        const int r = e / nslots, j = e - r * nslots;
         float x = -INFINITY;
         if (j < P) {
-            const uint32_t sel = (p.mode == MERGE_ALL) ? all_bits : sel_s[partition_of(row0 + r)];
+            const uint32_t sel = (MODE == MERGE_ALL) ? all_bits : sel_of(row0 + r);
             if (sel >> j & 1u) x = __ldg(p.lse_state + (long long)j * p.R + row0 + r);
-        } else if (j == P && p.mode == MERGE_PLANNED) {
+        } else {
             x = __ldg(p.comp_lse + row0 + r);
         }
         lse_s[r * NS + j] = x;
     }
-    __syncthreads();   // also publishes the mbarrier initialisation to the waiting threads
+    __syncthreads();   // also publishes the mbarrier initialisation and the staging order
 
     const int r = threadIdx.x / TPR, lane = threadIdx.x % TPR;
     const bool active = r < valid;
-    float w[NS];
+    const float *my_lse = lse_s + (active ? r : 0) * NS;
     float M = -INFINITY, Z = 0.f;
-    if (active) {
-#pragma unroll
-        for (int j = 0; j < NS; ++j) {
-            w[j] = (j < nslots) ? lse_s[r * NS + j] : -INFINITY;
-            M = fmaxf(M, w[j]);
-        }
-    }
+    for (int j = 0; j < nslots; ++j) M = fmaxf(M, my_lse[j]);
     const bool empty = (M == -INFINITY);   // no source has any mass: output 0, LSE = -inf
-#pragma unroll
-    for (int j = 0; j < NS; ++j) {
-        w[j] = (active && j < nslots && !empty) ? __expf(w[j] - M) : 0.f;
-        Z += w[j];
-    }
-
-    if (!mbar_wait_bounded(bar, 0, abort_flag, MERGE_WAIT_LIMIT)) {
-        if (p.status) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
-        *abort_flag = 1;
-        return;
-    }
-    if (!active) return;
+    if (!empty)
+        for (int j = 0; j < nslots; ++j) Z += __expf(my_lse[j] - M);
 
     float acc[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
-    const StateT *mine = tile + (size_t)r * D + lane * VEC;
+    const int nsrc = *nsrc_s;
+    const StateT *mine = tile + (size_t)(active ? r : 0) * D + lane * VEC;
+    for (int first = 0, phase = 0; first < nsrc; first += staged, phase ^= 1) {
+        const int count = min(nsrc - first, staged);
+        if (first > 0) {          // the tile buffer is reused: everyone must be done with the previous chunk
+            __syncthreads();
+            if (threadIdx.x == 0) stage(first, count);
+        }
+        if (!mbar_wait_bounded(bar, (uint32_t)phase, abort_flag, MERGE_WAIT_LIMIT)) {
+            if (p.status) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
+            *abort_flag = 1;
+            return;
+        }
+        if (active && !empty) {
+#pragma unroll 4
+            for (int k = 0; k < count; ++k) {
+                const int src = (MODE == MERGE_ALL) ? first + k : (int)src_s[first + k];
+                const float wt = __expf(my_lse[src] - M);
+                if (wt != 0.f) {   // rows of another partition may not use this source at all
+                    float v[VEC];
+                    StateVec<StateT>::load(mine + (size_t)k * ROWS * D, v);
 #pragma unroll
-    for (int j = 0; j < NS; ++j) {
-        if (j < nslots && w[j] != 0.f) {   // a source with zero weight may not even have been copied
-            float v[VEC];
-            StateVec<StateT>::load(mine + (size_t)j * ROWS * D, v);
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) acc[e] = fmaf(w[j], v[e], acc[e]);
+                    for (int e = 0; e < VEC; ++e) acc[e] = fmaf(wt, v[e], acc[e]);
+                }
+            }
         }
     }
+    if (!active) return;
     const float inv = empty ? 0.f : 1.f / Z;
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] *= inv;
     const float lse_row = empty ? -INFINITY : M + __logf(Z);
 
     const long long row = row0 + r;
-    if (p.mode == MERGE_COMPOSE) {
+    if (MODE == MERGE_COMPOSE) {
         store_state<VEC>(static_cast<StateT *>(p.comp_o_out) + row * D + lane * VEC, acc);
         if (lane == 0) p.comp_lse_out[row] = lse_row;
         return;
@@ -232,22 +243,44 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(MergeParams 
     if (lane == 0 && p.lse_out != nullptr) p.lse_out[row] = lse_row;
 }
 
-template <typename StateT, int D>
-cudaError_t launch(const MergeParams &p, cudaStream_t stream) {
+template <typename StateT, int D, int MODE>
+cudaError_t launch_mode(const MergeParams &p, cudaStream_t stream) {
     using Cf = MergeCfg<StateT, D>;
-    const int nslots = p.P + (p.mode == MERGE_PLANNED ? 1 : 0);
-    const int rows = Cf::rows(nslots);
-    const size_t smem = Cf::smem_bytes(nslots);
+    const int rows = Cf::rows(MODE, p.P);
+    const size_t smem = Cf::smem_bytes(MODE, p.P);
     const long long blocks = (p.R + rows - 1) / rows;
     if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(state_merge_kernel<StateT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         MERGE_STAGE_BYTES + MERGE_THREADS * (DT_MAX_P + 1) * (int)sizeof(float) + 32);
+    cudaError_t e = cudaFuncSetAttribute(state_merge_kernel<StateT, D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         MERGE_STAGE_BYTES + MERGE_THREADS * (DT_MAX_P + 1) * (int)sizeof(float) + 128);
     if (e != cudaSuccess) return e;
-    state_merge_kernel<StateT, D><<<(unsigned)blocks, MERGE_THREADS, smem, stream>>>(p, rows);
+    state_merge_kernel<StateT, D, MODE><<<(unsigned)blocks, MERGE_THREADS, smem, stream>>>(p, rows);
     return cudaGetLastError();
 }
 
+template <typename StateT, int D>
+cudaError_t launch(const MergeParams &p, cudaStream_t stream) {
+    if (p.mode == MERGE_ALL) return launch_mode<StateT, D, MERGE_ALL>(p, stream);
+    if (p.mode == MERGE_COMPOSE) return launch_mode<StateT, D, MERGE_COMPOSE>(p, stream);
+    return launch_mode<StateT, D, MERGE_PLANNED>(p, stream);
+}
+
+// mask -> per query partition the bit set of slots that take part (REUSE slots for the composition,
+// COMPUTE slots for the planned merge)
+__global__ void merge_select_kernel(const uint8_t *mask, int P, int want_compute, uint32_t *sel_bits) {
+    const int i = threadIdx.x;
+    if (i >= P) return;
+    uint32_t bits = 0;
+    for (int j = 0; j < P; ++j)
+        if ((mask[i * P + j] != 0) == (want_compute != 0)) bits |= 1u << j;
+    sel_bits[i] = bits;
+}
+
 }  // namespace
+
+cudaError_t launch_merge_select(const uint8_t *mask, int P, int want_compute, uint32_t *sel_bits, cudaStream_t stream) {
+    merge_select_kernel<<<1, 32, 0, stream>>>(mask, P, want_compute, sel_bits);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_state_merge(const MergeParams &p, int D, int state_dtype, cudaStream_t stream) {
     if (state_dtype == DT_STATE_FP32) {

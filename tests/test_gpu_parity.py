@@ -210,6 +210,29 @@ def test_composed_reuse_state_and_planned_merge(state_dtype):
     assert (lse2 - run.lse).abs().max().item() <= 5e-3
 
 
+def test_planned_merge_with_sixteen_partitions_odd_rows_per_block():
+    """P = 16 with fp32 states gives 17 sources and 7 rows per block in the planned merge: the shared
+    memory carve-up (tiles, LSEs, mbarrier) must stay aligned for every such combination."""
+    wl = inputs.Workload("p16", 1, 1, 128, (1, 16, 41), 0, 16, 2, 0.05)      # 656 tokens, 41 per partition
+    run = Run(wl, seed=17)
+    run.step(np.ones((16, 16), np.uint8))
+    mask = inputs.banded_mask(16, 2)
+    dev = run.dev
+    mask_dev = torch.from_numpy(mask.reshape(-1).copy()).to(dev)
+    comp_o = torch.empty((wl.B, wl.H, wl.L, wl.D), dtype=torch.float32, device=dev)
+    comp_l = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    run.ctx.dt_compose_reuse(mask_dev, comp_o, comp_l)
+    run.t += 1
+    q, k, v = run.gen.next()
+    run.ctx.dt_attn_states(q, k, v, mask_dev, run.t)
+    run.ctx.dt_state_merge_planned(mask_dev, comp_o, comp_l, run.out, run.lse)
+    torch.cuda.synchronize()
+    run.ctx.dt_poll()
+    outs, lses = run.ses.step(*(inputs.bf16_bits(x) for x in (q, k, v)), mask, run.t)
+    check_o(run.out[0, :, 0].float().cpu().numpy(), outs[(0, 0)], "planned merge P=16")
+    check_lse(run.lse[0, 0].cpu().numpy(), lses[(0, 0)], "planned merge P=16")
+
+
 def _plan_case(wl, lse_host, off, fractions, eps_list):
     """dt_plan on a given LSE cache (fp32 values) against the oracle fed the same values."""
     dev = torch.device("cuda", 0)
