@@ -127,6 +127,17 @@ dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const voi
 dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask_dev, double *w_dev,
                   double *eps_out_dev, void *stream);
 
+/* Group-wise planning (Section 4.2.1-4.2.3): the P KV partitions form ceil(P / group_size) groups of
+ * adjacent partitions; per query partition all states of a group share one decision.  The local
+ * (diagonal) state is handled separately -- always COMPUTE -- so the group that contains it has one
+ * member fewer.  The group's measure is the sum of its members' W (Eq. 12), compared with eps by a strict
+ * '>' (Eq. 13); with target_fraction >= 0 whole groups are taken in order of decreasing measure (ties:
+ * the group nearer to the local one, then the smaller index i * n_groups + k) while their members still
+ * fit into K - P pairs, and eps_out is the midpoint between the last taken and the first not taken
+ * measure.  group_size = 1 is dt_plan.  Other arguments as for dt_plan. */
+dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32_t group_size, uint8_t *mask_dev,
+                          double *w_dev, double *eps_out_dev, void *stream);
+
 /* The same plan computation for callers that cannot allocate device memory at the point of the
  * call: code running inside a region where the allocator must stay untouched (a fixed-memory
  * serving process that sized its pools up front, a callback on a latency-critical path, a host that

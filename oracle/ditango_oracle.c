@@ -287,3 +287,76 @@ int orc_target_fraction(const double *W, int P, double f, uint8_t *mask, double 
     free(rk);
     return K;
 }
+
+/*
+ * Group-wise organisation (Section 4.2.1-4.2.3): the P KV partitions are divided into contiguous groups
+ * of g; all states of a group share one decision per query partition i, the local (diagonal) state is
+ * handled separately (always computed), so the group that contains it has one member fewer.  The group
+ * measure is the sum of its members' measures (Eq. 12), thresholded with a strict '>' (Eq. 13).
+ *   unit (i, k): members j in [k g, min(P, (k+1) g)), j != i;   m(i,k) = sum_j W[i][j]
+ * target_fraction < 0: COMPUTE iff m > eps.
+ * target_fraction >= 0: K = round(f P^2) clipped to [P, P^2]; units are ranked by m (ties: smaller
+ *   |k - floor(i/g)|, then smaller i * n_groups + k) and taken in that order while the pairs selected so
+ *   far plus the unit's members still fit into K - P; eps = midpoint between the last taken and the first
+ *   not taken measure (0 if all are taken, the largest measure if none is).
+ * With g = 1 this is exactly orc_threshold / orc_target_fraction.  Returns the number of COMPUTE pairs.
+ */
+typedef struct { double m; int dist; int flat; int size; int i; int k; } orc_unit_t;
+
+static int orc_unit_cmp(const void *pa, const void *pb) {
+    const orc_unit_t *a = (const orc_unit_t *)pa, *b = (const orc_unit_t *)pb;
+    if (a->m != b->m) return a->m > b->m ? -1 : 1;
+    if (a->dist != b->dist) return a->dist - b->dist;
+    return a->flat - b->flat;
+}
+
+int orc_group_plan(const double *W, int P, int g, double eps, double target_fraction, uint8_t *mask,
+                   double *eps_out) {
+    if (g < 1) g = 1;
+    int ng = (P + g - 1) / g;
+    orc_unit_t *u = (orc_unit_t *)malloc((size_t)P * ng * sizeof(orc_unit_t));
+    int n = 0;
+    for (int i = 0; i < P; ++i)
+        for (int k = 0; k < ng; ++k) {
+            int lo = k * g, hi = (k + 1) * g < P ? (k + 1) * g : P;
+            double m = 0.0;
+            int size = 0;
+            for (int j = lo; j < hi; ++j)
+                if (j != i) { m += W[i * P + j]; ++size; }
+            if (size == 0) continue;
+            int gi = i / g;
+            u[n].m = m; u[n].dist = k > gi ? k - gi : gi - k; u[n].flat = i * ng + k; u[n].size = size;
+            u[n].i = i; u[n].k = k;
+            ++n;
+        }
+    for (int e = 0; e < P * P; ++e) mask[e] = 0;
+    for (int i = 0; i < P; ++i) mask[i * P + i] = 1;
+    int count = P;
+    double eps_used = eps;
+    if (target_fraction < 0) {
+        for (int s = 0; s < n; ++s)
+            if (u[s].m > eps) {
+                for (int j = u[s].k * g; j < (u[s].k + 1) * g && j < P; ++j)
+                    if (j != u[s].i) { mask[u[s].i * P + j] = 1; ++count; }
+            }
+    } else {
+        int total = P * P;
+        int K = (int)floor(target_fraction * total + 0.5);
+        if (K < P) K = P;
+        if (K > total) K = total;
+        qsort(u, (size_t)n, sizeof(orc_unit_t), orc_unit_cmp);
+        int budget = K - P, used = 0, taken = 0;
+        while (taken < n && used + u[taken].size <= budget) {
+            for (int j = u[taken].k * g; j < (u[taken].k + 1) * g && j < P; ++j)
+                if (j != u[taken].i) { mask[u[taken].i * P + j] = 1; ++count; }
+            used += u[taken].size;
+            ++taken;
+        }
+        if (n == 0 || taken == n) eps_used = 0.0;
+        else if (taken == 0) eps_used = u[0].m;
+        else eps_used = 0.5 * (u[taken - 1].m + u[taken].m);
+    }
+    *eps_out = eps_used;
+    free(u);
+    return count;
+}

@@ -41,6 +41,8 @@ def lib():
         L.orc_threshold.argtypes = [f64p, C.c_int, C.c_double, u8p]
         L.orc_target_fraction.restype = C.c_int
         L.orc_target_fraction.argtypes = [f64p, C.c_int, C.c_double, u8p, f64p]
+        L.orc_group_plan.restype = C.c_int
+        L.orc_group_plan.argtypes = [f64p, C.c_int, C.c_int, C.c_double, C.c_double, u8p, f64p]
         _lib = L
     return _lib
 
@@ -146,6 +148,18 @@ def target_fraction(W, f):
     eps = C.c_double()
     K = lib().orc_target_fraction(_p(W, C.c_double), P, float(f), _p(mask, C.c_uint8), C.byref(eps))
     return mask, eps.value, int(K)
+
+
+def group_plan(W, g, eps=0.0, target_fraction=-1.0):
+    """Group-wise decisions (Section 4.2.1-4.2.3): one decision per (query partition, group of g KV
+    partitions), diagonal always computed.  Returns (mask, eps_used, computed_pairs)."""
+    W = np.ascontiguousarray(W, dtype=np.float64)
+    P = W.shape[0]
+    mask = np.empty((P, P), dtype=np.uint8)
+    eps_out = C.c_double()
+    n = lib().orc_group_plan(_p(W, C.c_double), P, int(g), float(eps), float(target_fraction), _p(mask, C.c_uint8),
+                             C.byref(eps_out))
+    return mask, eps_out.value, int(n)
 
 
 def uniform_offsets(L, P):

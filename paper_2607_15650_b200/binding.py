@@ -20,7 +20,7 @@ DT_MAX_P = 32
 
 EXPORTS = [
     "dt_create", "dt_destroy", "dt_cache_bytes", "dt_bind_cache", "dt_attn_states", "dt_state_merge",
-    "dt_compose_reuse", "dt_state_merge_planned", "dt_plan", "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
+    "dt_compose_reuse", "dt_state_merge_planned", "dt_plan", "dt_plan_grouped", "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
     "dt_launch_count", "dt_selftest_wait_timeout", "dt_poll", "dt_status_str", "dt_last_error",
 ]
 
@@ -62,6 +62,7 @@ def lib():
         "dt_compose_reuse": (C.c_int, [vp, u8p, vp, f32p, vp]),
         "dt_state_merge_planned": (C.c_int, [vp, u8p, vp, f32p, vp, i64p, f32p, vp]),
         "dt_plan": (C.c_int, [vp, C.c_double, C.c_double, u8p, f64p, f64p, vp]),
+        "dt_plan_grouped": (C.c_int, [vp, C.c_double, C.c_double, C.c_int32, u8p, f64p, f64p, vp]),
         "dt_plan_static": (C.c_int, [f32p, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_double,
                            u8p, f64p, f64p, vp]),
         "dt_step_host_workspace_bytes": (C.c_int, [C.POINTER(dt_config), szp]),
@@ -199,6 +200,13 @@ class Context:
         self._check(lib().dt_state_merge_planned(self._h, C.c_void_p(mask_dev.data_ptr()), C.c_void_p(comp_o.data_ptr()),
                                                  C.c_void_p(comp_lse.data_ptr()), C.c_void_p(out.data_ptr()),
                                                  _strides4(out), lp, _stream_ptr(stream)))
+
+    def dt_plan_grouped(self, mask_dev, group_size, eps=0.0, target_fraction=-1.0, w_dev=None, eps_out_dev=None,
+                        stream=None):
+        wp = C.c_void_p(w_dev.data_ptr()) if w_dev is not None else C.c_void_p()
+        ep = C.c_void_p(eps_out_dev.data_ptr()) if eps_out_dev is not None else C.c_void_p()
+        self._check(lib().dt_plan_grouped(self._h, float(eps), float(target_fraction), int(group_size),
+                                          C.c_void_p(mask_dev.data_ptr()), wp, ep, _stream_ptr(stream)))
 
     def dt_plan(self, mask_dev, eps=0.0, target_fraction=-1.0, w_dev=None, eps_out_dev=None, stream=None):
         assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()

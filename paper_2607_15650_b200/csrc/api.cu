@@ -294,7 +294,13 @@ dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const voi
 
 dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask_dev, double *w_dev,
                   double *eps_out_dev, void *stream) {
+    return dt_plan_grouped(ctx, eps, target_fraction, 1, mask_dev, w_dev, eps_out_dev, stream);
+}
+
+dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32_t group_size, uint8_t *mask_dev,
+                          double *w_dev, double *eps_out_dev, void *stream) {
     if (!ctx) return DT_ERR_INVALID_ARG;
+    if (group_size < 1 || group_size > ctx->cfg.P) return fail(ctx, DT_ERR_INVALID_ARG, "group_size must be in [1, P]");
     if (!mask_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null mask pointer");
     if (!ctx->lse_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
     if (target_fraction < 0 && !std::isfinite(eps)) return fail(ctx, DT_ERR_INVALID_ARG, "eps must be finite");
@@ -318,6 +324,7 @@ dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask
     int K = (int)std::floor(target_fraction * total + 0.5);
     K = std::min(std::max(K, c.P), total);
     pf.K = K;
+    pf.group_size = group_size;
     pf.eps = eps;
     pf.mask = mask_dev;
     pf.w_out = w_dev;

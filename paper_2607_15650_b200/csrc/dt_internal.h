@@ -63,6 +63,7 @@ struct PlanFinalParams {
     int P, BH, chunks;
     int mode_target;   // 0: threshold with eps; 1: select K pairs by rank
     int K;
+    int group_size;    // g adjacent KV partitions share one decision (1 = per pair)
     double eps;
     uint8_t *mask;
     double *w_out;     // may be null

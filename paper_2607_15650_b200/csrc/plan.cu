@@ -67,57 +67,92 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_partial_kernel(PlanParams p
     }
 }
 
-// Strict total order used to rank off-diagonal pairs: larger W first, then smaller |i-j|, then
-// smaller flat index.
-__device__ __forceinline__ bool ranks_before(double wa, int da, int fa, double wb, int db, int fb) {
-    if (wa != wb) return wa > wb;
+// Strict total order used to rank decision units: larger measure first, then smaller group distance,
+// then smaller flat index.
+__device__ __forceinline__ bool ranks_before(double ma, int da, int fa, double mb, int db, int fb) {
+    if (ma != mb) return ma > mb;
     if (da != db) return da < db;
     return fa < fb;
 }
 
+// Stage 2.  W[i][j] from the partial sums, then one decision per unit (i, k): query partition i and the
+// k-th group of g adjacent KV partitions without the local one (Section 4.2.1; g = 1: single pairs).
+// Unit measure = sum of its members' W (Eq. 12); COMPUTE iff measure > eps (Eq. 13), or the units of
+// largest measure taken in rank order while their members fit into K - P pairs.
 __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
     __shared__ double W[DT_MAX_P * DT_MAX_P];
+    __shared__ double m_s[DT_MAX_P * DT_MAX_P];
+    __shared__ uint8_t size_s[DT_MAX_P * DT_MAX_P];
+    __shared__ uint8_t dec_s[DT_MAX_P * DT_MAX_P];
     __shared__ double edge[2];
-    const int P = p.P, total = P * P;
+    const int P = p.P, total = P * P, g = p.group_size;
+    const int ng = (P + g - 1) / g, nunits = P * ng;
     const int e = threadIdx.x;
-    const int i = e / P, j = e - i * P;
-    if (e < total) {
-        double s = 0.0;
-        for (int bh = 0; bh < p.BH; ++bh)
-            for (int c = 0; c < p.chunks; ++c) s += (double)p.partials[(((long long)bh * P + i) * p.chunks + c) * P + j];
-        const double cnt = (double)p.BH * (double)(p.off[i + 1] - p.off[i]);
-        W[e] = s / cnt;
-        if (p.w_out) p.w_out[e] = W[e];
+    {
+        const int i = e / P, j = e - i * P;
+        if (e < total) {
+            double s = 0.0;
+            for (int bh = 0; bh < p.BH; ++bh)
+                for (int c = 0; c < p.chunks; ++c) s += (double)p.partials[(((long long)bh * P + i) * p.chunks + c) * P + j];
+            const double cnt = (double)p.BH * (double)(p.off[i + 1] - p.off[i]);
+            W[e] = s / cnt;
+            if (p.w_out) p.w_out[e] = W[e];
+        }
     }
     if (e < 2) edge[e] = 0.0;
     __syncthreads();
-    if (!p.mode_target) {
-        if (e < total) p.mask[e] = (i == j || W[e] > p.eps) ? 1 : 0;
-        if (e == 0 && p.eps_out) *p.eps_out = p.eps;
-        return;
+    // unit e = (ui, uk)
+    const int ui = e / ng, uk = e - ui * ng;
+    double m = 0.0;
+    int size = 0, dist = 0;
+    if (e < nunits) {
+        const int lo = uk * g, hi = min(P, (uk + 1) * g);
+        for (int j = lo; j < hi; ++j)
+            if (j != ui) { m += W[ui * P + j]; ++size; }
+        const int gi = ui / g;
+        dist = uk > gi ? uk - gi : gi - uk;
+        m_s[e] = m;
+        size_s[e] = (uint8_t)size;
     }
-    const int noff = total - P, sel = p.K - P;
+    __syncthreads();
+    bool take = false;
     int rank = -1;
-    if (e < total && i != j) {
-        rank = 0;
-        const double w = W[e];
-        const int d = i > j ? i - j : j - i;
-        for (int o = 0; o < total; ++o) {
-            const int oi = o / P, oj = o - oi * P;
-            if (oi == oj || o == e) continue;
-            const int od = oi > oj ? oi - oj : oj - oi;
-            if (ranks_before(W[o], od, o, w, d, e)) ++rank;
+    const int budget = p.K - P;
+    if (e < nunits && size > 0) {
+        if (!p.mode_target) {
+            take = m > p.eps;
+        } else {
+            rank = 0;
+            int cum = size;
+            for (int o = 0; o < nunits; ++o) {
+                if (o == e || size_s[o] == 0) continue;
+                const int oi = o / ng, ok = o - oi * ng, ogi = oi / g;
+                const int od = ok > ogi ? ok - ogi : ogi - ok;
+                if (ranks_before(m_s[o], od, o, m, dist, e)) { ++rank; cum += size_s[o]; }
+            }
+            take = cum <= budget;
         }
-        if (rank == sel - 1) edge[0] = w;
-        if (rank == sel) edge[1] = w;
     }
-    if (e < total) p.mask[e] = (i == j || (rank >= 0 && rank < sel)) ? 1 : 0;
+    if (e < nunits) dec_s[e] = take ? 1 : 0;
+    const int taken = __syncthreads_count(take);
+    if (p.mode_target && rank >= 0) {
+        if (rank == taken - 1) edge[0] = m;
+        if (rank == taken) edge[1] = m;
+    }
+    if (e < total) {
+        const int i = e / P, j = e - i * P;
+        p.mask[e] = (i == j || dec_s[i * ng + j / g]) ? 1 : 0;
+    }
     __syncthreads();
     if (e == 0 && p.eps_out) {
-        double eps;
-        if (noff == 0 || sel == noff) eps = 0.0;
-        else if (sel == 0) eps = edge[1];
-        else eps = 0.5 * (edge[0] + edge[1]);
+        double eps = p.eps;
+        if (p.mode_target) {
+            int n = 0;
+            for (int o = 0; o < nunits; ++o) n += size_s[o] > 0;
+            if (n == 0 || taken == n) eps = 0.0;
+            else if (taken == 0) eps = edge[1];
+            else eps = 0.5 * (edge[0] + edge[1]);
+        }
         *p.eps_out = eps;
     }
 }
@@ -259,6 +294,7 @@ extern "C" dt_status dt_plan_static(const float *lse_state_dev, const int32_t *p
     int K = (int)floor(target_fraction * total + 0.5);
     K = K < P ? P : (K > total ? total : K);
     pf.K = K;
+    pf.group_size = 1;
     pf.eps = eps;
     pf.mask = mask_dev;
     pf.w_out = w_dev;

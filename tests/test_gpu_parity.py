@@ -291,6 +291,40 @@ def test_plan_on_synthetic_lse_uneven_partitions():
     _plan_case(wl, lse, off, [0.0, 0.2, 0.4, 0.52, 0.8, 1.0], [0.05, 0.2, 0.5])
 
 
+@pytest.mark.parametrize("P,g", [(8, 2), (8, 4), (12, 5), (32, 8), (6, 6)])
+def test_grouped_plan_matches_oracle_rule(P, g):
+    """dt_plan_grouped against the oracle's group rule applied to the GPU's own W (same fp64 decision),
+    in threshold and target-fraction mode, for group sizes that do and do not divide P."""
+    rng = np.random.default_rng(100 + P + g)
+    L = 40 * P
+    wl = inputs.Workload("grp", 1, 2, 64, (1, 1, L), 0, P, 1, 0.05)
+    off = wl.offsets()
+    dev = torch.device("cuda", 0)
+    part = np.searchsorted(off, np.arange(L), side="right") - 1
+    dist = np.abs(np.subtract.outer(np.arange(P), np.arange(P)))
+    lse = rng.standard_normal((P, wl.B, wl.H, L)) * 0.6
+    for j in range(P):
+        lse[j] += -0.7 * dist[part, j]
+    ctx = binding.Context(wl.B, wl.H, wl.D, L, off, wl.scale, alloc_cache=False)
+    ctx.dt_bind_cache(torch.empty((P, wl.B, wl.H, L, wl.D), device=dev), torch.from_numpy(lse.astype(np.float32)).to(dev))
+    mask = torch.empty(P * P, dtype=torch.uint8, device=dev)
+    W = torch.empty(P * P, dtype=torch.float64, device=dev)
+    eps_out = torch.empty(1, dtype=torch.float64, device=dev)
+    for f in (0.0, 0.25, 0.4, 0.7, 1.0):
+        ctx.dt_plan_grouped(mask, g, target_fraction=f, w_dev=W, eps_out_dev=eps_out)
+        torch.cuda.synchronize()
+        Wg = W.cpu().numpy().reshape(P, P)
+        ref_mask, ref_eps, n = orc.group_plan(Wg, g, target_fraction=f)
+        got = mask.cpu().numpy().reshape(P, P)
+        assert (got == ref_mask).all() and got.sum() == n and eps_out.item() == ref_eps
+    for eps in (0.02, 0.1, 0.3):
+        ctx.dt_plan_grouped(mask, g, eps=eps, w_dev=W, eps_out_dev=eps_out)
+        torch.cuda.synchronize()
+        Wg = W.cpu().numpy().reshape(P, P)
+        ref_mask, _, _ = orc.group_plan(Wg, g, eps=eps)
+        assert (mask.cpu().numpy().reshape(P, P) == ref_mask).all() and eps_out.item() == eps
+
+
 def test_plan_threshold_equality_is_reuse():
     """W exactly equal to eps must give REUSE (strict '>'): constant LSEs give W = 1/P exactly."""
     wl = inputs.Workload("eq", 1, 1, 64, (1, 1, 64), 0, 4, 1, 0.05)

@@ -388,6 +388,62 @@ def test_target_fraction_banded_measure_gives_banded_mask_and_tie_rule():
     assert mask1.sum() == P + 1 and mask1[0, 1] == 1
 
 
+def test_group_plan_with_group_size_one_is_the_ungrouped_rule():
+    """g = 1: every unit is a single off-diagonal pair, so the grouped rule must reproduce Eq. 13 and
+    the target-fraction selection exactly."""
+    rng = np.random.default_rng(15)
+    P = 7
+    W = rng.random((P, P)); W /= W.sum(1, keepdims=True)
+    for eps in (0.05, 0.12, 0.3):
+        m, e, n = orc.group_plan(W, 1, eps=eps)
+        assert (m == orc.threshold(W, eps)).all() and e == eps and n == m.sum()
+    for f in (0.0, 0.3, 0.5, 0.9, 1.0):
+        m, e, n = orc.group_plan(W, 1, target_fraction=f)
+        m2, e2, K = orc.target_fraction(W, f)
+        assert (m == m2).all() and e == e2 and n == K
+
+
+def test_group_plan_shares_one_decision_per_group_and_handles_the_local_state_separately():
+    """Section 4.2.1: p/g groups of g adjacent states share one decision; the local state is always
+    computed and the group that contains it has g - 1 members.  Measure = sum over the group (Eq. 12)."""
+    P, g = 8, 4
+    d = np.abs(np.subtract.outer(np.arange(P), np.arange(P))).astype(float)
+    W = np.exp(-0.8 * d); W /= W.sum(1, keepdims=True)
+    m, eps, n = orc.group_plan(W, g, eps=0.25)
+    for i in range(P):
+        for k in range(P // g):
+            members = [j for j in range(k * g, (k + 1) * g) if j != i]
+            assert len(set(m[i, members].tolist())) == 1                         # shared decision
+            assert m[i, members[0]] == int(W[i, members].sum() > 0.25)           # Eq. 12 + Eq. 13
+            assert len(members) == (g - 1 if i // g == k else g)
+    assert (m.diagonal() == 1).all() and n == m.sum()
+    # strictness at equality: a measure exactly equal to eps is REUSE
+    W2 = np.full((4, 4), 0.25)
+    m2, _, _ = orc.group_plan(W2, 2, eps=0.5)      # remote groups sum to exactly 0.5
+    assert (m2 == np.eye(4)).all()
+    m3, _, _ = orc.group_plan(W2, 2, eps=0.2)      # local groups (one member, 0.25) and remote ones (0.5) exceed it
+    assert m3.all()
+
+
+def test_group_plan_target_fraction_takes_whole_groups_in_rank_order():
+    P, g = 8, 2
+    d = np.abs(np.subtract.outer(np.arange(P), np.arange(P))).astype(float)
+    W = np.exp(-1.1 * d) * (1.0 + 0.02 * np.random.default_rng(16).random((P, P)))   # no tied measures
+    W /= W.sum(1, keepdims=True)
+    prev = None
+    for f in (0.125, 0.3, 0.5, 0.75, 1.0):
+        m, eps, n = orc.group_plan(W, g, target_fraction=f)
+        K = min(max(int(np.floor(f * P * P + 0.5)), P), P * P)
+        assert n == m.sum() and P <= n <= K and (m.diagonal() == 1).all()
+        # thresholding the group measures at the reported eps reproduces the selection
+        m_thr, _, _ = orc.group_plan(W, g, eps=eps)
+        assert (m_thr == m).all()
+        if prev is not None:
+            assert (m >= prev).all()
+        prev = m
+    assert orc.group_plan(W, g, target_fraction=1.0)[0].all()
+
+
 def test_uniform_offsets():
     off = orc.uniform_offsets(32760, 16)
     assert off[0] == 0 and off[-1] == 32760
