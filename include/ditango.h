@@ -87,6 +87,13 @@ dt_status dt_bind_cache(dt_ctx *ctx, void *o_state_dev, float *lse_state_dev, si
 dt_status dt_attn_states(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
                          const int64_t strides_blhd[4], const uint8_t *mask_dev, int32_t step, void *stream);
 
+/* The local (diagonal) pairs only -- Algorithm 1's first line of a step ("compute local attention"): the
+ * states AS_t(i, i) that the planner's drift estimate needs before the plan of the step exists.  Same
+ * tensors as dt_attn_states; no mask, and no REUSE check (the other pairs of the step are decided and
+ * launched afterwards with dt_attn_states). */
+dt_status dt_attn_local(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
+                        const int64_t strides_blhd[4], int32_t step, void *stream);
+
 /* Eq. 2 folded over all P cached states of each query row (fresh or reused alike):
  *   LSE[r] = log sum_j exp(LSE_ij[r]),  OUT[r] = sum_j exp(LSE_ij[r] - LSE[r]) OUT_ij[r].
  *   out_dev        device, bf16, logical [B, L, H, D] with out_strides_blhd (elements; D stride 1,
@@ -137,6 +144,44 @@ dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask
  * measure.  group_size = 1 is dt_plan.  Other arguments as for dt_plan. */
 dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32_t group_size, uint8_t *mask_dev,
                           double *w_dev, double *eps_out_dev, void *stream);
+
+/* Anchor-guided selection planning, Algorithm 1 (Section 4), with its state on the device.
+ *   partition importance  w(i,j)      Eq. 8, refreshed at anchors from the cached LSEs
+ *   scale ratio           alpha(i,j)  Eq. 9: ||AS_ta(i,j)||_2 / ||AS_ta(i,i)||_2, the state being OUT and LSE
+ *                                     stacked over all rows and heads of query partition i
+ *   age penalty           delta(i,j,t) = alpha(i,j) * ||AS_t(i,i) - AS_ta(i,i)||_2            (Eq. 10)
+ *   unit error            ASE(i,G,t) = sum_{j in G, j != i} w(i,j) * delta(i,j,t)            (Eq. 7, Eq. 12)
+ *   decision              COMPUTE iff ASE > eps (Eq. 13); anchor iff every unit exceeds eps or the relative
+ *                         drift of the local states exceeds eps_local (Eq. 14); the first step is an anchor
+ *   eps update            at an anchor, eps becomes the cache_ratio-quantile of the units' predicted ASE of that
+ *                         step (unchanged if they are all zero), so that about that fraction of the units is
+ *                         reused under a comparable drift
+ * Use per denoising step t:
+ *   1. dt_attn_local(q, k, v, t)                              the local states AS_t(i,i)
+ *   2. dt_planner_step(...)                                   mask of the step (diagonal included), anchor flag
+ *   3. dt_attn_states(q, k, v, that mask with the diagonal cleared, t)   -- or the whole mask again
+ *   4. dt_state_merge(...)
+ *   5. dt_planner_commit(...)                                 on an anchor: w, alpha and the snapshot of the local
+ *                                                             states are refreshed; otherwise nothing changes
+ * Everything is stream-ordered; the anchor decision stays on the device (steps 3-5 read it there).
+ *   snap_o_dev / snap_lse_dev   caller-owned device buffers of one cache slot ([B][H][L][D] in the cache's state
+ *                               dtype, [B][H][L] fp32): the local states of the last anchor
+ *   mask_dev        device, uint8 [P*P], written           is_anchor_dev  device, int32 [1] or NULL
+ *   ase_dev         device, double [P * ceil(P/group_size)] (NaN for a unit without members) or NULL
+ *   delta_rel_dev   device, double [1] or NULL */
+typedef struct {
+    int32_t group_size;   /* g of Section 4.2.1 (1 = per pair)                         */
+    double eps_initial;   /* eps until the first update                                */
+    double eps_local;     /* threshold on the relative drift of the local states (> 0) */
+    double cache_ratio;   /* R of Algorithm 1: fraction of units to reuse, in [0, 1]   */
+} dt_planner_config;
+dt_status dt_planner_init(dt_ctx *ctx, const dt_planner_config *pc, void *snap_o_dev, float *snap_lse_dev,
+                          size_t snap_o_bytes, size_t snap_lse_bytes, void *stream);
+dt_status dt_planner_step(dt_ctx *ctx, uint8_t *mask_dev, int32_t *is_anchor_dev, double *ase_dev, double *delta_rel_dev,
+                          void *stream);
+dt_status dt_planner_commit(dt_ctx *ctx, void *stream);
+/* Copy the planner state to the host (synchronises): w and alpha are double [P*P]; any pointer may be NULL. */
+dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double *eps_host, int32_t *have_anchor_host);
 
 /* The same plan computation for callers that cannot allocate device memory at the point of the
  * call: code running inside a region where the allocator must stay untouched (a fixed-memory

@@ -213,3 +213,74 @@ class OracleSession:
             outs[bh], lses[bh] = merge(self.o[bh], self.lse[bh])
         self.tc[mask.astype(bool)] = t
         return outs, lses
+
+
+# --------------------------------------------------------------------------------------------------
+# Anchor-guided selection planning (Section 4; Algorithm 1), in plain numpy fp64.
+#
+# Readings where the paper is silent (also listed in the design doc):
+#   * ||AS||_2 (Eq. 9, Eq. 10) is the 2-norm of OUT and LSE stacked, taken over all rows and heads of the
+#     query partition;
+#   * delta(j, t, t_c) is evaluated against the last anchor for every state (Eq. 10 defines it only for
+#     t_a), t_c is bookkeeping;
+#   * delta_local(t) of Eq. 14 is the relative change of the local states over all query partitions:
+#     sqrt(sum_i ||AS_t(i,i) - AS_ta(i,i)||^2) / sqrt(sum_i ||AS_ta(i,i)||^2);
+#   * "update eps based on R and anchor errors": eps becomes the R-quantile of the units' predicted ASE at
+#     the step that turned into an anchor (fraction R of the units would have been reused under that
+#     drift); it is left unchanged when those values are all zero (the very first anchor);
+#   * the first step is an anchor.
+# These parts are pinned only by closed forms and invariants ("parity unpinned" for the readings).
+
+def state_norm_sq(o, lse):
+    """||AS||_2^2 of a set of rows: OUT [n, D] and LSE [n] stacked (Eq. 1's AS)."""
+    o = np.asarray(o, dtype=np.float64); lse = np.asarray(lse, dtype=np.float64)
+    return float((o * o).sum() + (lse * lse).sum())
+
+
+def scale_ratios(norm_sq):
+    """Eq. 9: alpha(i, j) = ||AS_ta(i, j)||_2 / ||AS_ta(i, i_loc)||_2 with the local state on the diagonal."""
+    n = np.asarray(norm_sq, dtype=np.float64)
+    return np.sqrt(n / np.diag(n)[:, None])
+
+
+def planner_step(W, alpha, drift_sq, anchor_local_sq, g, eps, eps_local, R, have_anchor):
+    """One pass of Algorithm 1 given this step's local states.
+    drift_sq[i] = ||AS_t(i,i) - AS_ta(i,i)||^2, anchor_local_sq[i] = ||AS_ta(i,i)||^2.
+    Returns dict(is_anchor, mask [P,P] uint8 with the diagonal set, ase [P, n_groups] (nan where a unit
+    has no member), eps (possibly updated), delta_rel)."""
+    W = np.asarray(W, dtype=np.float64); alpha = np.asarray(alpha, dtype=np.float64)
+    P = W.shape[0]
+    g = max(1, int(g))
+    ng = (P + g - 1) // g
+    delta = np.sqrt(np.asarray(drift_sq, dtype=np.float64))
+    ase = np.full((P, ng), np.nan)
+    for i in range(P):
+        for k in range(ng):
+            members = [j for j in range(k * g, min(P, (k + 1) * g)) if j != i]
+            if members:
+                s = 0.0
+                for j in members:                                  # Eq. 7, Eq. 10, Eq. 12
+                    s += W[i, j] * alpha[i, j] * delta[i]
+                ase[i, k] = s
+    valid = ~np.isnan(ase)
+    vals = ase[valid]
+    den = float(np.sum(anchor_local_sq))
+    delta_rel = float(np.sqrt(np.sum(drift_sq) / den)) if den > 0 else 0.0
+    all_exceed = bool(vals.size > 0 and (vals > eps).all())
+    local_drift = delta_rel > eps_local
+    is_anchor = (not have_anchor) or all_exceed or local_drift      # Eq. 14; the first step is an anchor
+    mask = np.eye(P, dtype=np.uint8)
+    eps_new = eps
+    if is_anchor:
+        mask[:] = 1
+        if vals.size > 0 and vals.max() > 0.0:
+            a = np.sort(vals)
+            r = int(np.floor(R * a.size))
+            r = min(max(r, 0), a.size)
+            eps_new = 0.0 if r == 0 else (float(a[-1]) if r == a.size else 0.5 * float(a[r - 1] + a[r]))
+    else:
+        for i in range(P):
+            for j in range(P):
+                if i != j and ase[i, j // g] > eps:                # Eq. 13, strict
+                    mask[i, j] = 1
+    return dict(is_anchor=bool(is_anchor), mask=mask, ase=ase, eps=float(eps_new), delta_rel=delta_rel)

@@ -19,8 +19,9 @@ DT_STATE_FP32, DT_STATE_BF16 = 0, 1
 DT_MAX_P = 32
 
 EXPORTS = [
-    "dt_create", "dt_destroy", "dt_cache_bytes", "dt_bind_cache", "dt_attn_states", "dt_state_merge",
-    "dt_compose_reuse", "dt_state_merge_planned", "dt_plan", "dt_plan_grouped", "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
+    "dt_create", "dt_destroy", "dt_cache_bytes", "dt_bind_cache", "dt_attn_states", "dt_attn_local", "dt_state_merge",
+    "dt_compose_reuse", "dt_state_merge_planned", "dt_plan", "dt_plan_grouped", "dt_planner_init", "dt_planner_step", "dt_planner_commit", "dt_planner_get",
+    "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
     "dt_launch_count", "dt_selftest_wait_timeout", "dt_poll", "dt_status_str", "dt_last_error",
 ]
 
@@ -29,6 +30,11 @@ class dt_config(C.Structure):
     _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("L", C.c_int32), ("P", C.c_int32),
                 ("part_offsets", C.POINTER(C.c_int32)), ("softmax_scale", C.c_float),
                 ("state_dtype", C.c_int32), ("device", C.c_int32)]
+
+
+class dt_planner_config(C.Structure):
+    _fields_ = [("group_size", C.c_int32), ("eps_initial", C.c_double), ("eps_local", C.c_double),
+                ("cache_ratio", C.c_double)]
 
 
 class DitangoError(RuntimeError):
@@ -58,11 +64,16 @@ def lib():
         "dt_cache_bytes": (C.c_int, [C.POINTER(dt_config), szp, szp]),
         "dt_bind_cache": (C.c_int, [vp, vp, f32p, C.c_size_t, C.c_size_t]),
         "dt_attn_states": (C.c_int, [vp, vp, vp, vp, i64p, u8p, C.c_int32, vp]),
+        "dt_attn_local": (C.c_int, [vp, vp, vp, vp, i64p, C.c_int32, vp]),
         "dt_state_merge": (C.c_int, [vp, vp, i64p, f32p, vp]),
         "dt_compose_reuse": (C.c_int, [vp, u8p, vp, f32p, vp]),
         "dt_state_merge_planned": (C.c_int, [vp, u8p, vp, f32p, vp, i64p, f32p, vp]),
         "dt_plan": (C.c_int, [vp, C.c_double, C.c_double, u8p, f64p, f64p, vp]),
         "dt_plan_grouped": (C.c_int, [vp, C.c_double, C.c_double, C.c_int32, u8p, f64p, f64p, vp]),
+        "dt_planner_init": (C.c_int, [vp, C.POINTER(dt_planner_config), vp, f32p, C.c_size_t, C.c_size_t, vp]),
+        "dt_planner_step": (C.c_int, [vp, u8p, vp, f64p, f64p, vp]),
+        "dt_planner_commit": (C.c_int, [vp, vp]),
+        "dt_planner_get": (C.c_int, [vp, f64p, f64p, f64p, vp]),
         "dt_plan_static": (C.c_int, [f32p, i32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_double,
                            u8p, f64p, f64p, vp]),
         "dt_step_host_workspace_bytes": (C.c_int, [C.POINTER(dt_config), szp]),
@@ -181,6 +192,12 @@ class Context:
                                          C.c_void_p(v.data_ptr()), _strides4(q), C.c_void_p(mask_dev.data_ptr()),
                                          int(step), _stream_ptr(stream)))
 
+    def dt_attn_local(self, q, k, v, step, stream=None):
+        assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and q.is_cuda
+        assert q.stride() == k.stride() == v.stride() and q.shape == k.shape == v.shape
+        self._check(lib().dt_attn_local(self._h, C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()),
+                                        C.c_void_p(v.data_ptr()), _strides4(q), int(step), _stream_ptr(stream)))
+
     def dt_state_merge(self, out, lse_out=None, stream=None):
         assert out.dtype == torch.bfloat16 and out.is_cuda
         lp = C.c_void_p(lse_out.data_ptr()) if lse_out is not None else C.c_void_p()
@@ -200,6 +217,30 @@ class Context:
         self._check(lib().dt_state_merge_planned(self._h, C.c_void_p(mask_dev.data_ptr()), C.c_void_p(comp_o.data_ptr()),
                                                  C.c_void_p(comp_lse.data_ptr()), C.c_void_p(out.data_ptr()),
                                                  _strides4(out), lp, _stream_ptr(stream)))
+
+    def dt_planner_init(self, snap_o, snap_lse, group_size=1, eps_initial=0.0, eps_local=0.1, cache_ratio=0.5, stream=None):
+        assert snap_o.is_cuda and snap_o.is_contiguous() and snap_o.dtype == self.o_state.dtype
+        assert snap_lse.is_cuda and snap_lse.is_contiguous() and snap_lse.dtype == torch.float32
+        pc = dt_planner_config(int(group_size), float(eps_initial), float(eps_local), float(cache_ratio))
+        self._check(lib().dt_planner_init(self._h, C.byref(pc), C.c_void_p(snap_o.data_ptr()), C.c_void_p(snap_lse.data_ptr()),
+                                          snap_o.numel() * snap_o.element_size(), snap_lse.numel() * 4, _stream_ptr(stream)))
+        self._snap = (snap_o, snap_lse)
+
+    def dt_planner_step(self, mask_dev, is_anchor_dev=None, ase_dev=None, delta_rel_dev=None, stream=None):
+        opt = lambda t: C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p()
+        self._check(lib().dt_planner_step(self._h, C.c_void_p(mask_dev.data_ptr()), opt(is_anchor_dev), opt(ase_dev),
+                                          opt(delta_rel_dev), _stream_ptr(stream)))
+
+    def dt_planner_commit(self, stream=None):
+        self._check(lib().dt_planner_commit(self._h, _stream_ptr(stream)))
+
+    def dt_planner_get(self):
+        P = self.cfg.P
+        w = np.empty((P, P), dtype=np.float64); alpha = np.empty((P, P), dtype=np.float64)
+        eps = C.c_double(); have = C.c_int32()
+        self._check(lib().dt_planner_get(self._h, w.ctypes.data_as(C.c_void_p), alpha.ctypes.data_as(C.c_void_p),
+                                         C.byref(eps), C.byref(have)))
+        return w, alpha, eps.value, bool(have.value)
 
     def dt_plan_grouped(self, mask_dev, group_size, eps=0.0, target_fraction=-1.0, w_dev=None, eps_out_dev=None,
                         stream=None):

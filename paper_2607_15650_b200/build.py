@@ -15,7 +15,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libditango.so")
-SOURCES = ["api.cu", "attn_states.cu", "state_merge.cu", "plan.cu"]
+SOURCES = ["api.cu", "attn_states.cu", "state_merge.cu", "plan.cu", "planner.cu"]
 HEADERS = ["dt_internal.h", "ptx_sm100.cuh", os.path.join("..", "..", "include", "ditango.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 

@@ -158,6 +158,9 @@ dt_status dt_destroy(dt_ctx *ctx) {
     cudaFree(ctx->status_dev);
     cudaFree(ctx->plan_partials_dev);
     cudaFree(ctx->sel_bits_dev);
+    cudaFree(ctx->planner_state_dev);
+    cudaFree(ctx->planner_local_partials_dev);
+    cudaFree(ctx->planner_norm_partials_dev);
     delete ctx;
     return DT_OK;
 }
@@ -175,10 +178,11 @@ dt_status dt_bind_cache(dt_ctx *ctx, void *o_state_dev, float *lse_state_dev, si
     return DT_OK;
 }
 
-dt_status dt_attn_states(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
-                         const int64_t strides_blhd[4], const uint8_t *mask_dev, int32_t step, void *stream) {
-    if (!ctx) return DT_ERR_INVALID_ARG;
-    if (!q_dev || !k_dev || !v_dev || !mask_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null tensor pointer");
+namespace {
+// mask_dev == nullptr: local (diagonal) pairs only
+dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev, const int64_t strides_blhd[4],
+                      const uint8_t *mask_dev, int32_t step, void *stream) {
+    if (!q_dev || !k_dev || !v_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null tensor pointer");
     if (step < 0) return fail(ctx, DT_ERR_INVALID_ARG, "step must be >= 0");
     if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
     const char *why;
@@ -208,6 +212,20 @@ dt_status dt_attn_states(dt_ctx *ctx, const void *q_dev, const void *k_dev, cons
     if (e != cudaSuccess) return fail_cuda(ctx, e, "attention launch");
     ctx->launches += 2;
     return DT_OK;
+}
+}  // namespace
+
+dt_status dt_attn_states(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
+                         const int64_t strides_blhd[4], const uint8_t *mask_dev, int32_t step, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!mask_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null mask pointer");
+    return attn_launch(ctx, q_dev, k_dev, v_dev, strides_blhd, mask_dev, step, stream);
+}
+
+dt_status dt_attn_local(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
+                        const int64_t strides_blhd[4], int32_t step, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    return attn_launch(ctx, q_dev, k_dev, v_dev, strides_blhd, nullptr, step, stream);
 }
 
 dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev,
@@ -398,6 +416,112 @@ dt_status dt_set_tc(dt_ctx *ctx, const int32_t *tc_host) {
 dt_status dt_launch_count(dt_ctx *ctx, uint64_t *count) {
     if (!ctx || !count) return DT_ERR_INVALID_ARG;
     *count = ctx->launches;
+    return DT_OK;
+}
+
+namespace {
+dt::PlannerParams planner_params(dt_ctx *ctx) {
+    const dt_config &c = ctx->cfg;
+    dt::PlannerParams p = {};
+    p.state = ctx->planner_state_dev;
+    p.o_state = ctx->o_state;
+    p.lse_state = ctx->lse_state;
+    p.snap_o = ctx->snap_o;
+    p.snap_lse = ctx->snap_lse;
+    p.snap_o_out = ctx->snap_o;
+    p.snap_lse_out = ctx->snap_lse;
+    p.off = ctx->off_dev;
+    p.local_partials = ctx->planner_local_partials_dev;
+    p.norm_partials = ctx->planner_norm_partials_dev;
+    p.w_partials = ctx->plan_partials_dev;
+    p.P = c.P; p.BH = c.B * c.H; p.L = c.L; p.D = c.D; p.chunks = ctx->plan_chunks;
+    p.group_size = ctx->planner_group_size;
+    p.eps_local = ctx->planner_eps_local;
+    p.cache_ratio = ctx->planner_cache_ratio;
+    return p;
+}
+}  // namespace
+
+dt_status dt_planner_init(dt_ctx *ctx, const dt_planner_config *pc, void *snap_o_dev, float *snap_lse_dev,
+                          size_t snap_o_bytes, size_t snap_lse_bytes, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!pc || !snap_o_dev || !snap_lse_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null pointer");
+    const dt_config &c = ctx->cfg;
+    if (pc->group_size < 1 || pc->group_size > c.P) return fail(ctx, DT_ERR_INVALID_ARG, "group_size must be in [1, P]");
+    if (!(pc->eps_initial >= 0.0) || !(pc->eps_local > 0.0) || !(pc->cache_ratio >= 0.0 && pc->cache_ratio <= 1.0))
+        return fail(ctx, DT_ERR_INVALID_ARG, "eps_initial >= 0, eps_local > 0 and 0 <= cache_ratio <= 1 required");
+    if ((long long)c.B * c.H * c.P > 65535) return fail(ctx, DT_ERR_UNSUPPORTED, "B*H*P exceeds 65535");
+    const size_t rows = (size_t)c.B * c.H * c.L;
+    if (snap_o_bytes < rows * c.D * state_elem_bytes(c.state_dtype) || snap_lse_bytes < rows * 4)
+        return fail(ctx, DT_ERR_STATE, "snapshot buffers smaller than one cache slot");
+    if ((reinterpret_cast<uintptr_t>(snap_o_dev) & 15u) != 0) return fail(ctx, DT_ERR_INVALID_ARG, "snapshot must be 16-byte aligned");
+    if (!ctx->planner_state_dev) {
+        const size_t BH = (size_t)c.B * c.H;
+        bool ok = cudaMalloc(&ctx->planner_state_dev, sizeof(dt::PlannerState)) == cudaSuccess;
+        ok = ok && cudaMalloc(&ctx->planner_local_partials_dev, BH * c.P * ctx->plan_chunks * 2 * sizeof(float)) == cudaSuccess;
+        ok = ok && cudaMalloc(&ctx->planner_norm_partials_dev, BH * c.P * ctx->plan_chunks * c.P * sizeof(float)) == cudaSuccess;
+        if (!ok) return fail(ctx, DT_ERR_CUDA, "planner scratch allocation failed");
+    }
+    ctx->snap_o = snap_o_dev;
+    ctx->snap_lse = snap_lse_dev;
+    ctx->planner_group_size = pc->group_size;
+    ctx->planner_eps_local = pc->eps_local;
+    ctx->planner_cache_ratio = pc->cache_ratio;
+    cudaError_t e = dt::launch_planner_init(ctx->planner_state_dev, pc->eps_initial, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "planner init launch");
+    ctx->launches += 1;
+    return DT_OK;
+}
+
+dt_status dt_planner_step(dt_ctx *ctx, uint8_t *mask_dev, int32_t *is_anchor_dev, double *ase_dev, double *delta_rel_dev,
+                          void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!mask_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null mask pointer");
+    if (!ctx->planner_state_dev) return fail(ctx, DT_ERR_STATE, "dt_planner_init has not been called");
+    if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
+    dt::PlannerParams p = planner_params(ctx);
+    p.mask = mask_dev;
+    p.is_anchor_out = is_anchor_dev;
+    p.ase_out = ase_dev;
+    p.delta_rel_out = delta_rel_dev;
+    cudaError_t e = dt::launch_planner_step(p, ctx->cfg.state_dtype, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "planner step launch");
+    ctx->launches += 2;
+    return DT_OK;
+}
+
+dt_status dt_planner_commit(dt_ctx *ctx, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!ctx->planner_state_dev) return fail(ctx, DT_ERR_STATE, "dt_planner_init has not been called");
+    const dt_config &c = ctx->cfg;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    dt::PlanParams pp;
+    pp.lse_state = ctx->lse_state;
+    pp.off = ctx->off_dev;
+    pp.partials = ctx->plan_partials_dev;
+    pp.P = c.P; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
+    pp.R = (long long)c.B * c.H * c.L;
+    cudaError_t e = dt::launch_plan_partial(pp, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
+    dt::PlannerParams p = planner_params(ctx);
+    e = dt::launch_planner_commit(p, c.state_dtype, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "planner commit launch");
+    ctx->launches += 4;
+    return DT_OK;
+}
+
+dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double *eps_host, int32_t *have_anchor_host) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!ctx->planner_state_dev) return fail(ctx, DT_ERR_STATE, "dt_planner_init has not been called");
+    dt::PlannerState hs;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&hs, ctx->planner_state_dev, sizeof hs, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "dt_planner_get");
+    const int n = ctx->cfg.P * ctx->cfg.P;
+    if (w_host) memcpy(w_host, hs.w, n * sizeof(double));
+    if (alpha_host) memcpy(alpha_host, hs.alpha, n * sizeof(double));
+    if (eps_host) *eps_host = hs.eps;
+    if (have_anchor_host) *have_anchor_host = hs.have_anchor;
     return DT_OK;
 }
 

@@ -70,6 +70,39 @@ struct PlanFinalParams {
     double *eps_out;   // may be null
 };
 
+// Planner state of Algorithm 1, resident on the device.
+struct PlannerState {
+    double w[DT_MAX_P * DT_MAX_P];       // partition importance weights of the last anchor (Eq. 8)
+    double alpha[DT_MAX_P * DT_MAX_P];   // scale ratios of the last anchor (Eq. 9)
+    double eps;                          // current threshold (Eq. 13)
+    int have_anchor;                     // an anchor has been committed
+    int is_anchor;                       // the step being planned is an anchor
+};
+
+struct PlannerParams {
+    PlannerState *state;
+    const void *o_state;          // cache
+    const float *lse_state;
+    const void *snap_o;           // local states of the last anchor: [B][H][L][D] in the cache dtype
+    const float *snap_lse;        // [B][H][L]
+    void *snap_o_out;
+    float *snap_lse_out;
+    const int32_t *off;           // device, P+1
+    float *local_partials;        // [BH][P][chunks][2]
+    float *norm_partials;         // [BH][P][chunks][P]
+    const float *w_partials;      // [BH][P][chunks][P] from plan_partial_kernel
+    uint8_t *mask;                // out, P*P
+    int32_t *is_anchor_out;       // out, may be null
+    double *ase_out;              // out, P * n_groups, may be null
+    double *delta_rel_out;        // out, may be null
+    int P, BH, L, D, chunks, group_size;
+    double eps_local, cache_ratio;
+};
+
+cudaError_t launch_planner_init(PlannerState *st, double eps, cudaStream_t stream);
+cudaError_t launch_planner_step(const PlannerParams &p, int state_dtype, cudaStream_t stream);
+cudaError_t launch_planner_commit(const PlannerParams &p, int state_dtype, cudaStream_t stream);
+
 cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, int P, int step,
                             cudaStream_t stream);
 cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
@@ -95,7 +128,14 @@ struct dt_ctx {
     int32_t *worklist_dev = nullptr;
     int32_t *status_dev = nullptr;
     float *plan_partials_dev = nullptr;
-    uint32_t *sel_bits_dev = nullptr;   // 2 * DT_MAX_P words: composition, planned merge
+    uint32_t *sel_bits_dev = nullptr;
+    dt::PlannerState *planner_state_dev = nullptr;
+    float *planner_local_partials_dev = nullptr;
+    float *planner_norm_partials_dev = nullptr;
+    void *snap_o = nullptr;
+    float *snap_lse = nullptr;
+    int planner_group_size = 1;
+    double planner_eps_local = 0.0, planner_cache_ratio = 0.0;   // 2 * DT_MAX_P words: composition, planned merge
     void *o_state = nullptr;
     float *lse_state = nullptr;
     uint64_t launches = 0;

@@ -158,16 +158,18 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
 }
 
 // mask -> compact list of COMPUTE pairs (ordered by i*P+j), t_c update, REUSE-of-empty detection.
+// mask == nullptr: the local (diagonal) pairs only, and no REUSE-of-empty check (the other pairs of the
+// step are decided later).
 __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int32_t *tc, int32_t *worklist,
                                                         int32_t *status, int P, int step) {
     __shared__ uint8_t flag[DT_MAX_P * DT_MAX_P];
     const int total = P * P, e = threadIdx.x;
     bool f = false;
     if (e < total) {
-        f = mask[e] != 0;
+        f = mask ? (mask[e] != 0) : (e / P == e % P);
         flag[e] = f ? 1 : 0;
         if (f) tc[e] = step;
-        else if (tc[e] < 0) atomicOr(status, STATUS_REUSE_EMPTY);
+        else if (mask && tc[e] < 0) atomicOr(status, STATUS_REUSE_EMPTY);
     }
     __syncthreads();
     if (e < total) {

@@ -433,3 +433,85 @@ def test_step_from_host_buffers():
         ref, ref_l = orc.full_attention(qb, kb, vb, wl.scale, 0, h, np.arange(wl.L, dtype=np.int32))
         check_o(out[0, :, h].float().numpy(), ref, "host step")
         check_lse(lse[0, h].numpy(), ref_l, "host step")
+
+
+def test_algorithm1_planner_over_denoising_steps():
+    """Algorithm 1 on the device over several steps (local attention -> plan -> remaining pairs -> merge ->
+    commit), against the oracle's planner rule.  The decision is taken in fp64 on both sides from the GPU's
+    own w, alpha and local drift (recomputed on the host in fp64 from the GPU's cache and snapshot); w and
+    alpha themselves are compared with the oracle's values from the oracle's states."""
+    wl = inputs.Workload("alg1", 1, 2, 64, (4, 16, 16), 0, 4, 6, 0.05)
+    P, g, R, eps_local = 4, 1, 0.5, 0.5
+    run = Run(wl, seed=21)
+    dev, ctx, off = run.dev, run.ctx, run.off
+    snap_o = torch.zeros((wl.B, wl.H, wl.L, wl.D), dtype=torch.float32, device=dev)
+    snap_l = torch.zeros((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    ctx.dt_planner_init(snap_o, snap_l, group_size=g, eps_initial=0.0, eps_local=eps_local, cache_ratio=R)
+    mask = torch.zeros(P * P, dtype=torch.uint8, device=dev)
+    flag = torch.zeros(1, dtype=torch.int32, device=dev)
+    ase = torch.zeros(P * P, dtype=torch.float64, device=dev)
+    drel = torch.zeros(1, dtype=torch.float64, device=dev)
+    part = np.searchsorted(off, np.arange(wl.L), side="right") - 1
+    eps, have_anchor = 0.0, False
+    anchors, selective = 0, 0
+    for t in range(wl.steps):
+        q, k, v = run.gen.next()
+        ctx.dt_attn_local(q, k, v, t)                              # local states of the step
+        ctx.dt_planner_step(mask, flag, ase, drel)
+        torch.cuda.synchronize()
+        # --- the oracle rule on the GPU's own quantities
+        w_g, alpha_g, eps_before, have_g = ctx.dt_planner_get()
+        assert have_g == have_anchor
+        o_c = ctx.o_state.double().cpu().numpy(); l_c = ctx.lse_state.double().cpu().numpy()
+        so = snap_o.double().cpu().numpy(); sl = snap_l.double().cpu().numpy()
+        drift = np.zeros(P); base = np.zeros(P)
+        for i in range(P):
+            rows = part == i
+            drift[i] = ((o_c[i][:, :, rows] - so[:, :, rows]) ** 2).sum() + ((l_c[i][:, :, rows] - sl[:, :, rows]) ** 2).sum()
+            base[i] = (so[:, :, rows] ** 2).sum() + (sl[:, :, rows] ** 2).sum()
+        # eps_before already holds the updated value if this step is an anchor; the rule is applied with the
+        # value the device used, which the test tracks itself
+        ref = orc.planner_step(w_g, alpha_g, drift, base, g, eps, eps_local, R, have_anchor)
+        got_mask = mask.cpu().numpy().reshape(P, P)
+        assert bool(flag.item()) == ref["is_anchor"], (t, ref["delta_rel"])
+        assert (got_mask == ref["mask"]).all(), t
+        if have_anchor:
+            np.testing.assert_allclose(ase.cpu().numpy().reshape(P, P)[~np.eye(P, dtype=bool)],
+                                       ref["ase"][~np.eye(P, dtype=bool)], rtol=1e-4)
+            assert drel.item() == pytest.approx(ref["delta_rel"], rel=1e-4)
+            valid = ref["ase"][~np.isnan(ref["ase"])]
+            if not ref["is_anchor"]:                              # margin of the decision w.r.t. fp32 partial sums
+                assert (np.abs(valid - eps) / max(eps, 1e-300)).min() > 1e-5
+        assert eps_before == pytest.approx(ref["eps"], rel=1e-4)
+        eps = eps_before
+        # --- the rest of the step
+        rest = torch.from_numpy((got_mask * (1 - np.eye(P, dtype=np.uint8))).reshape(-1).copy()).to(dev)
+        ctx.dt_attn_states(q, k, v, rest, t)
+        ctx.dt_state_merge(run.out, run.lse)
+        ctx.dt_planner_commit()
+        torch.cuda.synchronize()
+        ctx.dt_poll()
+        outs, lses = run.ses.step(*(inputs.bf16_bits(x) for x in (q, k, v)), got_mask, t)
+        for (b, h), rows in run.rows.items():
+            check_o(run.out[b, :, h].float().cpu().numpy(), outs[(b, h)], f"alg1 step {t}")
+            check_lse(run.lse[b, h].cpu().numpy(), lses[(b, h)], f"alg1 step {t}")
+        assert (ctx.dt_get_tc() == run.ses.tc).all()
+        if ref["is_anchor"]:
+            anchors += 1
+            have_anchor = True
+            # w (Eq. 8) and alpha (Eq. 9) against the oracle's states of this anchor
+            w_g, alpha_g, _, _ = ctx.dt_planner_get()
+            lse_ref = np.empty((P, wl.B, wl.H, wl.L)); nsq = np.zeros((P, P))
+            for (b, h), rows in run.rows.items():
+                lse_ref[:, b, h, :] = run.ses.lse[(b, h)].T
+                for i in range(P):
+                    sel = part == i
+                    for j in range(P):
+                        nsq[i, j] += orc.state_norm_sq(run.ses.o[(b, h)][sel, j, :], run.ses.lse[(b, h)][sel, j])
+            np.testing.assert_allclose(w_g, orc.contribution(lse_ref, off), rtol=2e-3, atol=1e-6)
+            np.testing.assert_allclose(alpha_g, orc.scale_ratios(nsq), rtol=2e-3)
+            assert torch.equal(snap_l, torch.stack([ctx.lse_state[i] for i in range(P)])[torch.from_numpy(part).to(dev), :, :, torch.arange(wl.L, device=dev)].permute(1, 2, 0))
+        else:
+            selective += 1
+            assert 0 < got_mask.sum() < P * P
+    assert anchors >= 2 and selective >= 1

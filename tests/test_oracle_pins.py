@@ -444,6 +444,63 @@ def test_group_plan_target_fraction_takes_whole_groups_in_rank_order():
     assert orc.group_plan(W, g, target_fraction=1.0)[0].all()
 
 
+# ---------------------------------------------------------------- Algorithm 1 pieces
+
+def test_scale_ratio_and_state_norm_closed_forms():
+    """Eq. 9 on states with known norms: OUT = c_ij everywhere, LSE = 0 -> ||AS(i,j)||^2 = n_i H D c_ij^2,
+    so alpha(i,j) = |c_ij| / |c_ii|; scaling every state by the same factor leaves alpha unchanged."""
+    P, n, D = 3, 5, 4
+    c = np.array([[2.0, 1.0, 0.5], [3.0, 1.5, 6.0], [1.0, 1.0, 1.0]])
+    nsq = np.array([[orc.state_norm_sq(np.full((n, D), c[i, j]), np.zeros(n)) for j in range(P)] for i in range(P)])
+    np.testing.assert_allclose(nsq, n * D * c * c)
+    alpha = orc.scale_ratios(nsq)
+    np.testing.assert_allclose(alpha, np.abs(c) / np.abs(np.diag(c))[:, None])
+    np.testing.assert_allclose(orc.scale_ratios(9.0 * nsq), alpha)
+    assert orc.state_norm_sq(np.zeros((2, 3)), np.array([3.0, 4.0])) == 25.0      # the LSE is part of the state
+
+
+def test_planner_step_truth_table():
+    """Alg. 1: ASE = w * alpha * delta_local summed over the group (Eq. 7, 10, 12); anchor iff every unit
+    exceeds eps or the local drift exceeds eps_local (Eq. 14); otherwise COMPUTE iff ASE > eps (Eq. 13)."""
+    P = 4
+    W = np.array([[0.4, 0.3, 0.2, 0.1], [0.3, 0.4, 0.2, 0.1], [0.1, 0.2, 0.4, 0.3], [0.1, 0.2, 0.3, 0.4]])
+    alpha = np.ones((P, P)); alpha[0, 1] = 2.0
+    drift = np.array([1.0, 4.0, 0.25, 0.0])          # squared: deltas 1, 2, 0.5, 0
+    base = np.full(P, 100.0)
+    r = orc.planner_step(W, alpha, drift, base, 1, eps=0.25, eps_local=1.0, R=0.5, have_anchor=True)
+    assert not r["is_anchor"]
+    np.testing.assert_allclose(r["ase"][0, 1], 0.3 * 2.0 * 1.0)
+    np.testing.assert_allclose(r["ase"][1, 0], 0.3 * 2.0)
+    np.testing.assert_allclose(r["ase"][2, 3], 0.3 * 0.5)
+    assert np.isnan(r["ase"][2, 2]) and (r["ase"][3, :3] == 0).all()
+    expect = np.eye(P, dtype=np.uint8)
+    expect[0, 1] = 1                                   # 0.6 > 0.25 ; (0,2) = 0.2, (0,3) = 0.1 reuse
+    expect[1, 0] = expect[1, 2] = 1                    # 0.6, 0.4 ; (1,3) = 0.2 reuse
+    assert (r["mask"] == expect).all() and r["eps"] == 0.25
+    assert r["delta_rel"] == pytest.approx(np.sqrt(5.25 / 400.0))
+    # the local drift alone triggers an anchor
+    r2 = orc.planner_step(W, alpha, drift, base, 1, eps=0.25, eps_local=0.1, R=0.5, have_anchor=True)
+    assert r2["is_anchor"] and r2["mask"].all()
+    # eps becomes the R-quantile of the predicted unit errors: half of the 12 units at or below it
+    vals = np.sort(r["ase"][~np.isnan(r["ase"])])
+    assert r2["eps"] == pytest.approx(0.5 * (vals[5] + vals[6]))
+    assert (vals <= r2["eps"]).sum() == 6
+    # every unit above eps -> anchor; strictness: a unit exactly at eps is not "above"
+    r3 = orc.planner_step(W, alpha, np.full(P, 1.0), base, 1, eps=0.05, eps_local=10.0, R=0.5, have_anchor=True)
+    assert r3["is_anchor"]
+    r4 = orc.planner_step(W, alpha, np.full(P, 1.0), base, 1, eps=0.1, eps_local=10.0, R=0.5, have_anchor=True)
+    assert not r4["is_anchor"] and r4["mask"][0, 3] == 0 and r4["mask"][0, 2] == 1
+    # no anchor yet -> the first step is one, and eps is kept when nothing has drifted
+    r5 = orc.planner_step(W, alpha, np.zeros(P), base, 1, eps=0.3, eps_local=1.0, R=0.5, have_anchor=False)
+    assert r5["is_anchor"] and r5["eps"] == 0.3
+    # groups: the unit's error is the sum over its members, the local member excluded
+    r6 = orc.planner_step(W, alpha, drift, base, 2, eps=0.25, eps_local=1.0, R=0.5, have_anchor=True)
+    np.testing.assert_allclose(r6["ase"][0, 0], 0.6)              # only j = 1 (j = 0 is local)
+    np.testing.assert_allclose(r6["ase"][0, 1], 0.2 + 0.1)
+    np.testing.assert_allclose(r6["ase"][1, 1], (0.2 + 0.1) * 2.0)
+    assert r6["mask"][1].tolist() == [1, 1, 1, 1] and r6["mask"][0].tolist() == [1, 1, 1, 1] and r6["mask"][2].tolist() == [0, 0, 1, 0]
+
+
 def test_uniform_offsets():
     off = orc.uniform_offsets(32760, 16)
     assert off[0] == 0 and off[-1] == 32760
