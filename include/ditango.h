@@ -25,9 +25,17 @@
  *   - Limits: D in {64, 128}; 1 <= P <= 32; bf16 inputs; innermost stride 1.
  *
  * Memory layout of the state cache (caller-owned device memory, sized by dt_cache_bytes):
- *   o_state   [P (KV partition j)][B][H][L][D]   fp32 or bf16 (dt_config.state_dtype)
- *   lse_state [P (KV partition j)][B][H][L]      fp32
- * Row l of slot j belongs to pair (i, j) with i the partition that contains l.
+ *   o_state   [S (slot)][B][H][L][D]   fp32 or bf16 (dt_config.state_dtype)
+ *   lse_state [S (slot)][B][H][L]      fp32
+ * Pair mode (dt_config.group_size <= 1): S = P, slot j = KV partition j; row l of slot j belongs to
+ * pair (i, j) with i the partition that contains l.
+ * Group mode (group_size = g >= 2; Section 4.2.1): the P states of a query partition are organised as
+ * m = ceil(P / g) groups of g adjacent KV partitions plus the local state, which is handled separately:
+ * S = m + 1, slot 0 = the local state (i, i), slot 1 + k = the group state AS(G_k), i.e. the composition
+ * (Eq. 2) of the states of group k's partitions -- without partition i in the group that contains it,
+ * which therefore has g - 1 members.  A slot whose key set is empty for a query partition (a group of one
+ * that is the local partition) does not exist for its rows.  Masks, t_c and W are then [P][S] arrays
+ * indexed by (query partition, slot) instead of [P][P].
  */
 #ifndef DITANGO_H_
 #define DITANGO_H_
@@ -59,6 +67,7 @@ typedef struct {
     float softmax_scale;         /* s in exp(s * q.k); the paper's Eq. 1 leaves it implicit          */
     int32_t state_dtype;         /* DT_STATE_FP32 or DT_STATE_BF16: storage type of cached OUT_ij    */
     int32_t device;              /* CUDA device ordinal                                              */
+    int32_t group_size;          /* 0 or 1: pair mode; g >= 2: grouped cache with g partitions per group */
 } dt_config;
 
 /* Create / destroy a context.  dt_create makes `device` current, checks it is sm_100, copies the
@@ -66,7 +75,8 @@ typedef struct {
 dt_status dt_create(dt_ctx **ctx_out, const dt_config *cfg);
 dt_status dt_destroy(dt_ctx *ctx);
 
-/* Closed-form size of the state cache: o_bytes = P*B*H*L*D*sizeof(state), lse_bytes = P*B*H*L*4.
+/* Closed-form size of the state cache: o_bytes = S*B*H*L*D*sizeof(state), lse_bytes = S*B*H*L*4, with
+ * S = P in pair mode and ceil(P/g) + 1 in group mode (the memory saving of group-level composition).
  * Per pair this is OUT (n_i*H*D) + LSE (n_i*H) against 2*n_j*H*D for the KV it replaces
  * ("half of KV size", Section 2.2.4). */
 dt_status dt_cache_bytes(const dt_config *cfg, size_t *o_bytes, size_t *lse_bytes);
@@ -182,6 +192,32 @@ dt_status dt_planner_step(dt_ctx *ctx, uint8_t *mask_dev, int32_t *is_anchor_dev
 dt_status dt_planner_commit(dt_ctx *ctx, void *stream);
 /* Copy the planner state to the host (synchronises): w and alpha are double [P*P]; any pointer may be NULL. */
 dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double *eps_host, int32_t *have_anchor_host);
+
+/* Grouped state cache (Section 4.2.1, Section 4.2.2; Dynamic Group State Compose, Eq. 15).  With
+ * dt_config.group_size = g >= 2 the calls above work on slots instead of KV partitions:
+ *   dt_attn_states / dt_attn_local   mask is uint8 [P*S]; a COMPUTE slot is evaluated in one pass over all keys of
+ *                      its group, which yields exactly the composition (Eq. 2) of its members' states
+ *   dt_state_merge     composes the S slots of every row (slots that do not exist for a row's query partition
+ *                      are left out); dt_compose_reuse / dt_state_merge_planned likewise, mask [P*S]
+ *   dt_plan            W is double [P*S] (importance of the slot's whole key set = sum of its members' weights,
+ *                      Eq. 12); one decision per non-local slot, the local slot 0 always COMPUTE; the target
+ *                      fraction still counts pairs: K = round(f*P*P), a slot costs as many as it has members
+ *   dt_get_tc / dt_set_tc, dt_step_host   arrays are [P*S]
+ *   dt_plan_grouped with group_size > 1 and the dt_planner_* calls return DT_ERR_UNSUPPORTED.
+ * dt_num_slots       current S and g (either pointer may be NULL).
+ * dt_slot_ranges     key ranges of every (query partition, slot): int32 [P*S*4] = (r1, n1, r2, n2), the keys
+ *                    [r1, r1+n1) and [r2, r2+n2); n1 + n2 == 0 marks a slot that does not exist.
+ * dt_group_compose   Eq. 15 with k = 2: AS(G_2k) (+) AS(G_2k+1) -> AS(G'_k) for every query partition, in place
+ *                    in the cache (new slot 1 + k overwrites old slot 1 + k after both sources were read), g
+ *                    doubles, S becomes ceil(m/2) + 1; t_c of a new slot is the older of its sources' (-1 if one
+ *                    was never computed).  The memory behind the first S slots of the bound buffers is no
+ *                    longer used.  DT_ERR_STATE if only one group is left.  Synchronises the stream.
+ * dt_group_reset     back to the creation-time g (an anchor step recomputes every state): all t_c = -1, the
+ *                    cache contents are stale until the next all-COMPUTE step.  Synchronises the stream. */
+dt_status dt_num_slots(dt_ctx *ctx, int32_t *slots, int32_t *group_size);
+dt_status dt_slot_ranges(dt_ctx *ctx, int32_t *ranges_host);
+dt_status dt_group_compose(dt_ctx *ctx, void *stream);
+dt_status dt_group_reset(dt_ctx *ctx, void *stream);
 
 /* The same plan computation for callers that cannot allocate device memory at the point of the
  * call: code running inside a region where the allocator must stay untouched (a fixed-memory

@@ -284,3 +284,152 @@ def planner_step(W, alpha, drift_sq, anchor_local_sq, g, eps, eps_local, R, have
                 if i != j and ase[i, j // g] > eps:                # Eq. 13, strict
                     mask[i, j] = 1
     return dict(is_anchor=bool(is_anchor), mask=mask, ase=ase, eps=float(eps_new), delta_rel=delta_rel)
+
+
+# --------------------------------------------------------------------------------------------------
+# Grouped state cache (Section 4.2.1, Section 4.2.2; Dynamic Group State Compose, Eq. 15).
+#
+# The P states of a query partition i are organised as m = ceil(P / g) groups of g adjacent KV partitions
+# plus the local state, which is handled separately: slot 0 = local state (i, i); slot 1 + k = AS(G_k), the
+# composition (Eq. 2) of the states of group k's partitions, without partition i in the group that holds it.
+# Everything here is written as that definition: a group state is computed member by member (Eq. 1) and
+# composed with `merge` (Eq. 2); nothing evaluates a group in one pass.
+
+def group_slots(P, g):
+    """members[i][s]: KV partitions behind slot s of query partition i (an empty list: no such slot)."""
+    g = max(1, int(g))
+    m = (P + g - 1) // g
+    return [[[i]] + [[j for j in range(k * g, min(P, (k + 1) * g)) if j != i] for k in range(m)] for i in range(P)]
+
+
+def slot_contribution(lse_slots, off, members):
+    """Importance of every slot (Eq. 8 summed over the slot's members, Eq. 12): per query row the softmax of
+    the slots' LSEs, averaged over batch, heads and the rows of query partition i.  lse_slots [S, B, H, L]."""
+    lse_slots = np.asarray(lse_slots, dtype=np.float64)
+    S = lse_slots.shape[0]
+    P = len(off) - 1
+    W = np.zeros((P, S))
+    for i in range(P):
+        x = lse_slots[:, :, :, off[i]:off[i + 1]].copy()
+        for s in range(S):
+            if not members[i][s]:
+                x[s] = -np.inf
+        mx = x.max(axis=0, keepdims=True)
+        e = np.exp(x - mx)
+        w = e / e.sum(axis=0, keepdims=True)
+        W[i] = w.reshape(S, -1).mean(axis=1)
+    return W
+
+
+def slot_plan(W, members, g, eps=0.0, target_fraction=-1.0):
+    """One decision per non-local slot that exists (Section 4.2.3): COMPUTE iff W > eps (Eq. 13, strict), or,
+    for target_fraction >= 0, slots in order of decreasing W (ties: the group nearer to the local one, then
+    the smaller flat index i * S + s) while their members fit into K - P pairs, K = round(f P^2) clipped to
+    [P, P^2].  The local slot 0 is always COMPUTE.  Returns (mask [P, S] uint8, eps_used)."""
+    W = np.asarray(W, dtype=np.float64)
+    P, S = W.shape
+    mask = np.zeros((P, S), dtype=np.uint8)
+    mask[:, 0] = 1
+    units = [(i, s) for i in range(P) for s in range(1, S) if members[i][s]]
+    if target_fraction < 0:
+        for i, s in units:
+            if W[i, s] > eps:
+                mask[i, s] = 1
+        return mask, float(eps)
+    K = int(np.floor(target_fraction * P * P + 0.5))
+    K = min(max(K, P), P * P)
+    budget = K - P
+    order = sorted(units, key=lambda u: (-W[u], abs((u[1] - 1) - u[0] // g), u[0] * S + u[1]))
+    cum, taken = 0, 0
+    for r, u in enumerate(order):        # a unit is taken iff it and everything ranked before it fit
+        cum += len(members[u[0]][u[1]])
+        if cum <= budget:
+            mask[u] = 1
+            taken = r + 1
+    if not order or taken == len(order):
+        eps_used = 0.0
+    elif taken == 0:
+        eps_used = float(W[order[0]])
+    else:
+        eps_used = 0.5 * float(W[order[taken - 1]] + W[order[taken]])
+    return mask, eps_used
+
+
+class GroupedOracleSession:
+    """OracleSession for a grouped cache: per (query row, slot) the cached group state; COMPUTE slots are
+    recomputed member by member (Eq. 1) and composed (Eq. 2); the output composes all slots that exist.
+    compose() is Dynamic Group State Compose with k = 2 (Eq. 15); reset() returns to the original g."""
+
+    def __init__(self, B, L, H, D, off, scale, rows_by_bh, g):
+        self.B, self.L, self.H, self.D = B, L, H, D
+        self.off = np.ascontiguousarray(off, dtype=np.int32)
+        self.P = self.off.size - 1
+        self.scale = float(scale)
+        self.g0 = int(g)
+        self.rows = {bh: np.ascontiguousarray(r, dtype=np.int32) for bh, r in rows_by_bh.items()}
+        self.part = {bh: np.searchsorted(self.off, r, side="right") - 1 for bh, r in self.rows.items()}
+        self._layout(self.g0)
+        self.o = {bh: np.zeros((r.size, self.S, D)) for bh, r in self.rows.items()}
+        self.lse = {bh: np.full((r.size, self.S), -np.inf) for bh, r in self.rows.items()}
+        self.tc = -np.ones((self.P, self.S), dtype=np.int32)
+
+    def _layout(self, g):
+        self.g = g
+        self.members = group_slots(self.P, g)
+        self.S = len(self.members[0])
+
+    def step(self, q, k, v, mask, t):
+        mask = np.asarray(mask).reshape(self.P, self.S)
+        for i in range(self.P):
+            for s in range(self.S):
+                if self.members[i][s] and not mask[i, s] and self.tc[i, s] < 0:
+                    raise RuntimeError(f"REUSE of slot ({i},{s}) that was never computed")
+        outs, lses = {}, {}
+        for bh, rows in self.rows.items():
+            b, h = bh
+            for i in range(self.P):
+                sel = np.nonzero(self.part[bh] == i)[0]
+                if sel.size == 0:
+                    continue
+                for s in range(self.S):
+                    mem = self.members[i][s]
+                    if not mem or not mask[i, s]:
+                        continue
+                    po = np.empty((sel.size, len(mem), self.D)); pl = np.empty((sel.size, len(mem)))
+                    for a, j in enumerate(mem):                    # Eq. 1 per member partition
+                        po[:, a, :], pl[:, a] = pair_state(q, k, v, self.scale, b, h, rows[sel],
+                                                           int(self.off[j]), int(self.off[j + 1]))
+                    self.o[bh][sel, s, :], self.lse[bh][sel, s] = merge(po, pl)   # Eq. 2: the group state
+            outs[bh], lses[bh] = merge(self.o[bh], self.lse[bh])
+        for i in range(self.P):
+            for s in range(self.S):
+                if self.members[i][s] and mask[i, s]:
+                    self.tc[i, s] = t
+        return outs, lses
+
+    def compose(self):
+        """Eq. 15, k = 2: AS(G_2k) (+) AS(G_2k+1) -> AS(G'_k); the local slot stays."""
+        S_old, old_members = self.S, self.members
+        self._layout(self.g * 2)
+        for bh in self.rows:
+            o_old, l_old = self.o[bh], self.lse[bh]
+            o_new = np.zeros((o_old.shape[0], self.S, self.D)); l_new = np.full((o_old.shape[0], self.S), -np.inf)
+            o_new[:, 0], l_new[:, 0] = o_old[:, 0], l_old[:, 0]
+            for s in range(1, self.S):
+                src = [x for x in (2 * s - 1, 2 * s) if x < S_old]
+                o_new[:, s], l_new[:, s] = merge(o_old[:, src, :], l_old[:, src])
+            self.o[bh], self.lse[bh] = o_new, l_new
+        tc_new = -np.ones((self.P, self.S), dtype=np.int32)
+        tc_new[:, 0] = self.tc[:, 0]
+        for i in range(self.P):
+            for s in range(1, self.S):
+                src = [x for x in (2 * s - 1, 2 * s) if x < S_old and old_members[i][x]]
+                tc_new[i, s] = min(self.tc[i, x] for x in src) if src else -1
+        self.tc = tc_new
+
+    def reset(self):
+        self._layout(self.g0)
+        for bh, r in self.rows.items():
+            self.o[bh] = np.zeros((r.size, self.S, self.D))
+            self.lse[bh] = np.full((r.size, self.S), -np.inf)
+        self.tc = -np.ones((self.P, self.S), dtype=np.int32)

@@ -23,13 +23,14 @@ EXPORTS = [
     "dt_compose_reuse", "dt_state_merge_planned", "dt_plan", "dt_plan_grouped", "dt_planner_init", "dt_planner_step", "dt_planner_commit", "dt_planner_get",
     "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
     "dt_launch_count", "dt_selftest_wait_timeout", "dt_poll", "dt_status_str", "dt_last_error",
+    "dt_num_slots", "dt_slot_ranges", "dt_group_compose", "dt_group_reset",
 ]
 
 
 class dt_config(C.Structure):
     _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("L", C.c_int32), ("P", C.c_int32),
                 ("part_offsets", C.POINTER(C.c_int32)), ("softmax_scale", C.c_float),
-                ("state_dtype", C.c_int32), ("device", C.c_int32)]
+                ("state_dtype", C.c_int32), ("device", C.c_int32), ("group_size", C.c_int32)]
 
 
 class dt_planner_config(C.Structure):
@@ -83,6 +84,10 @@ def lib():
         "dt_launch_count": (C.c_int, [vp, C.POINTER(C.c_uint64)]),
         "dt_selftest_wait_timeout": (C.c_int, [vp, C.c_uint32, vp]),
         "dt_poll": (C.c_int, [vp]),
+        "dt_num_slots": (C.c_int, [vp, i32p, i32p]),
+        "dt_slot_ranges": (C.c_int, [vp, i32p]),
+        "dt_group_compose": (C.c_int, [vp, vp]),
+        "dt_group_reset": (C.c_int, [vp, vp]),
         "dt_status_str": (C.c_char_p, [C.c_int]),
         "dt_last_error": (C.c_char_p, [vp]),
     }
@@ -93,10 +98,10 @@ def lib():
     return L
 
 
-def make_config(B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0):
+def make_config(B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0, group_size=1):
     off = np.ascontiguousarray(offsets, dtype=np.int32)
     cfg = dt_config(B, H, D, L, off.size - 1, off.ctypes.data_as(C.POINTER(C.c_int32)), float(softmax_scale),
-                    int(state_dtype), int(device))
+                    int(state_dtype), int(device), int(group_size))
     cfg._keepalive = off
     return cfg
 
@@ -158,9 +163,10 @@ def dt_plan_static(lse_state, offsets, B, H, L, mask_dev, eps=0.0, target_fracti
 class Context:
     """Owns a dt_ctx and (optionally) the state-cache tensors bound to it."""
 
-    def __init__(self, B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0, alloc_cache=True):
+    def __init__(self, B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0, alloc_cache=True,
+                 group_size=1):
         self._h = C.c_void_p()
-        self.cfg = make_config(B, H, D, L, offsets, softmax_scale, state_dtype, device)
+        self.cfg = make_config(B, H, D, L, offsets, softmax_scale, state_dtype, device, group_size)
         self.device = torch.device("cuda", device)
         s = lib().dt_create(C.byref(self._h), C.byref(self.cfg))
         if s != DT_OK:
@@ -168,10 +174,10 @@ class Context:
             raise DitangoError(s, status_str(s), "dt_create")
         self.o_state = self.lse_state = None
         if alloc_cache:
-            P = self.cfg.P
+            S = self.dt_num_slots()[0]
             sdt = torch.float32 if state_dtype == DT_STATE_FP32 else torch.bfloat16
-            o = torch.empty((P, B, H, L, D), dtype=sdt, device=self.device)
-            l = torch.empty((P, B, H, L), dtype=torch.float32, device=self.device)
+            o = torch.empty((S, B, H, L, D), dtype=sdt, device=self.device)
+            l = torch.empty((S, B, H, L), dtype=torch.float32, device=self.device)
             self.dt_bind_cache(o, l)
 
     def _check(self, s):
@@ -267,9 +273,28 @@ class Context:
                                        C.c_void_p(out_host.data_ptr()), lp, C.c_void_p(workspace.data_ptr()),
                                        workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
 
+    def dt_num_slots(self):
+        """(cache slots S, current group size g)."""
+        S, g = C.c_int32(), C.c_int32()
+        self._check(lib().dt_num_slots(self._h, C.byref(S), C.byref(g)))
+        return int(S.value), int(g.value)
+
+    def dt_slot_ranges(self):
+        """int32 [P, S, 4]: keys [r1, r1+n1) and [r2, r2+n2) of every (query partition, slot)."""
+        S = self.dt_num_slots()[0]
+        r = np.empty((self.cfg.P, S, 4), dtype=np.int32)
+        self._check(lib().dt_slot_ranges(self._h, r.ctypes.data_as(C.POINTER(C.c_int32))))
+        return r
+
+    def dt_group_compose(self, stream=None):
+        self._check(lib().dt_group_compose(self._h, _stream_ptr(stream)))
+
+    def dt_group_reset(self, stream=None):
+        self._check(lib().dt_group_reset(self._h, _stream_ptr(stream)))
+
     def dt_get_tc(self):
         P = self.cfg.P
-        tc = np.empty((P, P), dtype=np.int32)
+        tc = np.empty((P, self.dt_num_slots()[0]), dtype=np.int32)
         self._check(lib().dt_get_tc(self._h, tc.ctypes.data_as(C.POINTER(C.c_int32))))
         return tc
 

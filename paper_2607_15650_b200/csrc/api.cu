@@ -35,7 +35,55 @@ dt_status check_config(const dt_config *c, const char **why) {
     for (int i = 0; i < c->P; ++i)
         if (c->part_offsets[i + 1] <= c->part_offsets[i]) { *why = "offsets must be strictly increasing"; return DT_ERR_INVALID_ARG; }
     if ((long long)c->B * c->H > 65535) { *why = "B*H exceeds 65535"; return DT_ERR_UNSUPPORTED; }
+    if (c->group_size < 0 || c->group_size > c->P) { *why = "group_size must be in [0, P]"; return DT_ERR_INVALID_ARG; }
     return DT_OK;
+}
+
+int slots_for(int P, int g) { return g <= 1 ? P : (P + g - 1) / g + 1; }
+
+// Slot table of a context for group size g (g <= 1: pair mode).
+void build_slot_table(dt_ctx *ctx, int g) {
+    const int P = ctx->cfg.P;
+    const std::vector<int32_t> &off = ctx->off;
+    const int S = slots_for(P, g);
+    ctx->group_size = g <= 1 ? 1 : g;
+    ctx->S = S;
+    ctx->slot_tab.assign((size_t)P * S, dt::SlotRange{0, 0, 0, 0});
+    ctx->members.assign((size_t)P * S, 0);
+    ctx->nonempty.assign(P, 0u);
+    for (int i = 0; i < P; ++i) {
+        for (int s = 0; s < S; ++s) {
+            dt::SlotRange r = {0, 0, 0, 0};
+            int mem = 0;
+            if (g <= 1) {
+                r.r1 = off[s]; r.n1 = off[s + 1] - off[s]; mem = 1;
+            } else if (s == 0) {
+                r.r1 = off[i]; r.n1 = off[i + 1] - off[i]; mem = 1;
+            } else {
+                const int lo = (s - 1) * g, hi = std::min(P, s * g);   // partitions [lo, hi) of group s - 1
+                if (i >= lo && i < hi) {   // the query partition's own group: the keys left and right of it
+                    r.r1 = off[lo]; r.n1 = off[i] - off[lo];
+                    r.r2 = off[i + 1]; r.n2 = off[hi] - off[i + 1];
+                    if (r.n1 == 0) { r.r1 = r.r2; r.n1 = r.n2; r.r2 = 0; r.n2 = 0; }
+                    mem = hi - lo - 1;
+                } else {
+                    r.r1 = off[lo]; r.n1 = off[hi] - off[lo]; mem = hi - lo;
+                }
+            }
+            ctx->slot_tab[(size_t)i * S + s] = r;
+            ctx->members[(size_t)i * S + s] = (uint8_t)mem;
+            if (r.n1 + r.n2 > 0) ctx->nonempty[i] |= 1u << s;
+        }
+    }
+}
+
+cudaError_t upload_slot_table(dt_ctx *ctx, cudaStream_t st) {
+    const size_t n = (size_t)ctx->cfg.P * ctx->S;
+    cudaError_t e = cudaMemcpyAsync(ctx->slot_tab_dev, ctx->slot_tab.data(), n * sizeof(dt::SlotRange), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->members_dev, ctx->members.data(), n, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->nonempty_dev, ctx->nonempty.data(), ctx->cfg.P * sizeof(uint32_t), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // the host vectors may change right after
+    return e;
 }
 
 size_t state_elem_bytes(int dtype) { return dtype == DT_STATE_FP32 ? 4 : 2; }
@@ -93,7 +141,7 @@ dt_status dt_cache_bytes(const dt_config *cfg, size_t *o_bytes, size_t *lse_byte
     dt_status s = check_config(cfg, &why);
     if (s != DT_OK) return s;
     if (!o_bytes || !lse_bytes) return DT_ERR_INVALID_ARG;
-    const size_t rows = (size_t)cfg->P * cfg->B * cfg->H * cfg->L;
+    const size_t rows = (size_t)slots_for(cfg->P, cfg->group_size) * cfg->B * cfg->H * cfg->L;
     *o_bytes = rows * cfg->D * state_elem_bytes(cfg->state_dtype);
     *lse_bytes = rows * 4;
     return DT_OK;
@@ -129,16 +177,25 @@ dt_status dt_create(dt_ctx **ctx_out, const dt_config *cfg) {
         return DT_ERR_CUDA;
     }
     const int P = cfg->P, BH = cfg->B * cfg->H;
+    build_slot_table(ctx, cfg->group_size);
+    ctx->group_size0 = ctx->group_size;
+    ctx->S0 = ctx->S;
+    ctx->cfg.group_size = ctx->group_size;
+    const int S = ctx->S;
     bool ok = true;
     ok = ok && cudaMalloc(&ctx->off_dev, (P + 1) * sizeof(int32_t)) == cudaSuccess;
-    ok = ok && cudaMalloc(&ctx->tc_dev, P * P * sizeof(int32_t)) == cudaSuccess;
-    ok = ok && cudaMalloc(&ctx->worklist_dev, (1 + P * P) * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->slot_tab_dev, (size_t)P * S * sizeof(dt::SlotRange)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->members_dev, (size_t)P * S) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->nonempty_dev, P * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->tc_dev, P * S * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->worklist_dev, (1 + P * S) * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->status_dev, sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->sel_bits_dev, 2 * DT_MAX_P * sizeof(uint32_t)) == cudaSuccess;
-    ok = ok && cudaMalloc(&ctx->plan_partials_dev, (size_t)BH * P * ctx->plan_chunks * P * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->plan_partials_dev, (size_t)BH * P * ctx->plan_chunks * S * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMemcpy(ctx->off_dev, ctx->off.data(), (P + 1) * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemset(ctx->tc_dev, 0xFF, P * P * sizeof(int32_t)) == cudaSuccess;  // -1 = empty
-    ok = ok && cudaMemset(ctx->worklist_dev, 0, (1 + P * P) * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && upload_slot_table(ctx, nullptr) == cudaSuccess;
+    ok = ok && cudaMemset(ctx->tc_dev, 0xFF, P * S * sizeof(int32_t)) == cudaSuccess;  // -1 = empty
+    ok = ok && cudaMemset(ctx->worklist_dev, 0, (1 + P * S) * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemset(ctx->status_dev, 0, sizeof(int32_t)) == cudaSuccess;
     ok = ok && dt::attn_states_configure() == cudaSuccess;
     if (!ok) {
@@ -153,6 +210,9 @@ dt_status dt_destroy(dt_ctx *ctx) {
     if (!ctx) return DT_OK;
     cudaSetDevice(ctx->cfg.device);
     cudaFree(ctx->off_dev);
+    cudaFree(ctx->slot_tab_dev);
+    cudaFree(ctx->members_dev);
+    cudaFree(ctx->nonempty_dev);
     cudaFree(ctx->tc_dev);
     cudaFree(ctx->worklist_dev);
     cudaFree(ctx->status_dev);
@@ -170,8 +230,8 @@ dt_status dt_bind_cache(dt_ctx *ctx, void *o_state_dev, float *lse_state_dev, si
     if (!o_state_dev || !lse_state_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null cache pointer");
     if ((reinterpret_cast<uintptr_t>(o_state_dev) & 15u) || (reinterpret_cast<uintptr_t>(lse_state_dev) & 15u))
         return fail(ctx, DT_ERR_INVALID_ARG, "cache pointers must be 16-byte aligned");
-    size_t need_o, need_l;
-    dt_cache_bytes(&ctx->cfg, &need_o, &need_l);
+    const size_t rows0 = (size_t)ctx->S0 * ctx->cfg.B * ctx->cfg.H * ctx->cfg.L;   // slots at creation (a composed cache needs fewer)
+    const size_t need_o = rows0 * ctx->cfg.D * state_elem_bytes(ctx->cfg.state_dtype), need_l = rows0 * 4;
     if (o_bytes < need_o || lse_bytes < need_l) return fail(ctx, DT_ERR_STATE, "cache buffers smaller than dt_cache_bytes");
     ctx->o_state = o_state_dev;
     ctx->lse_state = lse_state_dev;
@@ -197,15 +257,17 @@ dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const v
     if ((s = encode_qkv_map(ctx, &tv, v_dev, strides_blhd)) != DT_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dt_config &c = ctx->cfg;
-    cudaError_t e = dt::launch_worklist(mask_dev, ctx->tc_dev, ctx->worklist_dev, ctx->status_dev, c.P, step, st);
+    cudaError_t e = dt::launch_worklist(mask_dev, ctx->tc_dev, ctx->worklist_dev, ctx->status_dev, ctx->slot_tab_dev, c.P,
+                                        ctx->S, ctx->group_size0 > 1 ? 1 : 0, step, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "work-list launch");
     dt::AttnParams p;
     p.off = ctx->off_dev;
+    p.slot_tab = ctx->slot_tab_dev;
     p.worklist = ctx->worklist_dev;
     p.status = ctx->status_dev;
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
-    p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P;
+    p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P; p.S = ctx->S;
     p.qblocks_max = ctx->qblocks_max;
     p.scale_log2 = c.softmax_scale * 1.44269504088896340736f;
     e = dt::launch_attn_states(tq, tk, tv, p, c.D, c.state_dtype, ctx->num_sms, st);
@@ -239,12 +301,16 @@ dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_b
     const dt_config &c = ctx->cfg;
     dt::MergeParams p = {};
     p.mode = dt::MERGE_ALL;
+    if (ctx->group_size0 > 1) {   // a grouped cache has slots that do not exist for some query partitions
+        p.sel_bits = ctx->nonempty_dev;
+        for (int i = 0; i <= c.P; ++i) p.off_val[i] = ctx->off[i];
+    }
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
     p.out = out_dev;
     p.lse_out = lse_out_dev;
     p.status = ctx->status_dev;
-    p.P = c.P; p.H = c.H; p.L = c.L;
+    p.P = c.P; p.S = ctx->S; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
@@ -263,14 +329,14 @@ dt_status dt_compose_reuse(dt_ctx *ctx, const uint8_t *mask_dev, void *comp_o_de
     p.mode = dt::MERGE_COMPOSE;
     p.sel_bits = ctx->sel_bits_dev;
     for (int i = 0; i <= c.P; ++i) p.off_val[i] = ctx->off[i];
-    cudaError_t es = dt::launch_merge_select(mask_dev, c.P, 0, ctx->sel_bits_dev, static_cast<cudaStream_t>(stream));
+    cudaError_t es = dt::launch_merge_select(mask_dev, ctx->nonempty_dev, c.P, ctx->S, 0, ctx->sel_bits_dev, static_cast<cudaStream_t>(stream));
     if (es != cudaSuccess) return fail_cuda(ctx, es, "selection launch");
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
     p.comp_o_out = comp_o_dev;
     p.comp_lse_out = comp_lse_dev;
     p.status = ctx->status_dev;
-    p.P = c.P; p.H = c.H; p.L = c.L;
+    p.P = c.P; p.S = ctx->S; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "compose launch");
@@ -292,7 +358,7 @@ dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const voi
     p.mode = dt::MERGE_PLANNED;
     p.sel_bits = ctx->sel_bits_dev + DT_MAX_P;
     for (int i = 0; i <= c.P; ++i) p.off_val[i] = ctx->off[i];
-    cudaError_t es = dt::launch_merge_select(mask_dev, c.P, 1, ctx->sel_bits_dev + DT_MAX_P, static_cast<cudaStream_t>(stream));
+    cudaError_t es = dt::launch_merge_select(mask_dev, ctx->nonempty_dev, c.P, ctx->S, 1, ctx->sel_bits_dev + DT_MAX_P, static_cast<cudaStream_t>(stream));
     if (es != cudaSuccess) return fail_cuda(ctx, es, "selection launch");
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
@@ -301,7 +367,7 @@ dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const voi
     p.out = out_dev;
     p.lse_out = lse_out_dev;
     p.status = ctx->status_dev;
-    p.P = c.P; p.H = c.H; p.L = c.L;
+    p.P = c.P; p.S = ctx->S; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
@@ -319,6 +385,8 @@ dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32
                           double *w_dev, double *eps_out_dev, void *stream) {
     if (!ctx) return DT_ERR_INVALID_ARG;
     if (group_size < 1 || group_size > ctx->cfg.P) return fail(ctx, DT_ERR_INVALID_ARG, "group_size must be in [1, P]");
+    if (ctx->group_size0 > 1 && group_size != 1)
+        return fail(ctx, DT_ERR_UNSUPPORTED, "a grouped cache decides per slot: group_size must be 1 here");
     if (!mask_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null mask pointer");
     if (!ctx->lse_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
     if (target_fraction < 0 && !std::isfinite(eps)) return fail(ctx, DT_ERR_INVALID_ARG, "eps must be finite");
@@ -329,10 +397,30 @@ dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32
     pp.lse_state = ctx->lse_state;
     pp.off = ctx->off_dev;
     pp.partials = ctx->plan_partials_dev;
-    pp.P = c.P; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
+    pp.nonempty = ctx->group_size0 > 1 ? ctx->nonempty_dev : nullptr;
+    pp.P = c.P; pp.S = ctx->S; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
     pp.R = (long long)c.B * c.H * c.L;
     cudaError_t e = dt::launch_plan_partial(pp, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
+    if (ctx->group_size0 > 1) {
+        dt::PlanSlotsParams ps;
+        ps.partials = ctx->plan_partials_dev;
+        ps.off = ctx->off_dev;
+        ps.slot_tab = ctx->slot_tab_dev;
+        ps.members = ctx->members_dev;
+        ps.P = c.P; ps.S = ctx->S; ps.BH = pp.BH; ps.chunks = pp.chunks; ps.group_size = ctx->group_size;
+        ps.mode_target = target_fraction >= 0 ? 1 : 0;
+        int Kp = (int)std::floor(target_fraction * (c.P * c.P) + 0.5);   // the budget is counted in pairs
+        ps.K = std::min(std::max(Kp, c.P), c.P * c.P);
+        ps.eps = eps;
+        ps.mask = mask_dev;
+        ps.w_out = w_dev;
+        ps.eps_out = eps_out_dev;
+        e = dt::launch_plan_slots(ps, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "plan finalise launch");
+        ctx->launches += 2;
+        return DT_OK;
+    }
     dt::PlanFinalParams pf;
     pf.partials = ctx->plan_partials_dev;
     pf.off = ctx->off_dev;
@@ -387,7 +475,7 @@ dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, cons
     if ((e = cudaMemcpyAsync(qd, q_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy q");
     if ((e = cudaMemcpyAsync(kd, k_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy k");
     if ((e = cudaMemcpyAsync(vd, v_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy v");
-    if ((e = cudaMemcpyAsync(md, mask_host, (size_t)c.P * c.P, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy mask");
+    if ((e = cudaMemcpyAsync(md, mask_host, (size_t)c.P * ctx->S, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy mask");
     const int64_t strides[4] = {(int64_t)c.L * c.H * c.D, (int64_t)c.H * c.D, c.D, 1};
     dt_status s;
     if ((s = dt_attn_states(ctx, qd, kd, vd, strides, md, step, stream)) != DT_OK) return s;
@@ -402,14 +490,14 @@ dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, cons
 dt_status dt_get_tc(dt_ctx *ctx, int32_t *tc_host) {
     if (!ctx || !tc_host) return DT_ERR_INVALID_ARG;
     cudaError_t e = cudaDeviceSynchronize();
-    if (e == cudaSuccess) e = cudaMemcpy(tc_host, ctx->tc_dev, ctx->cfg.P * ctx->cfg.P * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(tc_host, ctx->tc_dev, ctx->cfg.P * ctx->S * sizeof(int32_t), cudaMemcpyDeviceToHost);
     return e == cudaSuccess ? DT_OK : fail_cuda(ctx, e, "dt_get_tc");
 }
 
 dt_status dt_set_tc(dt_ctx *ctx, const int32_t *tc_host) {
     if (!ctx || !tc_host) return DT_ERR_INVALID_ARG;
     cudaError_t e = cudaDeviceSynchronize();
-    if (e == cudaSuccess) e = cudaMemcpy(ctx->tc_dev, tc_host, ctx->cfg.P * ctx->cfg.P * sizeof(int32_t), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->tc_dev, tc_host, ctx->cfg.P * ctx->S * sizeof(int32_t), cudaMemcpyHostToDevice);
     return e == cudaSuccess ? DT_OK : fail_cuda(ctx, e, "dt_set_tc");
 }
 
@@ -447,6 +535,7 @@ dt_status dt_planner_init(dt_ctx *ctx, const dt_planner_config *pc, void *snap_o
     if (!ctx) return DT_ERR_INVALID_ARG;
     if (!pc || !snap_o_dev || !snap_lse_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null pointer");
     const dt_config &c = ctx->cfg;
+    if (ctx->group_size0 > 1) return fail(ctx, DT_ERR_UNSUPPORTED, "the Algorithm 1 planner runs on a pair-mode cache (dt_config.group_size <= 1)");
     if (pc->group_size < 1 || pc->group_size > c.P) return fail(ctx, DT_ERR_INVALID_ARG, "group_size must be in [1, P]");
     if (!(pc->eps_initial >= 0.0) || !(pc->eps_local > 0.0) || !(pc->cache_ratio >= 0.0 && pc->cache_ratio <= 1.0))
         return fail(ctx, DT_ERR_INVALID_ARG, "eps_initial >= 0, eps_local > 0 and 0 <= cache_ratio <= 1 required");
@@ -499,7 +588,8 @@ dt_status dt_planner_commit(dt_ctx *ctx, void *stream) {
     pp.lse_state = ctx->lse_state;
     pp.off = ctx->off_dev;
     pp.partials = ctx->plan_partials_dev;
-    pp.P = c.P; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
+    pp.nonempty = nullptr;
+    pp.P = c.P; pp.S = c.P; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
     pp.R = (long long)c.B * c.H * c.L;
     cudaError_t e = dt::launch_plan_partial(pp, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
@@ -522,6 +612,78 @@ dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double
     if (alpha_host) memcpy(alpha_host, hs.alpha, n * sizeof(double));
     if (eps_host) *eps_host = hs.eps;
     if (have_anchor_host) *have_anchor_host = hs.have_anchor;
+    return DT_OK;
+}
+
+dt_status dt_num_slots(dt_ctx *ctx, int32_t *slots, int32_t *group_size) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (slots) *slots = ctx->S;
+    if (group_size) *group_size = ctx->group_size;
+    return DT_OK;
+}
+
+dt_status dt_slot_ranges(dt_ctx *ctx, int32_t *ranges_host) {
+    if (!ctx || !ranges_host) return DT_ERR_INVALID_ARG;
+    memcpy(ranges_host, ctx->slot_tab.data(), ctx->slot_tab.size() * sizeof(dt::SlotRange));
+    return DT_OK;
+}
+
+dt_status dt_group_compose(dt_ctx *ctx, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (ctx->group_size0 <= 1) return fail(ctx, DT_ERR_UNSUPPORTED, "dt_group_compose needs a grouped cache (dt_config.group_size >= 2)");
+    if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
+    const int m_old = ctx->S - 1;
+    if (m_old < 2) return fail(ctx, DT_ERR_STATE, "one group left: nothing to compose");
+    const dt_config &c = ctx->cfg;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int S_old = ctx->S, m_new = (m_old + 1) / 2, S_new = m_new + 1;
+    const size_t R = (size_t)c.B * c.H * c.L;
+    const size_t esz = state_elem_bytes(c.state_dtype);
+    // new slot 1 + k <- old slots 1 + 2k and 2 + 2k, in ascending k: a block reads its rows of both sources
+    // before it writes the same rows of slot 1 + k <= 1 + 2k, and later slots only read higher ones
+    for (int k = 0; k < m_new; ++k) {
+        std::vector<uint32_t> sel(c.P);
+        uint32_t bits = 1u << (1 + 2 * k);
+        if (2 + 2 * k < S_old) bits |= 1u << (2 + 2 * k);
+        for (int i = 0; i < c.P; ++i) sel[i] = bits & ctx->nonempty[i];
+        cudaError_t e = cudaMemcpyAsync(ctx->sel_bits_dev, sel.data(), c.P * sizeof(uint32_t), cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // `sel` is a temporary
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "group compose selection");
+        dt::MergeParams p = {};
+        p.mode = dt::MERGE_COMPOSE;
+        p.sel_bits = ctx->sel_bits_dev;
+        for (int i = 0; i <= c.P; ++i) p.off_val[i] = ctx->off[i];
+        p.o_state = ctx->o_state;
+        p.lse_state = ctx->lse_state;
+        p.comp_o_out = static_cast<uint8_t *>(ctx->o_state) + (size_t)(1 + k) * R * c.D * esz;
+        p.comp_lse_out = ctx->lse_state + (size_t)(1 + k) * R;
+        p.status = ctx->status_dev;
+        p.P = c.P; p.S = S_old; p.H = c.H; p.L = c.L;
+        p.R = (long long)R;
+        e = dt::launch_state_merge(p, c.D, c.state_dtype, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "group compose launch");
+        ctx->launches += 1;
+    }
+    cudaError_t e = dt::launch_tc_compose(ctx->tc_dev, ctx->nonempty_dev, c.P, S_old, S_new, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // t_c is rewritten from the old table before it changes
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "group compose t_c");
+    ctx->launches += 1;
+    build_slot_table(ctx, ctx->group_size * 2);
+    e = upload_slot_table(ctx, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "group compose table upload");
+    return DT_OK;
+}
+
+dt_status dt_group_reset(dt_ctx *ctx, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (ctx->group_size0 <= 1) return fail(ctx, DT_ERR_UNSUPPORTED, "dt_group_reset needs a grouped cache (dt_config.group_size >= 2)");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "group reset");
+    build_slot_table(ctx, ctx->group_size0);
+    e = upload_slot_table(ctx, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->tc_dev, 0xFF, (size_t)ctx->cfg.P * ctx->S * sizeof(int32_t), st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "group reset");
     return DT_OK;
 }
 

@@ -1,7 +1,9 @@
 // dt_attn_states: Eq. 1 for every COMPUTE pair -- flash attention of one query block of
 // partition i against the keys of partition j only, emitting the partition-normalised output
 // OUT_ij and LSE_ij straight into the state cache.  REUSE pairs never appear in the work list,
-// so they cost no instruction and no byte.
+// so they cost no instruction and no byte.  With a grouped cache (Section 4.2.1) a work item is a
+// (query partition, slot) whose keys are the slot's one or two key ranges: the group's state, the
+// composition (Eq. 2) of its members' states, comes out of one pass over their keys.
 //
 // One persistent CTA per SM walks the work list (b*h slowest, then COMPUTE pair, then query
 // block), so CTAs running at the same time share one head's K/V partition through L2.
@@ -87,12 +89,20 @@ struct RingPos {
 };
 
 struct WorkItem {
-    int bh, b, h, i, j;
+    int bh, b, h, i, slot;
     int q_row0;     // first query row of the block (global token index)
     int n_q;        // valid query rows in the block (<= NQ*128)
-    int kv_row0;    // first key of partition j
-    int n_kv;       // keys in partition j
-    int tiles;      // ceil(n_kv / 128)
+    int r1, n1;     // first key range of the slot
+    int r2, n2;     // second key range (n2 == 0: none)
+    int tiles1;     // ceil(n1 / 128)
+    int tiles;      // tiles1 + ceil(n2 / 128)
+    // first key of K/V tile t, and how many of its 128 keys belong to the slot (may exceed 128)
+    __device__ __forceinline__ int tile_row(int t) const {
+        return t < tiles1 ? r1 + t * ATTN_TILE : r2 + (t - tiles1) * ATTN_TILE;
+    }
+    __device__ __forceinline__ int tile_valid(int t) const {
+        return t < tiles1 ? n1 - t * ATTN_TILE : n2 - (t - tiles1) * ATTN_TILE;
+    }
 };
 
 // Work index -> item.  Returns false when the block lies beyond the end of partition i.
@@ -104,15 +114,16 @@ __device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, lon
     const int qb = rem - pair * p.qblocks_max;
     const int code = p.worklist[1 + pair];
     it.i = code & 0xFF;
-    it.j = code >> 8;
+    it.slot = code >> 8;
     it.b = it.bh / p.H;
     it.h = it.bh - it.b * p.H;
     const int qs = p.off[it.i], qe = p.off[it.i + 1];
     it.q_row0 = qs + qb * (ATTN_NQ * ATTN_TILE);
     it.n_q = min(qe - it.q_row0, ATTN_NQ * ATTN_TILE);
-    it.kv_row0 = p.off[it.j];
-    it.n_kv = p.off[it.j + 1] - it.kv_row0;
-    it.tiles = (it.n_kv + ATTN_TILE - 1) / ATTN_TILE;
+    const int4 rg = *reinterpret_cast<const int4 *>(p.slot_tab + it.i * p.S + it.slot);
+    it.r1 = rg.x; it.n1 = rg.y; it.r2 = rg.z; it.n2 = rg.w;
+    it.tiles1 = (it.n1 + ATTN_TILE - 1) / ATTN_TILE;
+    it.tiles = it.tiles1 + (it.n2 + ATTN_TILE - 1) / ATTN_TILE;
     return it.n_q > 0;
 }
 
@@ -230,7 +241,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 #pragma unroll
                         for (int hf = 0; hf < C::NHALF; ++hf)
                             tma_load_4d(kv_smem + st * C::TILE_BYTES + hf * C::HALF_BYTES, kv == 0 ? &tmap_k : &tmap_v,
-                                        bars.kv_full + 8 * st, hf * 64, it.h, it.kv_row0 + t * ATTN_TILE, it.b);
+                                        bars.kv_full + 8 * st, hf * 64, it.h, it.tile_row(t), it.b);
                         ring.advance();
                     }
                 }
@@ -398,7 +409,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 tmem_ld_x32(s_tmem + 64, s[2]);
                 tmem_ld_x32(s_tmem + 96, s[3]);
                 tmem_wait_ld();
-                const int valid = it.n_kv - t * ATTN_TILE;   // keys of this tile that belong to partition j
+                const int valid = it.tile_valid(t);   // keys of this tile that belong to the slot
                 if (valid < ATTN_TILE) {
 #pragma unroll
                     for (int c = 0; c < 128; ++c)
@@ -481,7 +492,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             const int row_in_block = q * ATTN_TILE + row_in_tile;
             const bool row_valid = row_in_block < it.n_q;
             const float inv_l = 1.0f / l_sum;
-            const long long srow = ((long long)it.j * p.B * p.H + it.bh) * p.L + it.q_row0 + row_in_block;
+            const long long srow = ((long long)it.slot * p.B * p.H + it.bh) * p.L + it.q_row0 + row_in_block;
 #pragma unroll
             for (int c0 = 0; c0 < D; c0 += 32) {
                 uint32_t o[32];

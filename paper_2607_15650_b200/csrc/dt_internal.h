@@ -18,13 +18,22 @@ constexpr int PLAN_CHUNK_ROWS = 1024;  // rows of one (b, h, partition) handled 
 constexpr int ATTN_TILE = 128;         // query rows per TMEM accumulator / keys per KV tile
 constexpr int ATTN_NQ = 2;             // query tiles a CTA keeps in flight (ping-pong)
 
+// Keys covered by the state in slot s of query partition i: [r1, r1 + n1) and [r2, r2 + n2) (token indices).
+// Pair mode: slot j = KV partition j (one range).  Group mode (Section 4.2.1): slot 0 = the local partition,
+// slot 1 + k = group k of g adjacent partitions, without partition i when it belongs to that group (then the
+// keys left and right of it are the two ranges).  n1 + n2 == 0: the slot is empty for this query partition.
+struct alignas(16) SlotRange {
+    int32_t r1, n1, r2, n2;
+};
+
 struct AttnParams {
     const int32_t *off;       // device, P+1
-    const int32_t *worklist;  // device: [0] = number of COMPUTE pairs, then i | (j << 8) per pair
+    const SlotRange *slot_tab; // device, [P][S]
+    const int32_t *worklist;  // device: [0] = number of COMPUTE states, then i | (slot << 8) per state
     int32_t *status;          // device status word
-    void *o_state;            // [P][B][H][L][D]
-    float *lse_state;         // [P][B][H][L]
-    int B, H, L, P;
+    void *o_state;            // [S][B][H][L][D]
+    float *lse_state;         // [S][B][H][L]
+    int B, H, L, P, S;
     int qblocks_max;          // ceil(max_i n_i / (ATTN_NQ * ATTN_TILE))
     float scale_log2;         // softmax_scale * log2(e)
 };
@@ -33,8 +42,9 @@ enum : int { MERGE_ALL = 0, MERGE_COMPOSE = 1, MERGE_PLANNED = 2 };
 
 struct MergeParams {
     int mode;                 // MERGE_ALL / MERGE_COMPOSE / MERGE_PLANNED
-    const uint32_t *sel_bits; // device, P words from launch_merge_select (modes COMPOSE, PLANNED)
-    int32_t off_val[DT_MAX_P + 1];   // partition offsets by value (modes COMPOSE, PLANNED)
+    const uint32_t *sel_bits; // device, P words: bit s = slot s takes part for rows of that query partition
+                              // (from launch_merge_select; MERGE_ALL: null = every slot)
+    int32_t off_val[DT_MAX_P + 1];   // partition offsets by value (used whenever sel_bits is set)
     const void *comp_o;       // composed state read by PLANNED: [B][H][L][D] in the cache's dtype
     const float *comp_lse;    // [B][H][L]
     void *comp_o_out;         // composed state written by COMPOSE
@@ -44,17 +54,32 @@ struct MergeParams {
     void *out;       // bf16
     float *lse_out;  // may be null
     int32_t *status; // device status word
-    int P, H, L;
+    int P, S, H, L;  // query partitions, cache slots
     long long R;     // B*H*L rows
     long long sb, sl, sh;  // output strides in elements
 };
 
 struct PlanParams {
-    const float *lse_state;  // [P][R]
+    const float *lse_state;  // [S][R]
     const int32_t *off;      // device, P+1
-    float *partials;         // [BH][P][chunks][P]
-    int P, BH, L, chunks;
+    const uint32_t *nonempty; // device, P words: slots that exist for the query partition (null = all)
+    float *partials;         // [BH][P][chunks][S]
+    int P, S, BH, L, chunks;
     long long R;
+};
+
+// Decisions over the slots of a grouped cache: one unit per (query partition, non-local slot).
+struct PlanSlotsParams {
+    const float *partials;   // [BH][P][chunks][S]
+    const int32_t *off;
+    const SlotRange *slot_tab;
+    const uint8_t *members;  // device, [P][S]: KV partitions a slot stands for (its size in pairs)
+    int P, S, BH, chunks, group_size;
+    int mode_target, K;
+    double eps;
+    uint8_t *mask;           // out, [P][S]
+    double *w_out;           // out, [P][S], may be null
+    double *eps_out;         // may be null
 };
 
 struct PlanFinalParams {
@@ -103,13 +128,16 @@ cudaError_t launch_planner_init(PlannerState *st, double eps, cudaStream_t strea
 cudaError_t launch_planner_step(const PlannerParams &p, int state_dtype, cudaStream_t stream);
 cudaError_t launch_planner_commit(const PlannerParams &p, int state_dtype, cudaStream_t stream);
 
-cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, int P, int step,
-                            cudaStream_t stream);
+cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, const SlotRange *slot_tab,
+                            int P, int S, int group_mode, int step, cudaStream_t stream);
 cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                                const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream);
 cudaError_t attn_states_configure();  // sets the dynamic shared-memory attribute once per process/device
 cudaError_t launch_state_merge(const MergeParams &p, int D, int state_dtype, cudaStream_t stream);
-cudaError_t launch_merge_select(const uint8_t *mask, int P, int want_compute, uint32_t *sel_bits, cudaStream_t stream);
+cudaError_t launch_merge_select(const uint8_t *mask, const uint32_t *nonempty, int P, int S, int want_compute,
+                                uint32_t *sel_bits, cudaStream_t stream);
+cudaError_t launch_plan_slots(const PlanSlotsParams &p, cudaStream_t stream);
+cudaError_t launch_tc_compose(int32_t *tc, const uint32_t *nonempty_old, int P, int S_old, int S_new, cudaStream_t stream);
 cudaError_t launch_plan_partial(const PlanParams &p, cudaStream_t stream);
 cudaError_t launch_plan_final(const PlanFinalParams &p, cudaStream_t stream);
 cudaError_t launch_wait_timeout_selftest(int32_t *status, long long limit_cycles, cudaStream_t stream);
@@ -123,6 +151,15 @@ struct dt_ctx {
     int qblocks_max = 0;
     int plan_chunks = 0;
     int num_sms = 0;
+    int group_size0 = 1;   // group size the context was created with (1 = pair mode)
+    int group_size = 1;    // current group size (doubles with every dt_group_compose)
+    int S0 = 0, S = 0;     // cache slots at creation / now
+    std::vector<dt::SlotRange> slot_tab;      // [P][S]
+    std::vector<uint8_t> members;             // [P][S]
+    std::vector<uint32_t> nonempty;           // [P]
+    dt::SlotRange *slot_tab_dev = nullptr;    // sized for S0
+    uint8_t *members_dev = nullptr;
+    uint32_t *nonempty_dev = nullptr;
     int32_t *off_dev = nullptr;
     int32_t *tc_dev = nullptr;
     int32_t *worklist_dev = nullptr;

@@ -22,7 +22,8 @@ constexpr int PLAN_THREADS = 256;
 template <int PMAX>
 __global__ void __launch_bounds__(PLAN_THREADS) plan_partial_kernel(PlanParams p) {
     const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z;
-    const int P = p.P;
+    const int P = p.S;   // columns: cache slots (pair mode: one per KV partition)
+    const uint32_t have = p.nonempty ? p.nonempty[i] : 0xFFFFFFFFu;   // slots that exist for this query partition
     const int row0 = p.off[i] + c * PLAN_CHUNK_ROWS;
     const int row1 = min(row0 + PLAN_CHUNK_ROWS, p.off[i + 1]);
     float acc[PMAX];
@@ -34,7 +35,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_partial_kernel(PlanParams p
         float M = -INFINITY;
 #pragma unroll
         for (int j = 0; j < PMAX; ++j) {
-            x[j] = (j < P) ? __ldcs(base + (long long)j * p.R + l) : -INFINITY;
+            x[j] = (j < P && (have >> j & 1u)) ? __ldcs(base + (long long)j * p.R + l) : -INFINITY;
             M = fmaxf(M, x[j]);
         }
         if (M == -INFINITY) continue;  // row without any mass: contributes nothing
@@ -63,7 +64,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_partial_kernel(PlanParams p
         float v = 0.f;
 #pragma unroll
         for (int w = 0; w < PLAN_THREADS / 32; ++w) v += red[w][threadIdx.x];
-        p.partials[(((long long)bh * P + i) * p.chunks + c) * P + threadIdx.x] = v;
+        p.partials[(((long long)bh * p.P + i) * p.chunks + c) * P + threadIdx.x] = v;
     }
 }
 
@@ -157,19 +158,23 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
     }
 }
 
-// mask -> compact list of COMPUTE pairs (ordered by i*P+j), t_c update, REUSE-of-empty detection.
-// mask == nullptr: the local (diagonal) pairs only, and no REUSE-of-empty check (the other pairs of the
-// step are decided later).
+// mask -> compact list of COMPUTE states (ordered by i*S+slot), t_c update, REUSE-of-empty detection.
+// mask == nullptr: the local states only, and no REUSE-of-empty check (the other states of the step are
+// decided later).  Slots that do not exist for a query partition are never listed and never flagged.
 __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int32_t *tc, int32_t *worklist,
-                                                        int32_t *status, int P, int step) {
+                                                        int32_t *status, const SlotRange *slot_tab, int P, int S,
+                                                        int group_mode, int step) {
     __shared__ uint8_t flag[DT_MAX_P * DT_MAX_P];
-    const int total = P * P, e = threadIdx.x;
+    const int total = P * S, e = threadIdx.x;
     bool f = false;
     if (e < total) {
-        f = mask ? (mask[e] != 0) : (e / P == e % P);
+        const int i = e / S, s = e - i * S;
+        const bool exists = slot_tab[e].n1 + slot_tab[e].n2 > 0;
+        const int local = group_mode ? 0 : i;
+        f = exists && (mask ? (mask[e] != 0) : (s == local));
         flag[e] = f ? 1 : 0;
         if (f) tc[e] = step;
-        else if (mask && tc[e] < 0) atomicOr(status, STATUS_REUSE_EMPTY);
+        else if (exists && mask && tc[e] < 0) atomicOr(status, STATUS_REUSE_EMPTY);
     }
     __syncthreads();
     if (e < total) {
@@ -178,8 +183,96 @@ __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int
             cnt += flag[o];
             if (o < e) pos += flag[o];
         }
-        if (f) worklist[1 + pos] = (e / P) | ((e % P) << 8);
+        if (f) worklist[1 + pos] = (e / S) | ((e % S) << 8);
         if (e == 0) worklist[0] = cnt;
+    }
+}
+
+// Decisions for a grouped cache (Section 4.2.1 - 4.2.3): W[i][s] from the partial sums; every non-local slot
+// that exists is one decision unit whose measure is the importance of its whole key set (the sum of its
+// members' weights, Eq. 12, which is what the slot's LSE yields directly).  COMPUTE iff measure > eps
+// (Eq. 13), or the units of largest measure taken in rank order while their member pairs fit into K - P.
+__global__ void __launch_bounds__(1024) plan_slots_kernel(PlanSlotsParams p) {
+    __shared__ double m_s[DT_MAX_P * DT_MAX_P];
+    __shared__ uint8_t size_s[DT_MAX_P * DT_MAX_P];
+    __shared__ double edge[2];
+    const int P = p.P, S = p.S, total = P * S, g = p.group_size;
+    const int e = threadIdx.x;
+    const int i = e / S, s = e - i * S;
+    double m = 0.0;
+    int size = 0, dist = 0;
+    if (e < total) {
+        double sum = 0.0;
+        for (int bh = 0; bh < p.BH; ++bh)
+            for (int c = 0; c < p.chunks; ++c) sum += (double)p.partials[(((long long)bh * P + i) * p.chunks + c) * S + s];
+        m = sum / ((double)p.BH * (double)(p.off[i + 1] - p.off[i]));
+        if (p.w_out) p.w_out[e] = m;
+        size = (s == 0) ? 0 : (int)p.members[e];   // the local slot is no unit: always COMPUTE
+        const int gi = i / g, k = s - 1;
+        dist = k > gi ? k - gi : gi - k;
+        m_s[e] = m;
+        size_s[e] = (uint8_t)size;
+    }
+    if (e < 2) edge[e] = 0.0;
+    __syncthreads();
+    bool take = false;
+    int rank = -1;
+    const int budget = p.K - P;
+    if (e < total && size > 0) {
+        if (!p.mode_target) {
+            take = m > p.eps;
+        } else {
+            rank = 0;
+            int cum = size;
+            for (int o = 0; o < total; ++o) {
+                if (o == e || size_s[o] == 0) continue;
+                const int oi = o / S, ok = o - oi * S - 1, ogi = oi / g;
+                const int od = ok > ogi ? ok - ogi : ogi - ok;
+                if (ranks_before(m_s[o], od, o, m, dist, e)) { ++rank; cum += size_s[o]; }
+            }
+            take = cum <= budget;
+        }
+    }
+    const int taken = __syncthreads_count(take);
+    if (p.mode_target && rank >= 0) {
+        if (rank == taken - 1) edge[0] = m;
+        if (rank == taken) edge[1] = m;
+    }
+    if (e < total) p.mask[e] = (s == 0 || take) ? 1 : 0;
+    __syncthreads();
+    if (e == 0 && p.eps_out) {
+        double eps = p.eps;
+        if (p.mode_target) {
+            int n = 0;
+            for (int o = 0; o < total; ++o) n += size_s[o] > 0;
+            if (n == 0 || taken == n) eps = 0.0;
+            else if (taken == 0) eps = edge[1];
+            else eps = 0.5 * (edge[0] + edge[1]);
+        }
+        *p.eps_out = eps;
+    }
+}
+
+// t_c after Dynamic Group State Compose (Eq. 15, k = 2): slot 0 (local) keeps its step; new slot 1 + k takes
+// the older of old slots 1 + 2k and 2 + 2k that exist (-1 if one of them was never computed).
+__global__ void tc_compose_kernel(int32_t *tc, const uint32_t *nonempty_old, int P, int S_old, int S_new) {
+    __shared__ int32_t old_s[DT_MAX_P * DT_MAX_P];
+    const int e = threadIdx.x;
+    if (e < P * S_old) old_s[e] = tc[e];
+    __syncthreads();
+    if (e < P * S_new) {
+        const int i = e / S_new, s = e - i * S_new;
+        int32_t v;
+        if (s == 0) {
+            v = old_s[i * S_old];
+        } else {
+            v = 0x7FFFFFFF;
+            bool any = false;
+            for (int o = 2 * s - 1; o <= 2 * s && o < S_old; ++o)
+                if (nonempty_old[i] >> o & 1u) { v = min(v, old_s[i * S_old + o]); any = true; }
+            if (!any) v = -1;
+        }
+        tc[e] = v;
     }
 }
 
@@ -208,8 +301,8 @@ namespace {
 
 cudaError_t launch_plan_partial(const PlanParams &p, cudaStream_t stream) {
     dim3 grid((unsigned)p.chunks, (unsigned)p.P, (unsigned)p.BH);
-    if (p.P <= 8) plan_partial_kernel<8><<<grid, PLAN_THREADS, 0, stream>>>(p);
-    else if (p.P <= 16) plan_partial_kernel<16><<<grid, PLAN_THREADS, 0, stream>>>(p);
+    if (p.S <= 8) plan_partial_kernel<8><<<grid, PLAN_THREADS, 0, stream>>>(p);
+    else if (p.S <= 16) plan_partial_kernel<16><<<grid, PLAN_THREADS, 0, stream>>>(p);
     else plan_partial_kernel<32><<<grid, PLAN_THREADS, 0, stream>>>(p);
     return cudaGetLastError();
 }
@@ -219,9 +312,19 @@ cudaError_t launch_plan_final(const PlanFinalParams &p, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, int P, int step,
-                            cudaStream_t stream) {
-    worklist_kernel<<<1, 1024, 0, stream>>>(mask, tc, worklist, status, P, step);
+cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, const SlotRange *slot_tab,
+                            int P, int S, int group_mode, int step, cudaStream_t stream) {
+    worklist_kernel<<<1, 1024, 0, stream>>>(mask, tc, worklist, status, slot_tab, P, S, group_mode, step);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_plan_slots(const PlanSlotsParams &p, cudaStream_t stream) {
+    plan_slots_kernel<<<1, 1024, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tc_compose(int32_t *tc, const uint32_t *nonempty_old, int P, int S_old, int S_new, cudaStream_t stream) {
+    tc_compose_kernel<<<1, 1024, 0, stream>>>(tc, nonempty_old, P, S_old, S_new);
     return cudaGetLastError();
 }
 
@@ -284,7 +387,8 @@ extern "C" dt_status dt_plan_static(const float *lse_state_dev, const int32_t *p
     pp.lse_state = lse_state_dev;
     pp.off = off_dev;
     pp.partials = partials;
-    pp.P = P; pp.BH = B * H; pp.L = L; pp.chunks = chunks;
+    pp.nonempty = nullptr;
+    pp.P = P; pp.S = P; pp.BH = B * H; pp.L = L; pp.chunks = chunks;
     pp.R = (long long)B * H * L;
     if (dt::launch_plan_partial(pp, st) != cudaSuccess) return DT_ERR_CUDA;
     dt::PlanFinalParams pf;

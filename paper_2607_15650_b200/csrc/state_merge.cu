@@ -1,4 +1,4 @@
-// dt_state_merge: Eq. 2 folded over the P cached states of every query row.
+// dt_state_merge: Eq. 2 folded over the cached states (one per slot; P in pair mode) of every query row.
 //
 // HBM-bound streaming kernel.  A block owns ROWS consecutive rows (b, h, l) of the cache.  For each
 // KV partition j those rows are one contiguous run of ROWS * D state elements, which one thread
@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
     constexpr int VEC = Cf::VEC, TPR = Cf::TPR;
     constexpr int NS = DT_MAX_P + 1;   // sources per row at most: P slots + the composed state
     extern __shared__ __align__(128) uint8_t smem[];
-    const int P = p.P;
+    const int P = p.S;   // sources in the cache: one per slot
     constexpr int EXTRA = (MODE == MERGE_PLANNED) ? 1 : 0;
     const int nslots = P + EXTRA;
     const int staged = (MODE == MERGE_ALL) ? P : MERGE_CHUNK;
@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
         const int l = (int)(row % p.L);
         int i = 0;
 #pragma unroll 1
-        while (i + 1 < P && p.off_val[i + 1] <= l) ++i;
+        while (i + 1 < p.P && p.off_val[i + 1] <= l) ++i;
         return i;
     };
     // per query partition, bit j set = slot j takes part (prepared on the device from the mask)
@@ -159,9 +159,9 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
             // two ends and those between them matter
             uint32_t need = 0;
             const int i0 = partition_of(row0), i1 = partition_of(row0 + valid - 1);
-            if (valid >= p.L) { for (int i = 0; i < P; ++i) need |= __ldg(p.sel_bits + i); }   // a block longer than the sequence
+            if (valid >= p.L) { for (int i = 0; i < p.P; ++i) need |= __ldg(p.sel_bits + i); }   // a block longer than the sequence
             else if (i0 <= i1 && (row0 % p.L) + valid <= p.L) { for (int i = i0; i <= i1; ++i) need |= __ldg(p.sel_bits + i); }
-            else { for (int i = 0; i < P; ++i) if (i >= i0 || i <= i1) need |= __ldg(p.sel_bits + i); }   // wraps into the next (b, h)
+            else { for (int i = 0; i < p.P; ++i) if (i >= i0 || i <= i1) need |= __ldg(p.sel_bits + i); }   // wraps into the next (b, h)
             nsrc = 0;
             for (int j = 0; j < P; ++j) if (need >> j & 1u) src_s[nsrc++] = (uint8_t)j;
             if (MODE == MERGE_PLANNED) src_s[nsrc++] = (uint8_t)P;
@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
         const int r = e / nslots, j = e - r * nslots;
         float x = -INFINITY;
         if (j < P) {
-            const uint32_t sel = (MODE == MERGE_ALL) ? all_bits : sel_of(row0 + r);
+            const uint32_t sel = (MODE == MERGE_ALL && p.sel_bits == nullptr) ? all_bits : sel_of(row0 + r);
             if (sel >> j & 1u) x = __ldg(p.lse_state + (long long)j * p.R + row0 + r);
         } else {
             x = __ldg(p.comp_lse + row0 + r);
@@ -246,8 +246,8 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
 template <typename StateT, int D, int MODE>
 cudaError_t launch_mode(const MergeParams &p, cudaStream_t stream) {
     using Cf = MergeCfg<StateT, D>;
-    const int rows = Cf::rows(MODE, p.P);
-    const size_t smem = Cf::smem_bytes(MODE, p.P);
+    const int rows = Cf::rows(MODE, p.S);
+    const size_t smem = Cf::smem_bytes(MODE, p.S);
     const long long blocks = (p.R + rows - 1) / rows;
     if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(state_merge_kernel<StateT, D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -265,20 +265,22 @@ cudaError_t launch(const MergeParams &p, cudaStream_t stream) {
 }
 
 // mask -> per query partition the bit set of slots that take part (REUSE slots for the composition,
-// COMPUTE slots for the planned merge)
-__global__ void merge_select_kernel(const uint8_t *mask, int P, int want_compute, uint32_t *sel_bits) {
+// COMPUTE slots for the planned merge); slots that do not exist for the partition never do
+__global__ void merge_select_kernel(const uint8_t *mask, const uint32_t *nonempty, int P, int S, int want_compute,
+                                    uint32_t *sel_bits) {
     const int i = threadIdx.x;
     if (i >= P) return;
     uint32_t bits = 0;
-    for (int j = 0; j < P; ++j)
-        if ((mask[i * P + j] != 0) == (want_compute != 0)) bits |= 1u << j;
-    sel_bits[i] = bits;
+    for (int j = 0; j < S; ++j)
+        if ((mask[i * S + j] != 0) == (want_compute != 0)) bits |= 1u << j;
+    sel_bits[i] = nonempty ? (bits & nonempty[i]) : bits;
 }
 
 }  // namespace
 
-cudaError_t launch_merge_select(const uint8_t *mask, int P, int want_compute, uint32_t *sel_bits, cudaStream_t stream) {
-    merge_select_kernel<<<1, 32, 0, stream>>>(mask, P, want_compute, sel_bits);
+cudaError_t launch_merge_select(const uint8_t *mask, const uint32_t *nonempty, int P, int S, int want_compute,
+                                uint32_t *sel_bits, cudaStream_t stream) {
+    merge_select_kernel<<<1, 32, 0, stream>>>(mask, nonempty, P, S, want_compute, sel_bits);
     return cudaGetLastError();
 }
 

@@ -1,0 +1,224 @@
+"""GPU parity of the grouped state cache (Section 4.2.1, 4.2.2; Eq. 15) through the C ABI against the oracle's
+definition (group state = composition of member states).  Same tolerances as the pair-mode tests."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2607_15650_b200 import binding, build, inputs
+from tests.test_gpu_parity import check_lse, check_o
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    binding.lib()
+
+
+class GroupRun:
+    def __init__(self, wl, g, offsets=None, state_dtype=binding.DT_STATE_FP32, seed=0, rows_by_bh=None):
+        self.wl, self.g = wl, g
+        self.off = wl.offsets() if offsets is None else np.asarray(offsets, dtype=np.int32)
+        self.P = self.off.size - 1
+        self.dev = torch.device("cuda", 0)
+        self.ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, self.off, wl.scale, state_dtype, 0, group_size=g)
+        self.gen = inputs.StepInputs(wl, seed=seed, device=self.dev)
+        if rows_by_bh is None:
+            rows_by_bh = {(b, h): np.arange(wl.L, dtype=np.int32) for b in range(wl.B) for h in range(wl.H)}
+        self.rows = rows_by_bh
+        self.ses = orc.GroupedOracleSession(wl.B, wl.L, wl.H, wl.D, self.off, wl.scale, rows_by_bh, g)
+        self.out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=self.dev)
+        self.lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=self.dev)
+        self.t = 0
+
+    @property
+    def S(self):
+        return self.ctx.dt_num_slots()[0]
+
+    def check_layout(self):
+        S, g = self.ctx.dt_num_slots()
+        assert (S, g) == (self.ses.S, self.ses.g)
+        rng = self.ctx.dt_slot_ranges()
+        for i in range(self.P):
+            for s in range(S):
+                keys = np.concatenate([np.arange(rng[i, s, 0], rng[i, s, 0] + rng[i, s, 1]),
+                                       np.arange(rng[i, s, 2], rng[i, s, 2] + rng[i, s, 3])])
+                want = [x for j in self.ses.members[i][s] for x in range(self.off[j], self.off[j + 1])]
+                assert keys.tolist() == want, (i, s)
+
+    def check_merged(self, what):
+        out_h, lse_h = self.out.float().cpu().numpy(), self.lse.cpu().numpy()
+        for (b, h), rows in self.rows.items():
+            ro, rl = orc.merge(self.ses.o[(b, h)], self.ses.lse[(b, h)])
+            check_o(out_h[b, rows, h, :], ro, f"{what} head {h} merged")
+            check_lse(lse_h[b, h, rows], rl, f"{what} head {h} merged")
+
+    def check_states(self, what):
+        o_st = self.ctx.o_state.float().cpu().numpy()
+        l_st = self.ctx.lse_state.cpu().numpy()
+        for (b, h), rows in self.rows.items():
+            part = np.searchsorted(self.off, rows, side="right") - 1
+            for s in range(self.ses.S):
+                exists = np.array([bool(self.ses.members[i][s]) for i in part])
+                if not exists.any():
+                    continue
+                check_o(o_st[s, b, h, rows[exists], :], self.ses.o[(b, h)][exists, s, :], f"{what} slot {s}")
+                check_lse(l_st[s, b, h, rows[exists]], self.ses.lse[(b, h)][exists, s], f"{what} slot {s}")
+
+    def step(self, mask, check_states=True):
+        self.t += 1
+        q, k, v = self.gen.next()
+        mask = np.ascontiguousarray(mask, dtype=np.uint8).reshape(self.P, self.S)
+        self.ctx.dt_attn_states(q, k, v, torch.from_numpy(mask).to(self.dev), self.t)
+        self.ctx.dt_state_merge(self.out, self.lse)
+        torch.cuda.synchronize()
+        self.ctx.dt_poll()
+        qb, kb, vb = (inputs.bf16_bits(x) for x in (q, k, v))
+        self.ses.step(qb, kb, vb, mask, self.t)
+        self.check_merged(f"step {self.t}")
+        if check_states:
+            self.check_states(f"step {self.t}")
+        tc = self.ctx.dt_get_tc()
+        exists = np.array([[bool(self.ses.members[i][s]) for s in range(self.S)] for i in range(self.P)])
+        assert (tc[exists] == self.ses.tc[exists]).all()
+        return q, k, v
+
+
+@pytest.mark.parametrize("g", [2, 3, 4])
+def test_group_states_config0(g):
+    """Correctness config (1024 tokens, P = 4): every slot computed, then only the local slot and one group."""
+    wl = inputs.WORKLOADS["c0_correctness"]
+    run = GroupRun(wl, g)
+    run.check_layout()
+    S = run.S
+    run.step(np.ones((4, S), np.uint8))
+    m = np.zeros((4, S), np.uint8); m[:, 0] = 1; m[:, S - 1] = 1
+    run.step(m)
+    assert run.ctx.dt_launch_count() == 6
+
+
+@pytest.mark.parametrize("D,grid,n_text,offsets,g", [
+    (128, (4, 11, 13), 0, [0, 129, 385, 572], 2),               # own group with keys on one side only
+    (64, (5, 12, 13), 3, [0, 100, 300, 520, 700, 783], 3),       # own group with a hole; last group of two
+    (128, (3, 9, 11), 5, [0, 60, 100, 230, 302], 3),             # last group is one partition: no own-group slot for it
+    (64, (4, 16, 16), 0, [0, 200, 290, 640, 700, 1024], 5),      # one group: slot 1 = everything but the local keys
+])
+def test_group_states_ragged(D, grid, n_text, offsets, g):
+    wl = inputs.Workload("ragged_groups", 1, 3, D, grid, n_text, len(offsets) - 1, 2, 0.05)
+    assert wl.L == offsets[-1]
+    P = len(offsets) - 1
+    run = GroupRun(wl, g, offsets=offsets, seed=4)
+    run.check_layout()
+    run.step(np.ones((P, run.S), np.uint8))
+    m = np.zeros((P, run.S), np.uint8); m[:, 0] = 1; m[::2, 1] = 1
+    run.step(m)
+
+
+def test_group_states_bf16_cache_and_batch_two():
+    wl = inputs.Workload("b2g", 2, 2, 128, (2, 10, 13), 0, 4, 2, 0.05)
+    run = GroupRun(wl, 2, state_dtype=binding.DT_STATE_BF16, seed=3)
+    run.step(np.ones((4, run.S), np.uint8))
+    m = np.zeros((4, run.S), np.uint8); m[:, 0] = 1; m[1, 2] = 1
+    run.step(m)
+
+
+def test_reuse_of_an_empty_slot_is_reported_and_missing_slots_are_not():
+    wl = inputs.Workload("empty", 1, 2, 64, (2, 8, 9), 0, 3, 1, 0.05)      # groups {0,1} {2}: partition 2 has no slot 2
+    run = GroupRun(wl, 2)
+    q, k, v = run.gen.next()
+    m = np.zeros((3, run.S), np.uint8); m[:, 0] = 1
+    run.ctx.dt_attn_states(q, k, v, torch.from_numpy(m).to(run.dev), 1)
+    torch.cuda.synchronize()
+    with pytest.raises(binding.DitangoError) as e:
+        run.ctx.dt_poll()
+    assert e.value.status == binding.DT_ERR_STATE
+    full = np.ones((3, run.S), np.uint8); full[2, 2] = 0                   # the slot that does not exist: REUSE is fine
+    run.ctx.dt_attn_states(q, k, v, torch.from_numpy(full).to(run.dev), 2)
+    run.ctx.dt_attn_states(q, k, v, torch.from_numpy(m).to(run.dev), 3)
+    torch.cuda.synchronize()
+    run.ctx.dt_poll()
+
+
+@pytest.mark.parametrize("state_dtype", [binding.DT_STATE_FP32, binding.DT_STATE_BF16])
+def test_dynamic_group_compose_in_place(state_dtype):
+    """Eq. 15: g = 2 -> 4 -> 8 in place; each composed cache is compared slot by slot with the oracle's
+    composition, keeps merging to the same output, and takes further selective steps."""
+    wl = inputs.Workload("compose", 1, 2, 64, (4, 12, 13), 0, 8, 3, 0.05)
+    run = GroupRun(wl, 2, seed=9, state_dtype=state_dtype)
+    run.step(np.ones((8, run.S), np.uint8))
+    m = np.zeros((8, run.S), np.uint8); m[:, 0] = 1; m[:, 2] = 1
+    run.step(m)
+    for expect_S in (3, 2):
+        run.ctx.dt_group_compose()
+        run.ses.compose()
+        run.check_layout()
+        assert run.S == expect_S
+        torch.cuda.synchronize()
+        run.ctx.dt_poll()
+        run.check_states(f"composed to S={expect_S}")
+        run.ctx.dt_state_merge(run.out, run.lse)
+        torch.cuda.synchronize()
+        run.check_merged(f"composed to S={expect_S}")
+        tc = run.ctx.dt_get_tc()
+        assert (tc == run.ses.tc).all()
+        m = np.zeros((8, run.S), np.uint8); m[:, 0] = 1; m[3:, 1] = 1
+        run.step(m)
+    with pytest.raises(binding.DitangoError) as e:
+        run.ctx.dt_group_compose()
+    assert e.value.status == binding.DT_ERR_STATE
+    run.ctx.dt_group_reset()
+    run.ses.reset()
+    run.check_layout()
+    assert (run.ctx.dt_get_tc() == -1).all()
+    run.step(np.ones((8, run.S), np.uint8))
+
+
+def test_slot_plan_matches_oracle_rule():
+    """dt_plan on a grouped cache: W per slot against the oracle's slot importance; decisions bit-exact
+    against the oracle rule applied to the GPU's own W (threshold and target fraction)."""
+    wl = inputs.WORKLOADS["c0_correctness"]
+    P = 8
+    off = orc.uniform_offsets(wl.L, P)
+    run = GroupRun(wl, 2, offsets=off)
+    S = run.S
+    run.step(np.ones((P, S), np.uint8), check_states=False)
+    mem = run.ses.members
+    lse_slots = run.ctx.lse_state.double().cpu().numpy()
+    W_ref = orc.slot_contribution(lse_slots, off, mem)
+    mask_dev = torch.zeros(P * S, dtype=torch.uint8, device=run.dev)
+    w_dev = torch.zeros(P * S, dtype=torch.float64, device=run.dev)
+    eps_dev = torch.zeros(1, dtype=torch.float64, device=run.dev)
+    for kwargs in (dict(eps=0.05), dict(eps=0.2), dict(target_fraction=0.4), dict(target_fraction=0.75),
+                   dict(target_fraction=1.0), dict(target_fraction=0.0)):
+        run.ctx.dt_plan(mask_dev, w_dev=w_dev, eps_out_dev=eps_dev, **kwargs)
+        torch.cuda.synchronize()
+        W = w_dev.cpu().numpy().reshape(P, S)
+        np.testing.assert_allclose(W, W_ref, rtol=0, atol=2e-6)
+        want, eps_want = orc.slot_plan(W, mem, 2, **kwargs)
+        assert (mask_dev.cpu().numpy().reshape(P, S) == want).all(), kwargs
+        assert eps_dev.item() == pytest.approx(eps_want, abs=1e-15)
+    with pytest.raises(binding.DitangoError) as e:
+        run.ctx.dt_plan_grouped(mask_dev, 2)
+    assert e.value.status == binding.DT_ERR_UNSUPPORTED
+
+
+def test_composed_reuse_state_on_a_grouped_cache():
+    """dt_compose_reuse / dt_state_merge_planned with [P][S] masks."""
+    wl = inputs.Workload("planned", 1, 2, 128, (3, 10, 12), 0, 6, 2, 0.05)
+    run = GroupRun(wl, 2, seed=6)
+    S = run.S
+    run.step(np.ones((6, S), np.uint8), check_states=False)
+    m = np.zeros((6, S), np.uint8); m[:, 0] = 1; m[:3, 1] = 1; m[4, 3] = 1
+    q, k, v = run.step(m, check_states=False)
+    mask_dev = torch.from_numpy(m.reshape(-1)).to(run.dev)
+    comp_o = torch.empty((wl.B, wl.H, wl.L, wl.D), dtype=torch.float32, device=run.dev)
+    comp_l = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=run.dev)
+    run.ctx.dt_compose_reuse(mask_dev, comp_o, comp_l)
+    out2 = torch.empty_like(run.out); lse2 = torch.empty_like(run.lse)
+    run.ctx.dt_state_merge_planned(mask_dev, comp_o, comp_l, out2, lse2)
+    torch.cuda.synchronize()
+    run.ctx.dt_poll()
+    run.out, run.lse = out2, lse2
+    run.check_merged("planned merge")
