@@ -114,12 +114,35 @@ def computed_flops(wl, mask: np.ndarray) -> float:
     return 4.0 * wl.D * wl.H * wl.B * float((np.outer(n, n) * (mask.reshape(wl.P, wl.P) != 0)).sum())
 
 
-def merge_bytes(wl, state_bytes: int) -> float:
-    return float(wl.L) * wl.H * wl.B * (wl.P * (wl.D * state_bytes + 4) + 2 * wl.D + 4)
+def merge_bytes(wl, state_bytes: int, slots=None) -> float:
+    S = wl.P if slots is None else slots
+    return float(wl.L) * wl.H * wl.B * (S * (wl.D * state_bytes + 4) + 2 * wl.D + 4)
 
 
-def plan_bytes(wl) -> float:
-    return float(wl.L) * wl.H * wl.B * wl.P * 4
+def plan_bytes(wl, slots=None) -> float:
+    return float(wl.L) * wl.H * wl.B * (wl.P if slots is None else slots) * 4
+
+
+def slot_members(P: int, g: int):
+    """KV partitions behind every (query partition, slot) of a grouped cache: slot 0 = the local partition,
+    slot 1 + k = group k of g adjacent partitions without the local one (structure only, no arithmetic)."""
+    m = (P + g - 1) // g
+    return [[[i]] + [[j for j in range(k * g, min(P, (k + 1) * g)) if j != i] for k in range(m)] for i in range(P)]
+
+
+def slot_mask_to_pairs(mask: np.ndarray, P: int, g: int) -> np.ndarray:
+    """[P][S] slot decisions -> the [P][P] pair mask they stand for."""
+    if g <= 1:
+        return mask.reshape(P, P)
+    mem = slot_members(P, g)
+    S = len(mem[0])
+    mask = mask.reshape(P, S)
+    pairs = np.zeros((P, P), np.uint8)
+    for i in range(P):
+        for sl in range(S):
+            if mask[i, sl]:
+                pairs[i, mem[i][sl]] = 1
+    return pairs
 
 
 def dist_info():
@@ -232,14 +255,15 @@ def run_cuda(args, wl):
     state_dtype = binding.DT_STATE_BF16 if args.state_dtype == "bf16" else binding.DT_STATE_FP32
     sbytes = 2 if args.state_dtype == "bf16" else 4
 
-    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale, state_dtype, local)
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale, state_dtype, local, group_size=args.group_size)
+    S, g = ctx.dt_num_slots()
     gen = inputs.StepInputs(wl, seed=0, device=dev)
     steps_in = [gen.next() for _ in range(wl.steps)]          # resident bf16 inputs of every denoising step
     del gen
     torch.cuda.empty_cache()
     out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
     lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
-    PP = wl.P * wl.P
+    PP = wl.P * S            # decisions per plan: [P][S] (S = P without grouping)
     masks = [torch.ones(PP, dtype=torch.uint8, device=dev), torch.ones(PP, dtype=torch.uint8, device=dev)]
     ones = torch.ones(PP, dtype=torch.uint8, device=dev)
     W = torch.empty(PP, dtype=torch.float64, device=dev)
@@ -321,9 +345,10 @@ def run_cuda(args, wl):
     attn_ms = [e[0].elapsed_time(e[1]) for e in timers]
     merge_ms = [e[1].elapsed_time(e[2]) for e in timers]
     plan_ms = [e[2].elapsed_time(e[3]) for e in timers]
-    mask_np = masks[cur].cpu().numpy()
+    mask_np = slot_mask_to_pairs(masks[cur].cpu().numpy(), wl.P, g)   # as pairs: a slot stands for its members
     comp_fl = computed_flops(wl, mask_np)           # pair count is fixed by the target fraction
     n_comp = int((mask_np != 0).sum())
+    n_slots_comp = int((masks[cur] != 0).sum().item())
     value = aggregate_throughput(full_flops(wl) / 1e12, ms_per_step / 1e3, world)
 
     if rank != 0:
@@ -383,7 +408,9 @@ def run_cuda(args, wl):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "D": wl.D, "L": wl.L, "P": wl.P,
-                   "computed_pairs": n_comp, "computed_pair_fraction": n_comp / PP, "state_dtype": args.state_dtype,
+                   "computed_pairs": n_comp, "computed_pair_fraction": n_comp / (wl.P * wl.P),
+                   "group_size": g, "cache_slots": S, "computed_slots": n_slots_comp, "state_dtype": args.state_dtype,
+                   "cache_gb": S * wl.B * wl.H * wl.L * (wl.D * sbytes + 4) / 1e9,
                    "step": ("dt_attn_states + dt_state_merge_planned + dt_plan" if args.composed
                             else "dt_attn_states + dt_state_merge + dt_plan"), "multi_gpu": "independent replicas",
                    "l2": "inputs (%.1f GB) and state cache larger than L2; no flush" %
@@ -394,7 +421,8 @@ def run_cuda(args, wl):
         "roofline": {"kernel": "attn_states_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
                      "unit": "TFLOP/s", "frac": achieved / peak,
                      "traffic": (NCU_ATTN_TRAFFIC_PER_HEAD_PAIR[args.workload] * wl.H * n_comp
-                                 if args.workload in NCU_ATTN_TRAFFIC_PER_HEAD_PAIR and args.state_dtype == "fp32" else None),
+                                 if args.workload in NCU_ATTN_TRAFFIC_PER_HEAD_PAIR and args.state_dtype == "fp32" and g == 1
+                                 else None),
                      "traffic_note": "bytes per launch, ncu dram read+write of a 4-head capture scaled by heads x pairs",
                      "peak_source": f"{peaks['source']} bf16 sustained", "frac_of_burst": achieved / peaks["bf16_tflops"],
                      "frac_of_nominal_2250": achieved / 2250.0, "launch_ms": attn_avg_ms,
@@ -402,9 +430,9 @@ def run_cuda(args, wl):
         "cpu_baseline": cpu,
         "kernels": {
             "attn_ms": attn_avg_ms, "merge_ms": float(np.mean(merge_ms)), "plan_ms": float(np.mean(plan_ms)),
-            "merge_gbs": merge_bytes(wl, sbytes) / 1e9 / (float(np.mean(merge_ms)) / 1e3),
-            "merge_frac_of_hbm": merge_bytes(wl, sbytes) / 1e9 / (float(np.mean(merge_ms)) / 1e3) / peaks["hbm_gbs"],
-            "plan_gbs": plan_bytes(wl) / 1e9 / (float(np.mean(plan_ms)) / 1e3),
+            "merge_gbs": merge_bytes(wl, sbytes, S) / 1e9 / (float(np.mean(merge_ms)) / 1e3),
+            "merge_frac_of_hbm": merge_bytes(wl, sbytes, S) / 1e9 / (float(np.mean(merge_ms)) / 1e3) / peaks["hbm_gbs"],
+            "plan_gbs": plan_bytes(wl, S) / 1e9 / (float(np.mean(plan_ms)) / 1e3),
             "hbm_peak_gbs": peaks["hbm_gbs"], "compose_once_ms": compose_ms,
         },
         "vs_all_compute": {"all_compute_attn_ms": full_attn_ms, "all_compute_step_ms": full_step_ms,
@@ -429,6 +457,8 @@ def main():
     ap.add_argument("--composed", action="store_true",
                     help="compose the plan's REUSE states once after the anchor step and merge COMPUTE states + that "
                          "composed state in the selective steps (the plan then stays fixed between anchors)")
+    ap.add_argument("--group-size", type=int, default=1,
+                    help="g >= 2: grouped state cache (ceil(P/g) + 1 slots per row; group states computed in one pass)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -212,11 +212,15 @@ dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double
  *                    doubles, S becomes ceil(m/2) + 1; t_c of a new slot is the older of its sources' (-1 if one
  *                    was never computed).  The memory behind the first S slots of the bound buffers is no
  *                    longer used.  DT_ERR_STATE if only one group is left.  Synchronises the stream.
+ * dt_group_fit       the memory-driven trigger of Section 4.2: while the slots in use (S * B*H*L * (D*sizeof(state) + 4)
+ *                    bytes) exceed max_bytes and more than one group is left, dt_group_compose; *composed (may be
+ *                    NULL) = how many times.  DT_ERR_STATE if one group is left and the budget is still exceeded.
  * dt_group_reset     back to the creation-time g (an anchor step recomputes every state): all t_c = -1, the
  *                    cache contents are stale until the next all-COMPUTE step.  Synchronises the stream. */
 dt_status dt_num_slots(dt_ctx *ctx, int32_t *slots, int32_t *group_size);
 dt_status dt_slot_ranges(dt_ctx *ctx, int32_t *ranges_host);
 dt_status dt_group_compose(dt_ctx *ctx, void *stream);
+dt_status dt_group_fit(dt_ctx *ctx, size_t max_bytes, int32_t *composed, void *stream);
 dt_status dt_group_reset(dt_ctx *ctx, void *stream);
 
 /* The same plan computation for callers that cannot allocate device memory at the point of the

@@ -23,7 +23,7 @@ EXPORTS = [
     "dt_compose_reuse", "dt_state_merge_planned", "dt_plan", "dt_plan_grouped", "dt_planner_init", "dt_planner_step", "dt_planner_commit", "dt_planner_get",
     "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
     "dt_launch_count", "dt_selftest_wait_timeout", "dt_poll", "dt_status_str", "dt_last_error",
-    "dt_num_slots", "dt_slot_ranges", "dt_group_compose", "dt_group_reset",
+    "dt_num_slots", "dt_slot_ranges", "dt_group_compose", "dt_group_fit", "dt_group_reset",
 ]
 
 
@@ -87,6 +87,7 @@ def lib():
         "dt_num_slots": (C.c_int, [vp, i32p, i32p]),
         "dt_slot_ranges": (C.c_int, [vp, i32p]),
         "dt_group_compose": (C.c_int, [vp, vp]),
+        "dt_group_fit": (C.c_int, [vp, C.c_size_t, i32p, vp]),
         "dt_group_reset": (C.c_int, [vp, vp]),
         "dt_status_str": (C.c_char_p, [C.c_int]),
         "dt_last_error": (C.c_char_p, [vp]),
@@ -288,6 +289,12 @@ class Context:
 
     def dt_group_compose(self, stream=None):
         self._check(lib().dt_group_compose(self._h, _stream_ptr(stream)))
+
+    def dt_group_fit(self, max_bytes, stream=None) -> int:
+        """Compose groups (Eq. 15) until the slots in use fit into max_bytes; returns how many compositions ran."""
+        n = C.c_int32()
+        self._check(lib().dt_group_fit(self._h, int(max_bytes), C.byref(n), _stream_ptr(stream)))
+        return int(n.value)
 
     def dt_group_reset(self, stream=None):
         self._check(lib().dt_group_reset(self._h, _stream_ptr(stream)))

@@ -674,6 +674,22 @@ dt_status dt_group_compose(dt_ctx *ctx, void *stream) {
     return DT_OK;
 }
 
+dt_status dt_group_fit(dt_ctx *ctx, size_t max_bytes, int32_t *composed, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (composed) *composed = 0;
+    if (ctx->group_size0 <= 1) return fail(ctx, DT_ERR_UNSUPPORTED, "dt_group_fit needs a grouped cache (dt_config.group_size >= 2)");
+    const dt_config &c = ctx->cfg;
+    const size_t per_slot = (size_t)c.B * c.H * c.L * (c.D * state_elem_bytes(c.state_dtype) + 4);
+    int n = 0;
+    while ((size_t)ctx->S * per_slot > max_bytes && ctx->S - 1 >= 2) {
+        dt_status s = dt_group_compose(ctx, stream);
+        if (s != DT_OK) return s;
+        ++n;
+    }
+    if (composed) *composed = n;
+    return (size_t)ctx->S * per_slot > max_bytes ? fail(ctx, DT_ERR_STATE, "one group left and the cache is still above the budget") : DT_OK;
+}
+
 dt_status dt_group_reset(dt_ctx *ctx, void *stream) {
     if (!ctx) return DT_ERR_INVALID_ARG;
     if (ctx->group_size0 <= 1) return fail(ctx, DT_ERR_UNSUPPORTED, "dt_group_reset needs a grouped cache (dt_config.group_size >= 2)");

@@ -99,3 +99,69 @@ def test_full_size_c2_wan480p_uneven_partitions():
 def test_full_size_c4_hunyuan_p32_bf16_state_cache():
     """Largest footprint: 118 800 tokens, P = 32 (3712/3713-row partitions), states cached in bf16."""
     _run_full_size("c4_hunyuan720p", 0.125, n_samples=32, n_selective=1, state_dtype=binding.DT_STATE_BF16)
+
+
+def test_full_size_c4_hunyuan_grouped_cache_and_dynamic_compose():
+    """Grouped cache at the largest footprint (P = 32, g = 4: 9 slots instead of 32): anchor step, per-slot plan,
+    one selective step, then Dynamic Group State Compose (g -> 8, 5 slots) and another selective step -- sampled
+    rows against the oracle's member-by-member composition."""
+    build.build()
+    wl = inputs.WORKLOADS["c4_hunyuan720p"]
+    dev = torch.device("cuda", 0)
+    off, P, g = wl.offsets(), wl.P, 4
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, off, wl.scale, binding.DT_STATE_FP32, group_size=g)
+    S = ctx.dt_num_slots()[0]
+    assert S == 9
+    gen = inputs.StepInputs(wl, seed=0, device=dev)
+    rows = inputs.sample_rows(wl, 24, seed=12)
+    ses = orc.GroupedOracleSession(wl.B, wl.L, wl.H, wl.D, off, wl.scale, rows, g)
+    out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+
+    def check(what):
+        for (b, h), r in rows.items():
+            ridx = torch.from_numpy(r.astype(np.int64)).to(dev)
+            ro, rl = orc.merge(ses.o[(b, h)], ses.lse[(b, h)])
+            eo = np.abs(out[b, ridx, h].float().cpu().numpy() - ro)
+            el = np.abs(lse[b, h, ridx].cpu().numpy() - rl)
+            assert eo.max() <= O_MAX and eo.mean() <= O_MEAN and el.max() <= LSE_ABS, (what, b, h, eo.max(), el.max())
+            st_o = ctx.o_state[:ses.S, b, h][:, ridx].float().cpu().numpy().transpose(1, 0, 2)
+            st_l = ctx.lse_state[:ses.S, b, h][:, ridx].cpu().numpy().T
+            assert np.abs(st_o - ses.o[(b, h)]).max() <= O_MAX, what
+            assert np.abs(st_l - ses.lse[(b, h)]).max() <= LSE_ABS, what
+
+    def step(t, mask):
+        q, k, v = gen.next()
+        ctx.dt_attn_states(q, k, v, mask, t)
+        ctx.dt_state_merge(out, lse)
+        torch.cuda.synchronize()
+        ctx.dt_poll()
+        ses.step(*(inputs.bf16_bits(x) for x in (q, k, v)), mask.cpu().numpy().reshape(P, -1), t)
+        check(f"step {t}")
+        assert (ctx.dt_get_tc() == ses.tc).all()
+
+    mask = torch.ones(P * S, dtype=torch.uint8, device=dev)
+    step(0, mask)
+    W = torch.empty(P * S, dtype=torch.float64, device=dev)
+    eps = torch.empty(1, dtype=torch.float64, device=dev)
+    ctx.dt_plan(mask, target_fraction=0.25, w_dev=W, eps_out_dev=eps)
+    torch.cuda.synchronize()
+    Wg = W.cpu().numpy().reshape(P, S)
+    W_ref = orc.slot_contribution(ctx.lse_state.cpu().numpy().astype(np.float64), off, ses.members)
+    np.testing.assert_allclose(Wg, W_ref, rtol=2e-5, atol=1e-10)
+    want, eps_want = orc.slot_plan(Wg, ses.members, g, target_fraction=0.25)
+    assert (mask.cpu().numpy().reshape(P, S) == want).all() and eps.item() == eps_want
+    pairs = sum(len(ses.members[i][s]) for i in range(P) for s in range(S) if want[i, s])
+    assert P <= pairs <= round(0.25 * P * P)
+    step(1, mask)
+    ctx.dt_group_compose()
+    ses.compose()
+    assert ctx.dt_num_slots() == (5, 8) and ses.S == 5
+    ctx.dt_state_merge(out, lse)
+    torch.cuda.synchronize()
+    ctx.dt_poll()
+    check("after compose")
+    mask2 = torch.zeros(P * 5, dtype=torch.uint8, device=dev)
+    mask2.view(P, 5)[:, 0] = 1
+    mask2.view(P, 5)[::3, 2] = 1
+    step(2, mask2)

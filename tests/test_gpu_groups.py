@@ -222,3 +222,23 @@ def test_composed_reuse_state_on_a_grouped_cache():
     run.ctx.dt_poll()
     run.out, run.lse = out2, lse2
     run.check_merged("planned merge")
+
+
+def test_memory_budget_triggers_group_compose():
+    """Section 4.2 (Dynamic Group State Compose): compositions run until the slots in use fit the byte budget."""
+    wl = inputs.Workload("fit", 1, 2, 64, (4, 12, 13), 0, 8, 2, 0.05)
+    run = GroupRun(wl, 2, seed=10)
+    run.step(np.ones((8, run.S), np.uint8), check_states=False)
+    per_slot = wl.B * wl.H * wl.L * (wl.D * 4 + 4)
+    assert run.ctx.dt_group_fit(5 * per_slot) == 0 and run.S == 5          # already fits
+    assert run.ctx.dt_group_fit(3 * per_slot + 1) == 1 and run.S == 3      # g 2 -> 4
+    run.ses.compose()
+    run.check_layout()
+    torch.cuda.synchronize()
+    run.check_states("fit to 3 slots")
+    with pytest.raises(binding.DitangoError) as e:                          # g -> 8 leaves 2 slots: still above 1 slot
+        run.ctx.dt_group_fit(per_slot)
+    assert e.value.status == binding.DT_ERR_STATE and run.S == 2
+    run.ses.compose()
+    torch.cuda.synchronize()
+    run.check_states("fit to 2 slots")
