@@ -190,7 +190,8 @@ dt_status dt_planner_init(dt_ctx *ctx, const dt_planner_config *pc, void *snap_o
 dt_status dt_planner_step(dt_ctx *ctx, uint8_t *mask_dev, int32_t *is_anchor_dev, double *ase_dev, double *delta_rel_dev,
                           void *stream);
 dt_status dt_planner_commit(dt_ctx *ctx, void *stream);
-/* Copy the planner state to the host (synchronises): w and alpha are double [P*P]; any pointer may be NULL. */
+/* Copy the planner state to the host (synchronises): w and alpha are double [P*S] (S = P in pair mode); any
+ * pointer may be NULL. */
 dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double *eps_host, int32_t *have_anchor_host);
 
 /* Grouped state cache (Section 4.2.1, Section 4.2.2; Dynamic Group State Compose, Eq. 15).  With
@@ -203,7 +204,10 @@ dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double
  *                      Eq. 12); one decision per non-local slot, the local slot 0 always COMPUTE; the target
  *                      fraction still counts pairs: K = round(f*P*P), a slot costs as many as it has members
  *   dt_get_tc / dt_set_tc, dt_step_host   arrays are [P*S]
- *   dt_plan_grouped with group_size > 1 and the dt_planner_* calls return DT_ERR_UNSUPPORTED.
+ *   dt_planner_*       Algorithm 1 with one unit per non-local slot: w, alpha, ASE and the mask are [P*S]; a group
+ *                      state is one state, so ASE(i, G) = w(i, G) * alpha(i, G) * ||AS_t(i,i) - AS_ta(i,i)||_2 with
+ *                      alpha from the norm of the group state (dt_planner_config.group_size must be 1)
+ *   dt_plan_grouped with group_size > 1 returns DT_ERR_UNSUPPORTED (the slots already are the groups).
  * dt_num_slots       current S and g (either pointer may be NULL).
  * dt_slot_ranges     key ranges of every (query partition, slot): int32 [P*S*4] = (r1, n1, r2, n2), the keys
  *                    [r1, r1+n1) and [r2, r2+n2); n1 + n2 == 0 marks a slot that does not exist.
@@ -211,12 +215,14 @@ dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double
  *                    in the cache (new slot 1 + k overwrites old slot 1 + k after both sources were read), g
  *                    doubles, S becomes ceil(m/2) + 1; t_c of a new slot is the older of its sources' (-1 if one
  *                    was never computed).  The memory behind the first S slots of the bound buffers is no
- *                    longer used.  DT_ERR_STATE if only one group is left.  Synchronises the stream.
+ *                    longer used.  If the planner is initialised, its w and alpha are taken again from the
+ *                    composed cache (the anchor's snapshot of the local states stays).  DT_ERR_STATE if only one group is left.  Synchronises the stream.
  * dt_group_fit       the memory-driven trigger of Section 4.2: while the slots in use (S * B*H*L * (D*sizeof(state) + 4)
  *                    bytes) exceed max_bytes and more than one group is left, dt_group_compose; *composed (may be
  *                    NULL) = how many times.  DT_ERR_STATE if one group is left and the budget is still exceeded.
  * dt_group_reset     back to the creation-time g (an anchor step recomputes every state): all t_c = -1, the
- *                    cache contents are stale until the next all-COMPUTE step.  Synchronises the stream. */
+ *                    cache contents are stale until the next all-COMPUTE step; an initialised planner treats its
+ *                    next step as an anchor.  Synchronises the stream. */
 dt_status dt_num_slots(dt_ctx *ctx, int32_t *slots, int32_t *group_size);
 dt_status dt_slot_ranges(dt_ctx *ctx, int32_t *ranges_host);
 dt_status dt_group_compose(dt_ctx *ctx, void *stream);

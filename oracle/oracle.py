@@ -433,3 +433,38 @@ class GroupedOracleSession:
             self.o[bh] = np.zeros((r.size, self.S, self.D))
             self.lse[bh] = np.full((r.size, self.S), -np.inf)
         self.tc = -np.ones((self.P, self.S), dtype=np.int32)
+
+
+def planner_step_slots(W, alpha, members, drift_sq, anchor_local_sq, eps, eps_local, R, have_anchor):
+    """Algorithm 1 on a grouped cache: one unit per non-local slot that exists; a group state is one state, so
+    ASE(i, s) = W[i, s] * alpha[i, s] * delta(i) (Eq. 7, Eq. 10, Eq. 12 with the group as its single member).
+    Same anchor test (Eq. 14), threshold (Eq. 13) and eps update as planner_step.
+    Returns dict(is_anchor, mask [P, S], ase [P, S] (nan where there is no unit), eps, delta_rel)."""
+    W = np.asarray(W, dtype=np.float64); alpha = np.asarray(alpha, dtype=np.float64)
+    P, S = W.shape
+    delta = np.sqrt(np.asarray(drift_sq, dtype=np.float64))
+    ase = np.full((P, S), np.nan)
+    for i in range(P):
+        for s in range(1, S):
+            if members[i][s]:
+                ase[i, s] = W[i, s] * alpha[i, s] * delta[i]
+    vals = ase[~np.isnan(ase)]
+    den = float(np.sum(anchor_local_sq))
+    delta_rel = float(np.sqrt(np.sum(drift_sq) / den)) if den > 0 else 0.0
+    all_exceed = bool(vals.size > 0 and (vals > eps).all())
+    is_anchor = (not have_anchor) or all_exceed or (delta_rel > eps_local)
+    mask = np.zeros((P, S), dtype=np.uint8)
+    mask[:, 0] = 1
+    eps_new = eps
+    if is_anchor:
+        mask[:] = 1
+        if vals.size > 0 and vals.max() > 0.0:
+            a = np.sort(vals)
+            r = min(max(int(np.floor(R * a.size)), 0), a.size)
+            eps_new = 0.0 if r == 0 else (float(a[-1]) if r == a.size else 0.5 * float(a[r - 1] + a[r]))
+    else:
+        for i in range(P):
+            for s in range(1, S):
+                if members[i][s] and ase[i, s] > eps:
+                    mask[i, s] = 1
+    return dict(is_anchor=bool(is_anchor), mask=mask, ase=ase, eps=float(eps_new), delta_rel=delta_rel)

@@ -242,8 +242,8 @@ class Context:
         self._check(lib().dt_planner_commit(self._h, _stream_ptr(stream)))
 
     def dt_planner_get(self):
-        P = self.cfg.P
-        w = np.empty((P, P), dtype=np.float64); alpha = np.empty((P, P), dtype=np.float64)
+        P, S = self.cfg.P, self.dt_num_slots()[0]
+        w = np.empty((P, S), dtype=np.float64); alpha = np.empty((P, S), dtype=np.float64)
         eps = C.c_double(); have = C.c_int32()
         self._check(lib().dt_planner_get(self._h, w.ctypes.data_as(C.c_void_p), alpha.ctypes.data_as(C.c_void_p),
                                          C.byref(eps), C.byref(have)))

@@ -1,6 +1,7 @@
 // C-ABI of libditango: argument checking, tensor-map encoding, launches.  No arithmetic of the
 // method lives here.
 #include <cmath>
+#include <cstddef>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -519,11 +520,14 @@ dt::PlannerParams planner_params(dt_ctx *ctx) {
     p.snap_o_out = ctx->snap_o;
     p.snap_lse_out = ctx->snap_lse;
     p.off = ctx->off_dev;
+    p.nonempty = ctx->nonempty_dev;
     p.local_partials = ctx->planner_local_partials_dev;
     p.norm_partials = ctx->planner_norm_partials_dev;
     p.w_partials = ctx->plan_partials_dev;
-    p.P = c.P; p.BH = c.B * c.H; p.L = c.L; p.D = c.D; p.chunks = ctx->plan_chunks;
+    p.P = c.P; p.S = ctx->S; p.BH = c.B * c.H; p.L = c.L; p.D = c.D; p.chunks = ctx->plan_chunks;
     p.group_size = ctx->planner_group_size;
+    p.group_mode = ctx->group_size0 > 1 ? 1 : 0;
+    p.force = 0;
     p.eps_local = ctx->planner_eps_local;
     p.cache_ratio = ctx->planner_cache_ratio;
     return p;
@@ -535,8 +539,9 @@ dt_status dt_planner_init(dt_ctx *ctx, const dt_planner_config *pc, void *snap_o
     if (!ctx) return DT_ERR_INVALID_ARG;
     if (!pc || !snap_o_dev || !snap_lse_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null pointer");
     const dt_config &c = ctx->cfg;
-    if (ctx->group_size0 > 1) return fail(ctx, DT_ERR_UNSUPPORTED, "the Algorithm 1 planner runs on a pair-mode cache (dt_config.group_size <= 1)");
     if (pc->group_size < 1 || pc->group_size > c.P) return fail(ctx, DT_ERR_INVALID_ARG, "group_size must be in [1, P]");
+    if (ctx->group_size0 > 1 && pc->group_size != 1)
+        return fail(ctx, DT_ERR_UNSUPPORTED, "a grouped cache decides per slot: dt_planner_config.group_size must be 1");
     if (!(pc->eps_initial >= 0.0) || !(pc->eps_local > 0.0) || !(pc->cache_ratio >= 0.0 && pc->cache_ratio <= 1.0))
         return fail(ctx, DT_ERR_INVALID_ARG, "eps_initial >= 0, eps_local > 0 and 0 <= cache_ratio <= 1 required");
     if ((long long)c.B * c.H * c.P > 65535) return fail(ctx, DT_ERR_UNSUPPORTED, "B*H*P exceeds 65535");
@@ -548,7 +553,7 @@ dt_status dt_planner_init(dt_ctx *ctx, const dt_planner_config *pc, void *snap_o
         const size_t BH = (size_t)c.B * c.H;
         bool ok = cudaMalloc(&ctx->planner_state_dev, sizeof(dt::PlannerState)) == cudaSuccess;
         ok = ok && cudaMalloc(&ctx->planner_local_partials_dev, BH * c.P * ctx->plan_chunks * 2 * sizeof(float)) == cudaSuccess;
-        ok = ok && cudaMalloc(&ctx->planner_norm_partials_dev, BH * c.P * ctx->plan_chunks * c.P * sizeof(float)) == cudaSuccess;
+        ok = ok && cudaMalloc(&ctx->planner_norm_partials_dev, BH * c.P * ctx->plan_chunks * ctx->S0 * sizeof(float)) == cudaSuccess;
         if (!ok) return fail(ctx, DT_ERR_CUDA, "planner scratch allocation failed");
     }
     ctx->snap_o = snap_o_dev;
@@ -588,8 +593,8 @@ dt_status dt_planner_commit(dt_ctx *ctx, void *stream) {
     pp.lse_state = ctx->lse_state;
     pp.off = ctx->off_dev;
     pp.partials = ctx->plan_partials_dev;
-    pp.nonempty = nullptr;
-    pp.P = c.P; pp.S = c.P; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
+    pp.nonempty = ctx->group_size0 > 1 ? ctx->nonempty_dev : nullptr;
+    pp.P = c.P; pp.S = ctx->S; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
     pp.R = (long long)c.B * c.H * c.L;
     cudaError_t e = dt::launch_plan_partial(pp, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
@@ -607,7 +612,7 @@ dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double
     cudaError_t e = cudaDeviceSynchronize();
     if (e == cudaSuccess) e = cudaMemcpy(&hs, ctx->planner_state_dev, sizeof hs, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "dt_planner_get");
-    const int n = ctx->cfg.P * ctx->cfg.P;
+    const int n = ctx->cfg.P * ctx->S;
     if (w_host) memcpy(w_host, hs.w, n * sizeof(double));
     if (alpha_host) memcpy(alpha_host, hs.alpha, n * sizeof(double));
     if (eps_host) *eps_host = hs.eps;
@@ -671,6 +676,24 @@ dt_status dt_group_compose(dt_ctx *ctx, void *stream) {
     build_slot_table(ctx, ctx->group_size * 2);
     e = upload_slot_table(ctx, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "group compose table upload");
+    if (ctx->planner_state_dev) {
+        // the planner's w and alpha are indexed by slot: take them again from the composed cache (the importance
+        // of a composed slot is the sum of its sources', its scale ratio needs the composed state's norm)
+        dt::PlanParams pp;
+        pp.lse_state = ctx->lse_state;
+        pp.off = ctx->off_dev;
+        pp.partials = ctx->plan_partials_dev;
+        pp.nonempty = ctx->nonempty_dev;
+        pp.P = c.P; pp.S = ctx->S; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
+        pp.R = (long long)R;
+        e = dt::launch_plan_partial(pp, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
+        dt::PlannerParams p = planner_params(ctx);
+        p.force = 1;
+        e = dt::launch_planner_commit(p, c.state_dtype, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "planner refresh launch");
+        ctx->launches += 3;
+    }
     return DT_OK;
 }
 
@@ -699,6 +722,9 @@ dt_status dt_group_reset(dt_ctx *ctx, void *stream) {
     build_slot_table(ctx, ctx->group_size0);
     e = upload_slot_table(ctx, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(ctx->tc_dev, 0xFF, (size_t)ctx->cfg.P * ctx->S * sizeof(int32_t), st);
+    if (e == cudaSuccess && ctx->planner_state_dev)   // the planner starts over: its next step is an anchor
+        e = cudaMemsetAsync(reinterpret_cast<uint8_t *>(ctx->planner_state_dev) + offsetof(dt::PlannerState, have_anchor), 0,
+                            sizeof(int), st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "group reset");
     return DT_OK;
 }

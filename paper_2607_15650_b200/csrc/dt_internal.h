@@ -113,14 +113,17 @@ struct PlannerParams {
     void *snap_o_out;
     float *snap_lse_out;
     const int32_t *off;           // device, P+1
+    const uint32_t *nonempty;     // device, P words: slots that exist for the query partition
     float *local_partials;        // [BH][P][chunks][2]
-    float *norm_partials;         // [BH][P][chunks][P]
-    const float *w_partials;      // [BH][P][chunks][P] from plan_partial_kernel
-    uint8_t *mask;                // out, P*P
+    float *norm_partials;         // [BH][P][chunks][S]
+    const float *w_partials;      // [BH][P][chunks][S] from plan_partial_kernel
+    uint8_t *mask;                // out, P*S
     int32_t *is_anchor_out;       // out, may be null
-    double *ase_out;              // out, P * n_groups, may be null
+    double *ase_out;              // out, P * n_groups (pair mode) or P * S (grouped cache), may be null
     double *delta_rel_out;        // out, may be null
-    int P, BH, L, D, chunks, group_size;
+    int P, S, BH, L, D, chunks, group_size;
+    int group_mode;               // grouped cache: slot 0 is the local state and every other slot is one unit
+    int force;                    // refresh w and alpha although the step is no anchor (after a group compose)
     double eps_local, cache_ratio;
 };
 

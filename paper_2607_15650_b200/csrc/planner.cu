@@ -52,7 +52,8 @@ template <typename StateT>
 __global__ void __launch_bounds__(PL_THREADS) planner_local_kernel(PlannerParams p) {
     const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z;
     const int row0 = p.off[i] + c * PLAN_CHUNK_ROWS, row1 = min(row0 + PLAN_CHUNK_ROWS, p.off[i + 1]);
-    const long long slot = ((long long)i * p.BH + bh) * p.L;      // row index base of slot i in the cache
+    const int ls = p.group_mode ? 0 : i;                          // slot of the local state
+    const long long slot = ((long long)ls * p.BH + bh) * p.L;     // row index base of that slot in the cache
     const long long snap = (long long)bh * p.L;                   // row index base in the snapshot
     const StateT *o = static_cast<const StateT *>(p.o_state), *so = static_cast<const StateT *>(p.snap_o);
     float diff = 0.f, base = 0.f;
@@ -88,7 +89,10 @@ __global__ void __launch_bounds__(1024) planner_decide_kernel(PlannerParams p) {
     __shared__ double tot[2];
     __shared__ double edge[2];
     __shared__ int anchor_s;
-    const int P = p.P, g = p.group_size, ng = (P + g - 1) / g, nunits = P * ng;
+    // pair mode: unit (i, k) = the k-th group of g adjacent slots without the local one; grouped cache: unit
+    // (i, s) = slot s != 0, one state with one weight and one scale ratio
+    const int P = p.P, S = p.S, g = p.group_mode ? 1 : p.group_size;
+    const int ng = p.group_mode ? S : (P + g - 1) / g, nunits = P * ng;
     const int e = threadIdx.x;
     PlannerState *st = p.state;
     if (e < P) {
@@ -116,9 +120,13 @@ __global__ void __launch_bounds__(1024) planner_decide_kernel(PlannerParams p) {
     double ase = 0.0;
     bool valid = false;
     if (e < nunits) {
-        const int lo = uk * g, hi = min(P, (uk + 1) * g);
-        for (int j = lo; j < hi; ++j)
-            if (j != ui) { ase += st->w[ui * P + j] * st->alpha[ui * P + j] * delta_s[ui]; valid = true; }
+        if (p.group_mode) {
+            if (uk != 0 && (p.nonempty[ui] >> uk & 1u)) { ase = st->w[e] * st->alpha[e] * delta_s[ui]; valid = true; }
+        } else {
+            const int lo = uk * g, hi = min(P, (uk + 1) * g);
+            for (int j = lo; j < hi; ++j)
+                if (j != ui) { ase += st->w[ui * P + j] * st->alpha[ui * P + j] * delta_s[ui]; valid = true; }
+        }
     }
     __syncthreads();
     if (e < nunits) { ase_s[e] = ase; valid_s[e] = valid ? 1 : 0; }
@@ -148,9 +156,11 @@ __global__ void __launch_bounds__(1024) planner_decide_kernel(PlannerParams p) {
         __syncthreads();
         if (e == 0) st->eps = (r == 0) ? 0.0 : (r == n_valid ? edge[0] : 0.5 * (edge[0] + edge[1]));
     }
-    if (e < P * P) {
-        const int i = e / P, j = e - i * P;
-        p.mask[e] = (is_anchor || i == j || ase_s[i * ng + j / g] > eps) ? 1 : 0;
+    if (e < P * S) {
+        const int i = e / S, j = e - i * S;
+        const bool local = p.group_mode ? (j == 0) : (i == j);
+        const int unit = p.group_mode ? e : i * ng + j / g;
+        p.mask[e] = (is_anchor || local || (valid_s[unit] && ase_s[unit] > eps)) ? 1 : 0;
     }
     if (e < nunits && p.ase_out) p.ase_out[e] = valid ? ase : nan("");
     if (e == 0) {
@@ -159,11 +169,15 @@ __global__ void __launch_bounds__(1024) planner_decide_kernel(PlannerParams p) {
     }
 }
 
-// grid (chunks, P (query partition i), BH * P (slot j)): sum of squares of the state rows; anchor steps only
+// grid (chunks, P (query partition i), BH * S (slot j)): sum of squares of the state rows; anchor steps only
 template <typename StateT>
 __global__ void __launch_bounds__(PL_THREADS) planner_norm_kernel(PlannerParams p) {
-    if (!p.state->is_anchor) return;
-    const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z / p.P, j = blockIdx.z - bh * p.P;
+    if (!p.force && !p.state->is_anchor) return;
+    const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z / p.S, j = blockIdx.z - bh * p.S;
+    if (!(p.nonempty[i] >> j & 1u)) {   // no such slot for this query partition
+        if (threadIdx.x == 0) p.norm_partials[(((long long)bh * p.P + i) * p.chunks + c) * p.S + j] = 0.f;
+        return;
+    }
     const int row0 = p.off[i] + c * PLAN_CHUNK_ROWS, row1 = min(row0 + PLAN_CHUNK_ROWS, p.off[i + 1]);
     const long long slot = ((long long)j * p.BH + bh) * p.L;
     const StateT *o = static_cast<const StateT *>(p.o_state);
@@ -179,21 +193,21 @@ __global__ void __launch_bounds__(PL_THREADS) planner_norm_kernel(PlannerParams 
         sq += a * a;
     }
     block_sum2(sq, unused);
-    if (threadIdx.x == 0) p.norm_partials[(((long long)bh * p.P + i) * p.chunks + c) * p.P + j] = sq;
+    if (threadIdx.x == 0) p.norm_partials[(((long long)bh * p.P + i) * p.chunks + c) * p.S + j] = sq;
 }
 
 // one block: w (Eq. 8, mean over rows and heads) and alpha (Eq. 9) from the partial sums; anchor steps only
 __global__ void __launch_bounds__(1024) planner_commit_kernel(PlannerParams p) {
     PlannerState *st = p.state;
-    if (!st->is_anchor) return;
+    if (!p.force && !st->is_anchor) return;
     __shared__ double nsq[DT_MAX_P * DT_MAX_P];
-    const int P = p.P, e = threadIdx.x;
-    const int i = e / P, j = e - i * P;
-    if (e < P * P) {
+    const int P = p.P, S = p.S, e = threadIdx.x;
+    const int i = e / S, j = e - i * S;
+    if (e < P * S) {
         double w = 0.0, n = 0.0;
         for (int bh = 0; bh < p.BH; ++bh)
             for (int c = 0; c < p.chunks; ++c) {
-                const long long idx = (((long long)bh * P + i) * p.chunks + c) * P + j;
+                const long long idx = (((long long)bh * P + i) * p.chunks + c) * S + j;
                 w += (double)p.w_partials[idx];
                 n += (double)p.norm_partials[idx];
             }
@@ -201,8 +215,8 @@ __global__ void __launch_bounds__(1024) planner_commit_kernel(PlannerParams p) {
         nsq[e] = n;
     }
     __syncthreads();
-    if (e < P * P) st->alpha[e] = sqrt(nsq[e] / nsq[i * P + i]);
-    if (e == 0) st->have_anchor = 1;
+    if (e < P * S) st->alpha[e] = sqrt(nsq[e] / nsq[i * S + (p.group_mode ? 0 : i)]);
+    if (e == 0 && !p.force) st->have_anchor = 1;
 }
 
 // copies the local states (slot i, rows of partition i) into the snapshot; anchor steps only
@@ -212,7 +226,7 @@ __global__ void __launch_bounds__(PL_THREADS) planner_snapshot_kernel(PlannerPar
     const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z;
     const int row0 = p.off[i] + c * PLAN_CHUNK_ROWS, row1 = min(row0 + PLAN_CHUNK_ROWS, p.off[i + 1]);
     if (row1 <= row0) return;
-    const long long slot = ((long long)i * p.BH + bh) * p.L, snap = (long long)bh * p.L;
+    const long long slot = ((long long)(p.group_mode ? 0 : i) * p.BH + bh) * p.L, snap = (long long)bh * p.L;
     const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const StateT *>(p.o_state) + (slot + row0) * p.D);
     uint4 *dst = reinterpret_cast<uint4 *>(static_cast<StateT *>(p.snap_o_out) + (snap + row0) * p.D);
     const long long n16 = (long long)(row1 - row0) * p.D * (long long)sizeof(StateT) / 16;
@@ -250,7 +264,7 @@ cudaError_t launch_planner_step(const PlannerParams &p, int state_dtype, cudaStr
 }
 
 cudaError_t launch_planner_commit(const PlannerParams &p, int state_dtype, cudaStream_t stream) {
-    dim3 grid_n((unsigned)p.chunks, (unsigned)p.P, (unsigned)(p.BH * p.P));
+    dim3 grid_n((unsigned)p.chunks, (unsigned)p.P, (unsigned)(p.BH * p.S));
     dim3 grid_s((unsigned)p.chunks, (unsigned)p.P, (unsigned)p.BH);
     if (state_dtype == DT_STATE_FP32) planner_norm_kernel<float><<<grid_n, PL_THREADS, 0, stream>>>(p);
     else planner_norm_kernel<__nv_bfloat16><<<grid_n, PL_THREADS, 0, stream>>>(p);
@@ -258,6 +272,7 @@ cudaError_t launch_planner_commit(const PlannerParams &p, int state_dtype, cudaS
     if (e != cudaSuccess) return e;
     planner_commit_kernel<<<1, 1024, 0, stream>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (p.force) return cudaSuccess;   // a refresh after a group compose keeps the anchor's snapshot
     if (state_dtype == DT_STATE_FP32) planner_snapshot_kernel<float><<<grid_s, PL_THREADS, 0, stream>>>(p);
     else planner_snapshot_kernel<__nv_bfloat16><<<grid_s, PL_THREADS, 0, stream>>>(p);
     return cudaGetLastError();

@@ -242,3 +242,95 @@ def test_memory_budget_triggers_group_compose():
     run.ses.compose()
     torch.cuda.synchronize()
     run.check_states("fit to 2 slots")
+
+
+def test_algorithm1_planner_on_a_grouped_cache_with_a_compose_between_anchors():
+    """Algorithm 1 per slot on the device (local attention -> plan -> remaining slots -> merge -> commit) against
+    the oracle rule applied to the GPU's own w, alpha and local drift; after step 3 the cache is composed g 2 -> 4
+    (Eq. 15) and planning continues on the coarser slots with w and alpha taken again from the composed cache."""
+    wl = inputs.Workload("alg1g", 1, 2, 64, (4, 16, 16), 0, 8, 7, 0.05)
+    P, R, eps_local = 8, 0.5, 0.5
+    run = GroupRun(wl, 2, seed=21)
+    dev, ctx, off = run.dev, run.ctx, run.off
+    snap_o = torch.zeros((wl.B, wl.H, wl.L, wl.D), dtype=torch.float32, device=dev)
+    snap_l = torch.zeros((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    ctx.dt_planner_init(snap_o, snap_l, group_size=1, eps_initial=0.0, eps_local=eps_local, cache_ratio=R)
+    with pytest.raises(binding.DitangoError):
+        ctx.dt_planner_init(snap_o, snap_l, group_size=2)
+    flag = torch.zeros(1, dtype=torch.int32, device=dev)
+    drel = torch.zeros(1, dtype=torch.float64, device=dev)
+    part = np.searchsorted(off, np.arange(wl.L), side="right") - 1
+    eps, have_anchor = 0.0, False
+    anchors = selective = 0
+    for t in range(wl.steps):
+        S = run.S
+        mem = run.ses.members
+        mask = torch.zeros(P * S, dtype=torch.uint8, device=dev)
+        ase = torch.zeros(P * S, dtype=torch.float64, device=dev)
+        q, k, v = run.gen.next()
+        ctx.dt_attn_local(q, k, v, t)
+        ctx.dt_planner_step(mask, flag, ase, drel)
+        torch.cuda.synchronize()
+        w_g, alpha_g, eps_dev, have_g = ctx.dt_planner_get()
+        assert have_g == have_anchor and w_g.shape == (P, S)
+        o_c = ctx.o_state[0].double().cpu().numpy(); l_c = ctx.lse_state[0].double().cpu().numpy()   # slot 0: local states
+        so = snap_o.double().cpu().numpy(); sl = snap_l.double().cpu().numpy()
+        drift = np.zeros(P); base = np.zeros(P)
+        for i in range(P):
+            rows = part == i
+            drift[i] = ((o_c[:, :, rows] - so[:, :, rows]) ** 2).sum() + ((l_c[:, :, rows] - sl[:, :, rows]) ** 2).sum()
+            base[i] = (so[:, :, rows] ** 2).sum() + (sl[:, :, rows] ** 2).sum()
+        ref = orc.planner_step_slots(w_g, alpha_g, mem, drift, base, eps, eps_local, R, have_anchor)
+        got_mask = mask.cpu().numpy().reshape(P, S)
+        assert bool(flag.item()) == ref["is_anchor"], (t, ref["delta_rel"])
+        assert (got_mask == ref["mask"]).all(), t
+        if have_anchor:
+            units = ~np.isnan(ref["ase"])
+            got_ase = ase.cpu().numpy().reshape(P, S)
+            np.testing.assert_allclose(got_ase[units], ref["ase"][units], rtol=1e-4)
+            assert np.isnan(got_ase[~units]).all()
+            assert drel.item() == pytest.approx(ref["delta_rel"], rel=1e-4)
+            if not ref["is_anchor"]:
+                assert (np.abs(ref["ase"][units] - eps) / max(eps, 1e-300)).min() > 1e-5
+        assert eps_dev == pytest.approx(ref["eps"], rel=1e-4)
+        eps = eps_dev
+        rest = got_mask.copy(); rest[:, 0] = 0
+        ctx.dt_attn_states(q, k, v, torch.from_numpy(rest.reshape(-1).copy()).to(dev), t)
+        ctx.dt_state_merge(run.out, run.lse)
+        ctx.dt_planner_commit()
+        torch.cuda.synchronize()
+        ctx.dt_poll()
+        run.ses.step(*(inputs.bf16_bits(x) for x in (q, k, v)), got_mask, t)
+        run.check_merged(f"alg1 grouped step {t}")
+        assert (ctx.dt_get_tc() == run.ses.tc).all()
+
+        def check_stats(what):
+            """w (Eq. 8 / Eq. 12) and alpha (Eq. 9) against the oracle's states."""
+            w_g, alpha_g, _, _ = ctx.dt_planner_get()
+            S = run.ses.S
+            lse_ref = np.empty((S, wl.B, wl.H, wl.L)); nsq = np.zeros((P, S))
+            for (b, h), _rows in run.rows.items():
+                lse_ref[:, b, h, :] = run.ses.lse[(b, h)].T
+                for i in range(P):
+                    sel = part == i
+                    for s in range(S):
+                        if run.ses.members[i][s]:
+                            nsq[i, s] += orc.state_norm_sq(run.ses.o[(b, h)][sel, s, :], run.ses.lse[(b, h)][sel, s])
+            np.testing.assert_allclose(w_g, orc.slot_contribution(lse_ref, off, run.ses.members), rtol=2e-3, atol=1e-6, err_msg=what)
+            np.testing.assert_allclose(alpha_g, np.sqrt(nsq / nsq[:, :1]), rtol=2e-3, err_msg=what)
+
+        if ref["is_anchor"]:
+            anchors += 1
+            have_anchor = True
+            check_stats(f"anchor at step {t}")
+            assert torch.equal(snap_l, ctx.lse_state[0])
+        else:
+            selective += 1
+            assert P <= got_mask.sum() < P * S
+        if t == 3:
+            ctx.dt_group_compose()
+            run.ses.compose()
+            torch.cuda.synchronize()
+            assert run.S == 3
+            check_stats("after compose")
+    assert anchors >= 2 and selective >= 2

@@ -142,3 +142,34 @@ def test_slot_plan_agrees_with_the_group_rule_on_pairs(P, g):
     # strict inequality: a slot exactly at eps is reused
     ms, _ = orc.slot_plan(Ws, mem, g, eps=float(Ws[0, 1]))
     assert ms[0, 1] == 0
+
+
+def test_planner_rule_on_slots_reduces_to_the_pair_rule_when_every_group_is_one_partition():
+    """Algorithm 1 per slot: with groups of one partition the units, their ASE (Eq. 7, 10, 12), the anchor test
+    (Eq. 14), the threshold (Eq. 13) and the eps update must be those of the pair-level rule."""
+    rng = np.random.default_rng(11)
+    P = 5
+    mem = orc.group_slots(P, 1)                      # slot 0 local, slot 1 + j = [j] (empty for j == i)
+    S = P + 1
+    W = rng.random((P, P)); W /= W.sum(axis=1, keepdims=True)
+    alpha = 0.5 + rng.random((P, P)); alpha[np.arange(P), np.arange(P)] = 1.0
+    Ws = np.zeros((P, S)); As = np.zeros((P, S))
+    for i in range(P):
+        Ws[i, 0], As[i, 0] = W[i, i], 1.0
+        for j in range(P):
+            if j != i:
+                Ws[i, 1 + j], As[i, 1 + j] = W[i, j], alpha[i, j]
+    base = 1.0 + rng.random(P)
+    for scale, eps, have in ((1e-3, 0.02, True), (0.2, 0.02, True), (0.05, 0.004, True), (0.05, 0.02, False),
+                             (0.0, 0.0, True), (3.0, 0.02, True)):
+        drift = scale * rng.random(P)
+        a = orc.planner_step(W, alpha, drift, base, 1, eps, 0.4, 0.6, have)
+        b = orc.planner_step_slots(Ws, As, mem, drift, base, eps, 0.4, 0.6, have)
+        assert a["is_anchor"] == b["is_anchor"] and a["eps"] == pytest.approx(b["eps"], rel=1e-15)
+        assert a["delta_rel"] == b["delta_rel"]
+        for i in range(P):
+            assert b["mask"][i, 0] == 1
+            for j in range(P):
+                if j != i:
+                    assert a["mask"][i, j] == b["mask"][i, 1 + j]
+                    assert a["ase"][i, j] == pytest.approx(b["ase"][i, 1 + j], rel=1e-15)
