@@ -279,6 +279,13 @@ def run_cuda(args, wl):
         if timers is not None:
             e = [ev() for _ in range(4)]
             e[0].record(stream)
+        if args.fused:       # one pass: COMPUTE slots + composed reuse state -> output; no cache round trip, no re-plan
+            ctx.dt_attn_fused(q, k, v, masks[cur], comp_o, comp_l, out, lse)
+            if timers is not None:
+                for i in (1, 2, 3):
+                    e[i].record(stream)
+                timers.append(e)
+            return cur
         ctx.dt_attn_states(q, k, v, masks[cur], t)
         if timers is not None:
             e[1].record(stream)
@@ -301,7 +308,7 @@ def run_cuda(args, wl):
     ctx.dt_plan(masks[0], target_fraction=frac, w_dev=W)
     comp_o = comp_l = None
     compose_ms = None
-    if args.composed:
+    if args.composed or args.fused:
         comp_o = torch.empty((wl.B, wl.H, wl.L, wl.D), dtype=ctx.o_state.dtype, device=dev)
         comp_l = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
         c0, c1 = ev(), ev()
@@ -370,6 +377,17 @@ def run_cuda(args, wl):
             full_ms.append((a.elapsed_time(b), b.elapsed_time(c)))
     full_attn_ms = float(np.mean([x[0] for x in full_ms]))
     full_step_ms = float(np.mean([x[0] + x[1] for x in full_ms]))
+    dense_ms = []
+    for i in range(3 + 1):          # plain full attention: every slot in one pass, nothing cached, nothing merged
+        a, b = ev(), ev()
+        q, k, v = steps_in[i % wl.steps]
+        a.record(stream)
+        ctx.dt_attn_fused(q, k, v, ones, None, None, out, lse)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i > 0:
+            dense_ms.append(a.elapsed_time(b))
+    dense_ms = float(np.mean(dense_ms))
 
     # ---- end to end through the C ABI with host buffers (pinned): H2D of q, k, v, mask; D2H of out, lse
     e2e = None
@@ -411,7 +429,8 @@ def run_cuda(args, wl):
                    "computed_pairs": n_comp, "computed_pair_fraction": n_comp / (wl.P * wl.P),
                    "group_size": g, "cache_slots": S, "computed_slots": n_slots_comp, "state_dtype": args.state_dtype,
                    "cache_gb": S * wl.B * wl.H * wl.L * (wl.D * sbytes + 4) / 1e9,
-                   "step": ("dt_attn_states + dt_state_merge_planned + dt_plan" if args.composed
+                   "step": ("dt_attn_fused (COMPUTE slots in one pass + composed reuse state in the epilogue)" if args.fused
+                            else "dt_attn_states + dt_state_merge_planned + dt_plan" if args.composed
                             else "dt_attn_states + dt_state_merge + dt_plan"), "multi_gpu": "independent replicas",
                    "l2": "inputs (%.1f GB) and state cache larger than L2; no flush" %
                          ((3 * wl.L * wl.H * wl.D * 2) / 1e9)},
@@ -438,7 +457,9 @@ def run_cuda(args, wl):
         "vs_all_compute": {"all_compute_attn_ms": full_attn_ms, "all_compute_step_ms": full_step_ms,
                            "all_compute_tflops": full_flops(wl) / 1e12 / (full_attn_ms / 1e3),
                            "all_compute_frac_of_peak": full_flops(wl) / 1e12 / (full_attn_ms / 1e3) / peak,
-                           "step_time_ratio": ms_per_step / full_step_ms},
+                           "step_time_ratio": ms_per_step / full_step_ms,
+                           "full_attention_one_pass_ms": dense_ms,
+                           "full_attention_one_pass_tflops": full_flops(wl) / 1e12 / (dense_ms / 1e3)},
     }
     print(json.dumps(line))
 
@@ -457,6 +478,9 @@ def main():
     ap.add_argument("--composed", action="store_true",
                     help="compose the plan's REUSE states once after the anchor step and merge COMPUTE states + that "
                          "composed state in the selective steps (the plan then stays fixed between anchors)")
+    ap.add_argument("--fused", action="store_true",
+                    help="between anchors: dt_attn_fused per step (all COMPUTE slots in one pass, composed with the plan's "
+                         "composed reuse state in the epilogue; no state-cache round trip, the plan stays fixed)")
     ap.add_argument("--group-size", type=int, default=1,
                     help="g >= 2: grouped state cache (ceil(P/g) + 1 slots per row; group states computed in one pass)")
     ap.add_argument("--no-e2e", action="store_true")

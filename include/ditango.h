@@ -194,6 +194,24 @@ dt_status dt_planner_commit(dt_ctx *ctx, void *stream);
  * pointer may be NULL. */
 dt_status dt_planner_get(dt_ctx *ctx, double *w_host, double *alpha_host, double *eps_host, int32_t *have_anchor_host);
 
+/* Attention output of a selective step in one pass, without the round trip through the cache: for every query
+ * row the state over the keys of ALL COMPUTE slots of its partition is accumulated in one flash pass (adjacent
+ * key ranges are joined), composed in the kernel's epilogue (Eq. 2) with the composed reuse state of the same
+ * mask (dt_compose_reuse), and written as the attention output.  For the steps between two anchors of a plan
+ * that holds: there the COMPUTE states are recomputed every step and never reused, so caching them would only
+ * cost a write here and a read in the merge.
+ *   mask_dev                    device, uint8 [P*S] (pair mode: [P*P]); the local slot must be COMPUTE
+ *   comp_o_dev / comp_lse_dev   device, composed reuse state [B][H][L][D] (cache dtype) / [B][H][L] from
+ *                               dt_compose_reuse with the same mask; both NULL: the COMPUTE slots alone
+ *                               (with an all-ones mask: plain full attention)
+ *   out_dev, out_strides_blhd, lse_out_dev   as for dt_state_merge
+ * The state cache, t_c and the device status word are not touched: cached states of COMPUTE slots keep the
+ * values of the step that last went through dt_attn_states. */
+dt_status dt_attn_fused(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
+                        const int64_t strides_blhd[4], const uint8_t *mask_dev, const void *comp_o_dev,
+                        const float *comp_lse_dev, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev,
+                        void *stream);
+
 /* Grouped state cache (Section 4.2.1, Section 4.2.2; Dynamic Group State Compose, Eq. 15).  With
  * dt_config.group_size = g >= 2 the calls above work on slots instead of KV partitions:
  *   dt_attn_states / dt_attn_local   mask is uint8 [P*S]; a COMPUTE slot is evaluated in one pass over all keys of

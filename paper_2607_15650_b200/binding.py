@@ -23,7 +23,7 @@ EXPORTS = [
     "dt_compose_reuse", "dt_state_merge_planned", "dt_plan", "dt_plan_grouped", "dt_planner_init", "dt_planner_step", "dt_planner_commit", "dt_planner_get",
     "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
     "dt_launch_count", "dt_selftest_wait_timeout", "dt_poll", "dt_status_str", "dt_last_error",
-    "dt_num_slots", "dt_slot_ranges", "dt_group_compose", "dt_group_fit", "dt_group_reset",
+    "dt_attn_fused", "dt_num_slots", "dt_slot_ranges", "dt_group_compose", "dt_group_fit", "dt_group_reset",
 ]
 
 
@@ -84,6 +84,7 @@ def lib():
         "dt_launch_count": (C.c_int, [vp, C.POINTER(C.c_uint64)]),
         "dt_selftest_wait_timeout": (C.c_int, [vp, C.c_uint32, vp]),
         "dt_poll": (C.c_int, [vp]),
+        "dt_attn_fused": (C.c_int, [vp, vp, vp, vp, i64p, u8p, vp, f32p, vp, i64p, f32p, vp]),
         "dt_num_slots": (C.c_int, [vp, i32p, i32p]),
         "dt_slot_ranges": (C.c_int, [vp, i32p]),
         "dt_group_compose": (C.c_int, [vp, vp]),
@@ -204,6 +205,18 @@ class Context:
         assert q.stride() == k.stride() == v.stride() and q.shape == k.shape == v.shape
         self._check(lib().dt_attn_local(self._h, C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()),
                                         C.c_void_p(v.data_ptr()), _strides4(q), int(step), _stream_ptr(stream)))
+
+    def dt_attn_fused(self, q, k, v, mask_dev, comp_o, comp_lse, out, lse_out=None, stream=None):
+        assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and q.is_cuda
+        assert q.stride() == k.stride() == v.stride() and q.shape == k.shape == v.shape
+        assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()
+        assert out.dtype == torch.bfloat16 and out.is_cuda
+        opt = lambda t: C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p()
+        if comp_o is not None and comp_lse is not None:
+            assert comp_o.is_contiguous() and comp_lse.is_contiguous() and comp_o.dtype == self.o_state.dtype
+        self._check(lib().dt_attn_fused(self._h, C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()), C.c_void_p(v.data_ptr()),
+                                        _strides4(q), C.c_void_p(mask_dev.data_ptr()), opt(comp_o), opt(comp_lse),
+                                        C.c_void_p(out.data_ptr()), _strides4(out), opt(lse_out), _stream_ptr(stream)))
 
     def dt_state_merge(self, out, lse_out=None, stream=None):
         assert out.dtype == torch.bfloat16 and out.is_cuda

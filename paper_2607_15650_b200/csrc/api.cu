@@ -190,6 +190,9 @@ dt_status dt_create(dt_ctx **ctx_out, const dt_config *cfg) {
     ok = ok && cudaMalloc(&ctx->nonempty_dev, P * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->tc_dev, P * S * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->worklist_dev, (1 + P * S) * sizeof(int32_t)) == cudaSuccess;
+    ctx->max_tiles = cfg->L / dt::ATTN_TILE + 2 * DT_MAX_P + 4;   // one pass over all keys + one ragged tile per run
+    ok = ok && cudaMalloc(&ctx->tile_tab_dev, (size_t)P * ctx->max_tiles * sizeof(int2)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->tile_cnt_dev, P * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->status_dev, sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->sel_bits_dev, 2 * DT_MAX_P * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->plan_partials_dev, (size_t)BH * P * ctx->plan_chunks * S * sizeof(float)) == cudaSuccess;
@@ -216,6 +219,8 @@ dt_status dt_destroy(dt_ctx *ctx) {
     cudaFree(ctx->nonempty_dev);
     cudaFree(ctx->tc_dev);
     cudaFree(ctx->worklist_dev);
+    cudaFree(ctx->tile_tab_dev);
+    cudaFree(ctx->tile_cnt_dev);
     cudaFree(ctx->status_dev);
     cudaFree(ctx->plan_partials_dev);
     cudaFree(ctx->sel_bits_dev);
@@ -261,7 +266,7 @@ dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const v
     cudaError_t e = dt::launch_worklist(mask_dev, ctx->tc_dev, ctx->worklist_dev, ctx->status_dev, ctx->slot_tab_dev, c.P,
                                         ctx->S, ctx->group_size0 > 1 ? 1 : 0, step, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "work-list launch");
-    dt::AttnParams p;
+    dt::AttnParams p = {};
     p.off = ctx->off_dev;
     p.slot_tab = ctx->slot_tab_dev;
     p.worklist = ctx->worklist_dev;
@@ -289,6 +294,52 @@ dt_status dt_attn_local(dt_ctx *ctx, const void *q_dev, const void *k_dev, const
                         const int64_t strides_blhd[4], int32_t step, void *stream) {
     if (!ctx) return DT_ERR_INVALID_ARG;
     return attn_launch(ctx, q_dev, k_dev, v_dev, strides_blhd, nullptr, step, stream);
+}
+
+dt_status dt_attn_fused(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev,
+                        const int64_t strides_blhd[4], const uint8_t *mask_dev, const void *comp_o_dev,
+                        const float *comp_lse_dev, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev,
+                        void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!q_dev || !k_dev || !v_dev || !mask_dev || !out_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null pointer");
+    if ((comp_o_dev == nullptr) != (comp_lse_dev == nullptr)) return fail(ctx, DT_ERR_INVALID_ARG, "composed state needs both OUT and LSE");
+    if (comp_o_dev && (reinterpret_cast<uintptr_t>(comp_o_dev) & 15u) != 0) return fail(ctx, DT_ERR_INVALID_ARG, "composed state must be 16-byte aligned");
+    const char *why;
+    for (const void *t : {q_dev, k_dev, v_dev}) {
+        dt_status s = check_strides(strides_blhd, t, &why);
+        if (s != DT_OK) return fail(ctx, s, why);
+    }
+    dt_status s = check_strides(out_strides_blhd, out_dev, &why);
+    if (s != DT_OK) return fail(ctx, s, why);
+    CUtensorMap tq, tk, tv;
+    if ((s = encode_qkv_map(ctx, &tq, q_dev, strides_blhd)) != DT_OK) return s;
+    if ((s = encode_qkv_map(ctx, &tk, k_dev, strides_blhd)) != DT_OK) return s;
+    if ((s = encode_qkv_map(ctx, &tv, v_dev, strides_blhd)) != DT_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dt_config &c = ctx->cfg;
+    cudaError_t e = dt::launch_fused_tiles(mask_dev, ctx->slot_tab_dev, c.P, ctx->S, ctx->max_tiles, ctx->tile_tab_dev,
+                                           ctx->tile_cnt_dev, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "tile-table launch");
+    dt::AttnParams p = {};
+    p.off = ctx->off_dev;
+    p.slot_tab = ctx->slot_tab_dev;
+    p.worklist = ctx->worklist_dev;
+    p.status = ctx->status_dev;
+    p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P; p.S = ctx->S;
+    p.qblocks_max = ctx->qblocks_max;
+    p.scale_log2 = c.softmax_scale * 1.44269504088896340736f;
+    p.tile_tab = ctx->tile_tab_dev;
+    p.tile_cnt = ctx->tile_cnt_dev;
+    p.max_tiles = ctx->max_tiles;
+    p.comp_o = comp_o_dev;
+    p.comp_lse = comp_lse_dev;
+    p.out = out_dev;
+    p.lse_out = lse_out_dev;
+    p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
+    e = dt::launch_attn_fused(tq, tk, tv, p, c.D, c.state_dtype, ctx->num_sms, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fused attention launch");
+    ctx->launches += 2;
+    return DT_OK;
 }
 
 dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev,

@@ -95,24 +95,27 @@ struct WorkItem {
     int r1, n1;     // first key range of the slot
     int r2, n2;     // second key range (n2 == 0: none)
     int tiles1;     // ceil(n1 / 128)
-    int tiles;      // tiles1 + ceil(n2 / 128)
-    // first key of K/V tile t, and how many of its 128 keys belong to the slot (may exceed 128)
-    __device__ __forceinline__ int tile_row(int t) const {
-        return t < tiles1 ? r1 + t * ATTN_TILE : r2 + (t - tiles1) * ATTN_TILE;
-    }
-    __device__ __forceinline__ int tile_valid(int t) const {
-        return t < tiles1 ? n1 - t * ATTN_TILE : n2 - (t - tiles1) * ATTN_TILE;
+    int tiles;      // tiles1 + ceil(n2 / 128); fused mode: tiles of the partition's tile table
+    const int2 *tab; // fused mode: (first key, keys that count) per tile
+    // first key of K/V tile t, and how many of its 128 keys count (may exceed 128)
+    template <bool FUSED>
+    __device__ __forceinline__ int2 tile(int t) const {
+        if constexpr (FUSED) return __ldg(tab + t);
+        return t < tiles1 ? make_int2(r1 + t * ATTN_TILE, n1 - t * ATTN_TILE)
+                          : make_int2(r2 + (t - tiles1) * ATTN_TILE, n2 - (t - tiles1) * ATTN_TILE);
     }
 };
 
-// Work index -> item.  Returns false when the block lies beyond the end of partition i.
+// Work index -> item.  Returns false when the block lies beyond the end of partition i (or has no keys).
+// npairs = work items per (b, h) and query block: COMPUTE states of the work list, or P in fused mode.
+template <bool FUSED>
 __device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, long long w, WorkItem &it) {
     const long long per_bh = (long long)npairs * p.qblocks_max;
     it.bh = (int)(w / per_bh);
     const int rem = (int)(w - (long long)it.bh * per_bh);
     const int pair = rem / p.qblocks_max;
     const int qb = rem - pair * p.qblocks_max;
-    const int code = p.worklist[1 + pair];
+    const int code = FUSED ? pair : p.worklist[1 + pair];
     it.i = code & 0xFF;
     it.slot = code >> 8;
     it.b = it.bh / p.H;
@@ -120,6 +123,13 @@ __device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, lon
     const int qs = p.off[it.i], qe = p.off[it.i + 1];
     it.q_row0 = qs + qb * (ATTN_NQ * ATTN_TILE);
     it.n_q = min(qe - it.q_row0, ATTN_NQ * ATTN_TILE);
+    if constexpr (FUSED) {
+        it.tab = p.tile_tab + (long long)it.i * p.max_tiles;
+        it.tiles = p.tile_cnt[it.i];
+        it.r1 = it.n1 = it.r2 = it.n2 = it.tiles1 = 0;
+        return it.n_q > 0 && it.tiles > 0;
+    }
+    it.tab = nullptr;
     const int4 rg = *reinterpret_cast<const int4 *>(p.slot_tab + it.i * p.S + it.slot);
     it.r1 = rg.x; it.n1 = rg.y; it.r2 = rg.z; it.n2 = rg.w;
     it.tiles1 = (it.n1 + ATTN_TILE - 1) / ATTN_TILE;
@@ -152,7 +162,28 @@ __device__ __forceinline__ void store_state_chunk<__nv_bfloat16>(__nv_bfloat16 *
     }
 }
 
-template <int D, typename StateT>
+// 32 consecutive elements of a cached state row as fp32
+__device__ __forceinline__ void load_state_chunk(const float *src, float (&v)[32]) {
+#pragma unroll
+    for (int c = 0; c < 32; c += 4) {
+        const float4 x = __ldcs(reinterpret_cast<const float4 *>(src + c));
+        v[c] = x.x; v[c + 1] = x.y; v[c + 2] = x.z; v[c + 3] = x.w;
+    }
+}
+__device__ __forceinline__ void load_state_chunk(const __nv_bfloat16 *src, float (&v)[32]) {
+#pragma unroll
+    for (int c = 0; c < 32; c += 8) {
+        const uint4 x = __ldcs(reinterpret_cast<const uint4 *>(src + c));
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            v[c + 2 * e] = __uint_as_float(w[e] << 16);
+            v[c + 2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+        }
+    }
+}
+
+template <int D, typename StateT, bool FUSED>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                    const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
@@ -204,7 +235,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    const int npairs = p.worklist[0];
+    const int npairs = FUSED ? p.P : p.worklist[0];
     const long long total_work = (long long)npairs * p.qblocks_max * p.B * p.H;
 
     if (warp >= TMA_WARP) {
@@ -220,7 +251,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             bool ok = true;
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
-                if (!decode_work(p, npairs, w, it)) continue;
+                if (!decode_work<FUSED>(p, npairs, w, it)) continue;
                 ok = mbar_wait_bounded(bars.q_empty, q_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
                 if (!ok) break;
                 mbar_arrive_expect_tx(bars.q_full, C::Q_BYTES);
@@ -232,6 +263,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                                     it.q_row0 + q * ATTN_TILE, it.b);
                 q_phase ^= 1u;
                 for (int t = 0; t < it.tiles && ok; ++t) {
+                    const int key0 = it.template tile<FUSED>(t).x;
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
                         const uint32_t st = ring.st, ph = ring.ph;
@@ -241,7 +273,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 #pragma unroll
                         for (int hf = 0; hf < C::NHALF; ++hf)
                             tma_load_4d(kv_smem + st * C::TILE_BYTES + hf * C::HALF_BYTES, kv == 0 ? &tmap_k : &tmap_v,
-                                        bars.kv_full + 8 * st, hf * 64, it.h, it.tile_row(t), it.b);
+                                        bars.kv_full + 8 * st, hf * 64, it.h, key0, it.b);
                         ring.advance();
                     }
                 }
@@ -290,7 +322,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
-                if (!decode_work(p, npairs, w, it)) continue;
+                if (!decode_work<FUSED>(p, npairs, w, it)) continue;
                 ok = mbar_wait_bounded(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
                 if (!ok) break;
                 q_phase ^= 1u;
@@ -360,7 +392,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             bool ok = true;
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
-                if (!decode_work(p, npairs, w, it)) continue;
+                if (!decode_work<FUSED>(p, npairs, w, it)) continue;
                 ring.advance();   // K_0 of the item: the MMA thread waits for that one itself
                 for (int t = 0; t < it.tiles && ok; ++t) {
                     ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
@@ -396,9 +428,10 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 
         for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             WorkItem it;
-            if (!decode_work(p, npairs, w, it)) continue;
+            if (!decode_work<FUSED>(p, npairs, w, it)) continue;
             float m_used = -INFINITY, l_sum = 0.f;
             for (int t = 0; t < it.tiles; ++t) {
+                const int valid = it.template tile<FUSED>(t).y;   // keys of this tile that count (issued before the wait)
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.s_full + 8 * q, s_phase, abort_ptr, WAIT_LIMIT_NS));
                 if (!ok) break;
                 s_phase ^= 1u;
@@ -409,7 +442,6 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 tmem_ld_x32(s_tmem + 64, s[2]);
                 tmem_ld_x32(s_tmem + 96, s[3]);
                 tmem_wait_ld();
-                const int valid = it.tile_valid(t);   // keys of this tile that belong to the slot
                 if (valid < ATTN_TILE) {
 #pragma unroll
                     for (int c = 0; c < 128; ++c)
@@ -492,19 +524,67 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             const int row_in_block = q * ATTN_TILE + row_in_tile;
             const bool row_valid = row_in_block < it.n_q;
             const float inv_l = 1.0f / l_sum;
-            const long long srow = ((long long)it.slot * p.B * p.H + it.bh) * p.L + it.q_row0 + row_in_block;
-#pragma unroll
-            for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t o[32];
-                tmem_ld_x32(o_tmem + c0, o);
-                tmem_wait_ld();
-                if (c0 + 32 >= D) {  // O[q] fully read: the next item's first PV may overwrite it
-                    tc_fence_before();
-                    mbar_arrive(bars.o_free + 8 * q);
+            const float lse_fresh = 0.69314718055994530942f * (m_used + log2f(l_sum));
+            if constexpr (FUSED) {
+                // fresh state (+) composed reuse state (Eq. 2), straight to the attention output
+                const long long crow = (long long)it.bh * p.L + it.q_row0 + row_in_block;
+                float w_f = inv_l, w_c = 0.f, lse_row = lse_fresh;
+                if (p.comp_o != nullptr && row_valid) {
+                    const float lc = __ldcs(p.comp_lse + crow);
+                    const float M = fmaxf(lse_fresh, lc);
+                    const float ef = __expf(lse_fresh - M), ec = __expf(lc - M);   // lc = -inf: weight 0
+                    const float z = ef + ec;
+                    w_f = inv_l * ef / z;
+                    w_c = ec / z;
+                    lse_row = M + __logf(z);
                 }
-                if (row_valid) store_state_chunk<StateT>(o_state + srow * D + c0, o, inv_l);
+                __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) + it.b * p.sb + (long long)(it.q_row0 + row_in_block) * p.sl +
+                                     it.h * p.sh;
+                const StateT *csrc = static_cast<const StateT *>(p.comp_o) + crow * D;
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t o[32];
+                    tmem_ld_x32(o_tmem + c0, o);
+                    tmem_wait_ld();
+                    if (c0 + 32 >= D) {  // O[q] fully read: the next item's first PV may overwrite it
+                        tc_fence_before();
+                        mbar_arrive(bars.o_free + 8 * q);
+                    }
+                    if (row_valid) {
+                        float cv[32];
+                        if (w_c != 0.f) {
+                            load_state_chunk(csrc + c0, cv);
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) cv[c] = 0.f;
+                        }
+#pragma unroll
+                        for (int c = 0; c < 32; c += 8) {
+                            uint4 v;
+                            v.x = pack_bf16x2(fmaf(w_f, __uint_as_float(o[c]), w_c * cv[c]), fmaf(w_f, __uint_as_float(o[c + 1]), w_c * cv[c + 1]));
+                            v.y = pack_bf16x2(fmaf(w_f, __uint_as_float(o[c + 2]), w_c * cv[c + 2]), fmaf(w_f, __uint_as_float(o[c + 3]), w_c * cv[c + 3]));
+                            v.z = pack_bf16x2(fmaf(w_f, __uint_as_float(o[c + 4]), w_c * cv[c + 4]), fmaf(w_f, __uint_as_float(o[c + 5]), w_c * cv[c + 5]));
+                            v.w = pack_bf16x2(fmaf(w_f, __uint_as_float(o[c + 6]), w_c * cv[c + 6]), fmaf(w_f, __uint_as_float(o[c + 7]), w_c * cv[c + 7]));
+                            __stcs(reinterpret_cast<uint4 *>(dst + c0 + c), v);
+                        }
+                    }
+                }
+                if (row_valid && p.lse_out != nullptr) p.lse_out[crow] = lse_row;
+            } else {
+                const long long srow = ((long long)it.slot * p.B * p.H + it.bh) * p.L + it.q_row0 + row_in_block;
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t o[32];
+                    tmem_ld_x32(o_tmem + c0, o);
+                    tmem_wait_ld();
+                    if (c0 + 32 >= D) {  // O[q] fully read: the next item's first PV may overwrite it
+                        tc_fence_before();
+                        mbar_arrive(bars.o_free + 8 * q);
+                    }
+                    if (row_valid) store_state_chunk<StateT>(o_state + srow * D + c0, o, inv_l);
+                }
+                if (row_valid) p.lse_state[srow] = lse_fresh;
             }
-            if (row_valid) p.lse_state[srow] = 0.69314718055994530942f * (m_used + log2f(l_sum));
         }
         if (!ok && lane == 0) {
             if (!*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
@@ -518,21 +598,58 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp == 0) tmem_dealloc(tmem_base, 512);
 }
 
-template <int D, typename StateT>
+template <int D, typename StateT, bool FUSED>
 cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const AttnParams &p,
                    int num_ctas, cudaStream_t stream) {
-    attn_states_kernel<D, StateT><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, p);
+    attn_states_kernel<D, StateT, FUSED><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, p);
     return cudaGetLastError();
+}
+
+template <int D, typename StateT, bool FUSED>
+cudaError_t configure_one() {
+    cudaFuncAttributes attr;
+    cudaError_t e = cudaFuncGetAttributes(&attr, attn_states_kernel<D, StateT, FUSED>);
+    if (e != cudaSuccess) return e;
+    if (attr.numRegs != LAUNCH_REGS) return cudaErrorInvalidConfiguration;   // the register hand-over would not balance
+    return cudaFuncSetAttribute(attn_states_kernel<D, StateT, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Cfg<D>::SMEM_BYTES);
 }
 
 template <int D, typename StateT>
 cudaError_t configure() {
-    cudaFuncAttributes attr;
-    cudaError_t e = cudaFuncGetAttributes(&attr, attn_states_kernel<D, StateT>);
-    if (e != cudaSuccess) return e;
-    if (attr.numRegs != LAUNCH_REGS) return cudaErrorInvalidConfiguration;   // the register hand-over would not balance
-    return cudaFuncSetAttribute(attn_states_kernel<D, StateT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                Cfg<D>::SMEM_BYTES);
+    cudaError_t e = configure_one<D, StateT, false>();
+    return e != cudaSuccess ? e : configure_one<D, StateT, true>();
+}
+
+// Fused mode: per query partition the K/V tiles of one pass over the keys of all its COMPUTE slots.  The slots'
+// key ranges are sorted and ranges that touch are joined, so only the last tile of a maximal run is ragged.
+__global__ void fused_tiles_kernel(const uint8_t *mask, const SlotRange *slot_tab, int P, int S, int max_tiles, int2 *tile_tab,
+                                   int32_t *tile_cnt) {
+    const int i = threadIdx.x;
+    if (i >= P) return;
+    int start[2 * DT_MAX_P + 2], len[2 * DT_MAX_P + 2];
+    int n = 0;
+    for (int s = 0; s < S; ++s) {
+        if (mask[i * S + s] == 0) continue;
+        const SlotRange r = slot_tab[i * S + s];
+        if (r.n1 > 0) { start[n] = r.r1; len[n] = r.n1; ++n; }
+        if (r.n2 > 0) { start[n] = r.r2; len[n] = r.n2; ++n; }
+    }
+    for (int a = 1; a < n; ++a) {   // insertion sort by first key
+        const int s0 = start[a], l0 = len[a];
+        int b = a - 1;
+        while (b >= 0 && start[b] > s0) { start[b + 1] = start[b]; len[b + 1] = len[b]; --b; }
+        start[b + 1] = s0; len[b + 1] = l0;
+    }
+    int2 *tab = tile_tab + (long long)i * max_tiles;
+    int cnt = 0;
+    for (int a = 0; a < n;) {
+        int s0 = start[a], l0 = len[a];
+        ++a;
+        while (a < n && start[a] == s0 + l0) { l0 += len[a]; ++a; }
+        for (int k = 0; k < l0 && cnt < max_tiles; k += ATTN_TILE) tab[cnt++] = make_int2(s0 + k, l0 - k);
+    }
+    tile_cnt[i] = cnt;
 }
 
 }  // namespace
@@ -548,11 +665,27 @@ cudaError_t attn_states_configure() {
 cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                                const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream) {
     if (state_dtype == DT_STATE_FP32) {
-        return D == 64 ? launch<64, float>(tq, tk, tv, p, num_ctas, stream)
-                       : launch<128, float>(tq, tk, tv, p, num_ctas, stream);
+        return D == 64 ? launch<64, float, false>(tq, tk, tv, p, num_ctas, stream)
+                       : launch<128, float, false>(tq, tk, tv, p, num_ctas, stream);
     }
-    return D == 64 ? launch<64, __nv_bfloat16>(tq, tk, tv, p, num_ctas, stream)
-                   : launch<128, __nv_bfloat16>(tq, tk, tv, p, num_ctas, stream);
+    return D == 64 ? launch<64, __nv_bfloat16, false>(tq, tk, tv, p, num_ctas, stream)
+                   : launch<128, __nv_bfloat16, false>(tq, tk, tv, p, num_ctas, stream);
+}
+
+cudaError_t launch_attn_fused(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
+                              const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream) {
+    if (state_dtype == DT_STATE_FP32) {
+        return D == 64 ? launch<64, float, true>(tq, tk, tv, p, num_ctas, stream)
+                       : launch<128, float, true>(tq, tk, tv, p, num_ctas, stream);
+    }
+    return D == 64 ? launch<64, __nv_bfloat16, true>(tq, tk, tv, p, num_ctas, stream)
+                   : launch<128, __nv_bfloat16, true>(tq, tk, tv, p, num_ctas, stream);
+}
+
+cudaError_t launch_fused_tiles(const uint8_t *mask, const SlotRange *slot_tab, int P, int S, int max_tiles, int2 *tile_tab,
+                               int32_t *tile_cnt, cudaStream_t stream) {
+    fused_tiles_kernel<<<1, 32, 0, stream>>>(mask, slot_tab, P, S, max_tiles, tile_tab, tile_cnt);
+    return cudaGetLastError();
 }
 
 }  // namespace dt

@@ -36,6 +36,16 @@ struct AttnParams {
     int B, H, L, P, S;
     int qblocks_max;          // ceil(max_i n_i / (ATTN_NQ * ATTN_TILE))
     float scale_log2;         // softmax_scale * log2(e)
+    // fused mode (dt_attn_fused): one pass per query block over the keys of all COMPUTE slots of its partition,
+    // composed in the epilogue with the composed reuse state and written as the attention output
+    const int2 *tile_tab;     // device, [P][max_tiles]: (first key, keys that count) of every K/V tile
+    const int32_t *tile_cnt;  // device, [P]: tiles per query partition
+    int max_tiles;
+    const void *comp_o;       // composed reuse state [B][H][L][D] in the cache dtype, or null
+    const float *comp_lse;    // [B][H][L]
+    void *out;                // bf16 [B, L, H, D] with the strides below
+    float *lse_out;           // [B][H][L], may be null
+    long long sb, sl, sh;
 };
 
 enum : int { MERGE_ALL = 0, MERGE_COMPOSE = 1, MERGE_PLANNED = 2 };
@@ -135,6 +145,10 @@ cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist,
                             int P, int S, int group_mode, int step, cudaStream_t stream);
 cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                                const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream);
+cudaError_t launch_attn_fused(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
+                              const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream);
+cudaError_t launch_fused_tiles(const uint8_t *mask, const SlotRange *slot_tab, int P, int S, int max_tiles, int2 *tile_tab,
+                               int32_t *tile_cnt, cudaStream_t stream);
 cudaError_t attn_states_configure();  // sets the dynamic shared-memory attribute once per process/device
 cudaError_t launch_state_merge(const MergeParams &p, int D, int state_dtype, cudaStream_t stream);
 cudaError_t launch_merge_select(const uint8_t *mask, const uint32_t *nonempty, int P, int S, int want_compute,
@@ -166,6 +180,9 @@ struct dt_ctx {
     int32_t *off_dev = nullptr;
     int32_t *tc_dev = nullptr;
     int32_t *worklist_dev = nullptr;
+    int2 *tile_tab_dev = nullptr;     // fused mode: [P][max_tiles]
+    int32_t *tile_cnt_dev = nullptr;  // [P]
+    int max_tiles = 0;
     int32_t *status_dev = nullptr;
     float *plan_partials_dev = nullptr;
     uint32_t *sel_bits_dev = nullptr;
