@@ -58,11 +58,13 @@ struct Cfg {
     static constexpr int NHALF = D / 64;                      // 64-element (128-byte) swizzle atoms per row
     static constexpr int HALF_BYTES = ATTN_TILE * 128;        // one [128 rows x 64 bf16] box
     static constexpr int TILE_BYTES = NHALF * HALF_BYTES;     // one Q, K or V tile
-    static constexpr int STAGES = (D == 128) ? 5 : 10;        // K/V ring depth
+    static constexpr int STAGES = (D == 128) ? 4 : 8;         // K/V ring depth
     static constexpr int Q_BYTES = ATTN_NQ * TILE_BYTES;
     static constexpr int KV_BYTES = STAGES * TILE_BYTES;
+    static constexpr int OUT_STAGE_BYTES = ATTN_TILE * 128;   // epilogue staging per query tile: 128 rows x 128 bytes
+    static constexpr int OUT_BYTES = ATTN_NQ * OUT_STAGE_BYTES;
     static constexpr int NBARS = 2 + 2 * STAGES + 4 * ATTN_NQ;
-    static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + Q_BYTES + KV_BYTES + NBARS * 8 + 64;
+    static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + Q_BYTES + KV_BYTES + OUT_BYTES + NBARS * 8 + 64;
     // TMEM columns
     static constexpr int S_COL = 0;                           // S tile q: S_COL + q*128
     static constexpr int O_COL = ATTN_NQ * 128;               // O tile q: O_COL + q*D
@@ -186,7 +188,8 @@ __device__ __forceinline__ void load_state_chunk(const __nv_bfloat16 *src, float
 template <int D, typename StateT, bool FUSED>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                   const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
+                   const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_state,
+                   const AttnParams p) {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_slot;
@@ -196,7 +199,8 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t q_smem = smem_base;
     const uint32_t kv_smem = q_smem + C::Q_BYTES;
-    const uint32_t bar_base = kv_smem + C::KV_BYTES;
+    const uint32_t out_smem = kv_smem + C::KV_BYTES;        // 1024-byte aligned: every size above is a multiple
+    const uint32_t bar_base = out_smem + C::OUT_BYTES;
     Bars bars;
     bars.q_full = bar_base;
     bars.q_empty = bar_base + 8;
@@ -572,16 +576,64 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 if (row_valid && p.lse_out != nullptr) p.lse_out[crow] = lse_row;
             } else {
                 const long long srow = ((long long)it.slot * p.B * p.H + it.bh) * p.L + it.q_row0 + row_in_block;
+                if (it.n_q >= (q + 1) * ATTN_TILE) {
+                    // Whole query tile inside the partition: rows go through shared memory (128 bytes of every row
+                    // at a time, 128-byte swizzle) and leave as one tiled bulk store per chunk -- whole lines instead
+                    // of 16 bytes per lane at a 512-byte stride.
+                    constexpr int CH = 128 / (int)sizeof(StateT);          // state elements per 128-byte chunk
+                    const uint32_t stage = out_smem + q * C::OUT_STAGE_BYTES;
+                    const uint32_t my_row = stage + row_in_tile * 128;
+                    const bool issuer = ((warp % 4) == 0 && lane == 0);
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 32) {
-                    uint32_t o[32];
-                    tmem_ld_x32(o_tmem + c0, o);
-                    tmem_wait_ld();
-                    if (c0 + 32 >= D) {  // O[q] fully read: the next item's first PV may overwrite it
-                        tc_fence_before();
-                        mbar_arrive(bars.o_free + 8 * q);
+                    for (int c0 = 0; c0 < D; c0 += CH) {
+                        uint32_t o[CH / 32][32];
+#pragma unroll
+                        for (int u = 0; u < CH / 32; ++u) tmem_ld_x32(o_tmem + c0 + 32 * u, o[u]);
+                        tmem_wait_ld();
+                        if (c0 + CH >= D) {  // O[q] fully read: the next item's first PV may overwrite it
+                            tc_fence_before();
+                            mbar_arrive(bars.o_free + 8 * q);
+                        }
+                        if (issuer) bulk_wait_group_read0();   // the previous chunk's store has read the staging tile
+                        named_bar_sync(1 + q, 128);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {   // 16-byte piece c of this row's 128 bytes
+                            uint4 v;
+                            if constexpr (sizeof(StateT) == 4) {
+                                v.x = __float_as_uint(__uint_as_float(o[0][4 * c]) * inv_l);
+                                v.y = __float_as_uint(__uint_as_float(o[0][4 * c + 1]) * inv_l);
+                                v.z = __float_as_uint(__uint_as_float(o[0][4 * c + 2]) * inv_l);
+                                v.w = __float_as_uint(__uint_as_float(o[0][4 * c + 3]) * inv_l);
+                            } else {
+                                const uint32_t(&oo)[32] = o[(8 * c) / 32];
+                                const int b0 = (8 * c) % 32;
+                                v.x = pack_bf16x2(__uint_as_float(oo[b0]) * inv_l, __uint_as_float(oo[b0 + 1]) * inv_l);
+                                v.y = pack_bf16x2(__uint_as_float(oo[b0 + 2]) * inv_l, __uint_as_float(oo[b0 + 3]) * inv_l);
+                                v.z = pack_bf16x2(__uint_as_float(oo[b0 + 4]) * inv_l, __uint_as_float(oo[b0 + 5]) * inv_l);
+                                v.w = pack_bf16x2(__uint_as_float(oo[b0 + 6]) * inv_l, __uint_as_float(oo[b0 + 7]) * inv_l);
+                            }
+                            const uint32_t dst = my_row + (uint32_t)((c ^ (row_in_tile & 7)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+                        }
+                        fence_proxy_async_smem();
+                        named_bar_sync(1 + q, 128);
+                        if (issuer) {
+                            tma_store_2d(&tmap_state, stage, c0, (int)(srow - row_in_tile));
+                            bulk_commit_group();
+                        }
                     }
-                    if (row_valid) store_state_chunk<StateT>(o_state + srow * D + c0, o, inv_l);
+                } else {
+#pragma unroll
+                    for (int c0 = 0; c0 < D; c0 += 32) {
+                        uint32_t o[32];
+                        tmem_ld_x32(o_tmem + c0, o);
+                        tmem_wait_ld();
+                        if (c0 + 32 >= D) {  // O[q] fully read: the next item's first PV may overwrite it
+                            tc_fence_before();
+                            mbar_arrive(bars.o_free + 8 * q);
+                        }
+                        if (row_valid) store_state_chunk<StateT>(o_state + srow * D + c0, o, inv_l);
+                    }
                 }
                 if (row_valid) p.lse_state[srow] = lse_fresh;
             }
@@ -590,6 +642,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             if (!*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
             *abort_ptr = 1;
         }
+        if ((warp % 4) == 0 && lane == 0) bulk_wait_group0();   // this thread's state stores have left shared memory
     }
 
     tc_fence_before();
@@ -599,9 +652,9 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 }
 
 template <int D, typename StateT, bool FUSED>
-cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const AttnParams &p,
-                   int num_ctas, cudaStream_t stream) {
-    attn_states_kernel<D, StateT, FUSED><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, p);
+cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
+                   const AttnParams &p, int num_ctas, cudaStream_t stream) {
+    attn_states_kernel<D, StateT, FUSED><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, ts, p);
     return cudaGetLastError();
 }
 
@@ -662,24 +715,25 @@ cudaError_t attn_states_configure() {
     return configure<128, __nv_bfloat16>();
 }
 
-cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
+cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
                                const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream) {
     if (state_dtype == DT_STATE_FP32) {
-        return D == 64 ? launch<64, float, false>(tq, tk, tv, p, num_ctas, stream)
-                       : launch<128, float, false>(tq, tk, tv, p, num_ctas, stream);
+        return D == 64 ? launch<64, float, false>(tq, tk, tv, ts, p, num_ctas, stream)
+                       : launch<128, float, false>(tq, tk, tv, ts, p, num_ctas, stream);
     }
-    return D == 64 ? launch<64, __nv_bfloat16, false>(tq, tk, tv, p, num_ctas, stream)
-                   : launch<128, __nv_bfloat16, false>(tq, tk, tv, p, num_ctas, stream);
+    return D == 64 ? launch<64, __nv_bfloat16, false>(tq, tk, tv, ts, p, num_ctas, stream)
+                   : launch<128, __nv_bfloat16, false>(tq, tk, tv, ts, p, num_ctas, stream);
 }
 
 cudaError_t launch_attn_fused(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                               const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream) {
+    // the fused epilogue stores the attention output itself: the state map is not used (any valid map will do)
     if (state_dtype == DT_STATE_FP32) {
-        return D == 64 ? launch<64, float, true>(tq, tk, tv, p, num_ctas, stream)
-                       : launch<128, float, true>(tq, tk, tv, p, num_ctas, stream);
+        return D == 64 ? launch<64, float, true>(tq, tk, tv, tq, p, num_ctas, stream)
+                       : launch<128, float, true>(tq, tk, tv, tq, p, num_ctas, stream);
     }
-    return D == 64 ? launch<64, __nv_bfloat16, true>(tq, tk, tv, p, num_ctas, stream)
-                   : launch<128, __nv_bfloat16, true>(tq, tk, tv, p, num_ctas, stream);
+    return D == 64 ? launch<64, __nv_bfloat16, true>(tq, tk, tv, tq, p, num_ctas, stream)
+                   : launch<128, __nv_bfloat16, true>(tq, tk, tv, tq, p, num_ctas, stream);
 }
 
 cudaError_t launch_fused_tiles(const uint8_t *mask, const SlotRange *slot_tab, int P, int S, int max_tiles, int2 *tile_tab,
