@@ -273,9 +273,12 @@ dt_status dt_plan_static(const float *lse_state_dev, const int32_t *part_offsets
 
 /* One whole step from HOST buffers: copies q, k, v (bf16 [B,L,H,D] contiguous) and the mask to the
  * device workspace, runs dt_attn_states and dt_state_merge, copies out (bf16 [B,L,H,D]) and lse
- * (fp32 [B,H,L], may be NULL) back and synchronises `stream`.  workspace_dev must hold
- * dt_step_host_workspace_bytes() bytes of device memory.  Host buffers should be pinned for
- * full copy bandwidth. */
+ * (fp32 [B,H,L], may be NULL) back and synchronises `stream`.  Heads are independent, so the step runs
+ * in up to 8 head chunks: the kernels of one chunk (on `stream`) overlap the host-to-device copy of the next
+ * and the device-to-host copy of the previous one, which run on two streams the context owns (ordered against
+ * `stream` with events; the call returns with all three idle).  workspace_dev must hold
+ * dt_step_host_workspace_bytes() bytes of device memory.  Host buffers should be pinned: pageable memory
+ * makes the copies synchronous and loses the overlap. */
 dt_status dt_step_host_workspace_bytes(const dt_config *cfg, size_t *bytes);
 dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, const void *v_host,
                        const uint8_t *mask_host, int32_t step, void *out_host, float *lse_out_host,

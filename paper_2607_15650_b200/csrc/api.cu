@@ -1,5 +1,6 @@
 // C-ABI of libditango: argument checking, tensor-map encoding, launches.  No arithmetic of the
 // method lives here.
+#include <algorithm>
 #include <cmath>
 #include <cstddef>
 #include <cstdio>
@@ -250,6 +251,9 @@ dt_status dt_destroy(dt_ctx *ctx) {
     cudaFree(ctx->planner_state_dev);
     cudaFree(ctx->planner_local_partials_dev);
     cudaFree(ctx->planner_norm_partials_dev);
+    for (cudaEvent_t ev : ctx->events) cudaEventDestroy(ev);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     delete ctx;
     return DT_OK;
 }
@@ -268,9 +272,9 @@ dt_status dt_bind_cache(dt_ctx *ctx, void *o_state_dev, float *lse_state_dev, si
 }
 
 namespace {
-// mask_dev == nullptr: local (diagonal) pairs only
+// mask_dev == nullptr: local (diagonal) pairs only.  Heads [h0, h0 + hc) of every batch entry.
 dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const void *v_dev, const int64_t strides_blhd[4],
-                      const uint8_t *mask_dev, int32_t step, void *stream) {
+                      const uint8_t *mask_dev, int32_t step, void *stream, int h0 = 0, int hc = -1) {
     if (!q_dev || !k_dev || !v_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null tensor pointer");
     if (step < 0) return fail(ctx, DT_ERR_INVALID_ARG, "step must be >= 0");
     if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
@@ -298,6 +302,7 @@ dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const v
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
     p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P; p.S = ctx->S;
+    p.h0 = h0; p.H_launch = hc < 0 ? c.H : hc;
     p.qblocks_max = ctx->qblocks_max;
     p.scale_log2 = c.softmax_scale * 1.44269504088896340736f;
     e = dt::launch_attn_states(tq, tk, tv, ts, p, c.D, c.state_dtype, ctx->num_sms, st);
@@ -350,6 +355,7 @@ dt_status dt_attn_fused(dt_ctx *ctx, const void *q_dev, const void *k_dev, const
     p.worklist = ctx->worklist_dev;
     p.status = ctx->status_dev;
     p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P; p.S = ctx->S;
+    p.h0 = 0; p.H_launch = c.H;
     p.qblocks_max = ctx->qblocks_max;
     p.scale_log2 = c.softmax_scale * 1.44269504088896340736f;
     p.tile_tab = ctx->tile_tab_dev;
@@ -366,9 +372,20 @@ dt_status dt_attn_fused(dt_ctx *ctx, const void *q_dev, const void *k_dev, const
     return DT_OK;
 }
 
+namespace {
+dt_status merge_rows(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev, void *stream,
+                     long long row_begin, long long row_count);
+}
+
 dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev,
                          void *stream) {
     if (!ctx) return DT_ERR_INVALID_ARG;
+    return merge_rows(ctx, out_dev, out_strides_blhd, lse_out_dev, stream, 0, (long long)ctx->cfg.B * ctx->cfg.H * ctx->cfg.L);
+}
+
+namespace {
+dt_status merge_rows(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[4], float *lse_out_dev, void *stream,
+                     long long row_begin, long long row_count) {
     if (!out_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null output pointer");
     if (!ctx->o_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
     const char *why;
@@ -388,12 +405,14 @@ dt_status dt_state_merge(dt_ctx *ctx, void *out_dev, const int64_t out_strides_b
     p.status = ctx->status_dev;
     p.P = c.P; p.S = ctx->S; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
+    p.row_begin = row_begin; p.row_count = row_count;
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "merge launch");
     ctx->launches += 1;
     return DT_OK;
 }
+}  // namespace
 
 dt_status dt_compose_reuse(dt_ctx *ctx, const uint8_t *mask_dev, void *comp_o_dev, float *comp_lse_dev, void *stream) {
     if (!ctx) return DT_ERR_INVALID_ARG;
@@ -414,6 +433,7 @@ dt_status dt_compose_reuse(dt_ctx *ctx, const uint8_t *mask_dev, void *comp_o_de
     p.status = ctx->status_dev;
     p.P = c.P; p.S = ctx->S; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
+    p.row_begin = 0; p.row_count = p.R;
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "compose launch");
     ctx->launches += 2;
@@ -445,6 +465,7 @@ dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const voi
     p.status = ctx->status_dev;
     p.P = c.P; p.S = ctx->S; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
+    p.row_begin = 0; p.row_count = p.R;
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "planned merge launch");
@@ -548,17 +569,56 @@ dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, cons
     uint8_t *md = w + 4 * tb + ((lse_b + 255) & ~(size_t)255);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(qd, q_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy q");
-    if ((e = cudaMemcpyAsync(kd, k_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy k");
-    if ((e = cudaMemcpyAsync(vd, v_host, elems * 2, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy v");
+    // Heads are independent, so the step is cut into head chunks: chunk c + 1 is copied in (copy_in stream) and
+    // chunk c - 1 copied out (copy_out stream) while chunk c is in the kernels (the caller's stream).
+    const int nchunks = std::min(c.H, 8);
+    if (!ctx->copy_in) {
+        bool ok = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking) == cudaSuccess;
+        if (!ok) return fail(ctx, DT_ERR_CUDA, "stream creation failed");
+    }
+    while ((int)ctx->events.size() < 2 * nchunks + 1) {
+        cudaEvent_t ev;
+        if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(ctx, e, "event creation");
+        ctx->events.push_back(ev);
+    }
+    // the copies may not start before earlier work of the caller's stream that uses the workspace has finished
+    cudaEvent_t ev_start = ctx->events[2 * nchunks];
+    if ((e = cudaEventRecord(ev_start, st)) != cudaSuccess) return fail_cuda(ctx, e, "event record");
+    if ((e = cudaStreamWaitEvent(ctx->copy_in, ev_start, 0)) != cudaSuccess) return fail_cuda(ctx, e, "stream wait");
+    if ((e = cudaStreamWaitEvent(ctx->copy_out, ev_start, 0)) != cudaSuccess) return fail_cuda(ctx, e, "stream wait");
     if ((e = cudaMemcpyAsync(md, mask_host, (size_t)c.P * ctx->S, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy mask");
     const int64_t strides[4] = {(int64_t)c.L * c.H * c.D, (int64_t)c.H * c.D, c.D, 1};
+    const size_t pitch = (size_t)c.H * c.D * 2, rows2d = (size_t)c.B * c.L;
     dt_status s;
-    if ((s = dt_attn_states(ctx, qd, kd, vd, strides, md, step, stream)) != DT_OK) return s;
-    if ((s = dt_state_merge(ctx, od, strides, ld, stream)) != DT_OK) return s;
-    if ((e = cudaMemcpyAsync(out_host, od, elems * 2, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail_cuda(ctx, e, "copy out");
-    if (lse_out_host && (e = cudaMemcpyAsync(lse_out_host, ld, lse_b, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-        return fail_cuda(ctx, e, "copy lse");
+    for (int ch = 0; ch < nchunks; ++ch) {
+        const int h0 = (int)((long long)ch * c.H / nchunks), h1 = (int)((long long)(ch + 1) * c.H / nchunks), hc = h1 - h0;
+        const size_t col = (size_t)h0 * c.D * 2, width = (size_t)hc * c.D * 2;
+        const void *src[3] = {q_host, k_host, v_host};
+        void *dst[3] = {qd, kd, vd};
+        for (int x = 0; x < 3; ++x)
+            if ((e = cudaMemcpy2DAsync(static_cast<uint8_t *>(dst[x]) + col, pitch, static_cast<const uint8_t *>(src[x]) + col, pitch, width,
+                                       rows2d, cudaMemcpyHostToDevice, ctx->copy_in)) != cudaSuccess)
+                return fail_cuda(ctx, e, "copy q, k, v");
+        cudaEvent_t ev_in = ctx->events[2 * ch], ev_done = ctx->events[2 * ch + 1];
+        if ((e = cudaEventRecord(ev_in, ctx->copy_in)) != cudaSuccess) return fail_cuda(ctx, e, "event record");
+        if ((e = cudaStreamWaitEvent(st, ev_in, 0)) != cudaSuccess) return fail_cuda(ctx, e, "stream wait");
+        if ((s = attn_launch(ctx, qd, kd, vd, strides, md, step, stream, h0, hc)) != DT_OK) return s;
+        for (int b = 0; b < c.B; ++b)
+            if ((s = merge_rows(ctx, od, strides, ld, stream, ((long long)b * c.H + h0) * c.L, (long long)hc * c.L)) != DT_OK) return s;
+        if ((e = cudaEventRecord(ev_done, st)) != cudaSuccess) return fail_cuda(ctx, e, "event record");
+        if ((e = cudaStreamWaitEvent(ctx->copy_out, ev_done, 0)) != cudaSuccess) return fail_cuda(ctx, e, "stream wait");
+        if ((e = cudaMemcpy2DAsync(static_cast<uint8_t *>(out_host) + col, pitch, static_cast<uint8_t *>(od) + col, pitch, width, rows2d,
+                                   cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
+            return fail_cuda(ctx, e, "copy out");
+        if (lse_out_host)
+            for (int b = 0; b < c.B; ++b) {
+                const size_t o = ((size_t)b * c.H + h0) * c.L;
+                if ((e = cudaMemcpyAsync(lse_out_host + o, ld + o, (size_t)hc * c.L * 4, cudaMemcpyDeviceToHost, ctx->copy_out)) != cudaSuccess)
+                    return fail_cuda(ctx, e, "copy lse");
+            }
+    }
+    if ((e = cudaStreamSynchronize(ctx->copy_out)) != cudaSuccess) return fail_cuda(ctx, e, "synchronise");
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(ctx, e, "synchronise");
     return DT_OK;
 }
@@ -740,6 +800,7 @@ dt_status dt_group_compose(dt_ctx *ctx, void *stream) {
         p.status = ctx->status_dev;
         p.P = c.P; p.S = S_old; p.H = c.H; p.L = c.L;
         p.R = (long long)R;
+        p.row_begin = 0; p.row_count = p.R;
         e = dt::launch_state_merge(p, c.D, c.state_dtype, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e, "group compose launch");
         ctx->launches += 1;

@@ -113,15 +113,16 @@ struct WorkItem {
 template <bool FUSED>
 __device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, long long w, WorkItem &it) {
     const long long per_bh = (long long)npairs * p.qblocks_max;
-    it.bh = (int)(w / per_bh);
-    const int rem = (int)(w - (long long)it.bh * per_bh);
+    const int bh_launch = (int)(w / per_bh);          // index among the (b, h) of this launch
+    const int rem = (int)(w - (long long)bh_launch * per_bh);
     const int pair = rem / p.qblocks_max;
     const int qb = rem - pair * p.qblocks_max;
     const int code = FUSED ? pair : p.worklist[1 + pair];
     it.i = code & 0xFF;
     it.slot = code >> 8;
-    it.b = it.bh / p.H;
-    it.h = it.bh - it.b * p.H;
+    it.b = bh_launch / p.H_launch;
+    it.h = p.h0 + bh_launch - it.b * p.H_launch;
+    it.bh = it.b * p.H + it.h;
     const int qs = p.off[it.i], qe = p.off[it.i + 1];
     it.q_row0 = qs + qb * (ATTN_NQ * ATTN_TILE);
     it.n_q = min(qe - it.q_row0, ATTN_NQ * ATTN_TILE);
@@ -240,7 +241,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     const uint32_t tmem_base = tmem_base_slot;
 
     const int npairs = FUSED ? p.P : p.worklist[0];
-    const long long total_work = (long long)npairs * p.qblocks_max * p.B * p.H;
+    const long long total_work = (long long)npairs * p.qblocks_max * p.B * p.H_launch;
 
     if (warp >= TMA_WARP) {
       reg_dealloc<REGS_PRODUCER>();

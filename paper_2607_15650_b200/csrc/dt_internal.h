@@ -34,6 +34,7 @@ struct AttnParams {
     void *o_state;            // [S][B][H][L][D]
     float *lse_state;         // [S][B][H][L]
     int B, H, L, P, S;
+    int h0, H_launch;         // heads [h0, h0 + H_launch) are processed by this launch (the whole range: 0, H)
     int qblocks_max;          // ceil(max_i n_i / (ATTN_NQ * ATTN_TILE))
     float scale_log2;         // softmax_scale * log2(e)
     // fused mode (dt_attn_fused): one pass per query block over the keys of all COMPUTE slots of its partition,
@@ -65,7 +66,8 @@ struct MergeParams {
     float *lse_out;  // may be null
     int32_t *status; // device status word
     int P, S, H, L;  // query partitions, cache slots
-    long long R;     // B*H*L rows
+    long long R;     // B*H*L rows (the slot stride of the cache)
+    long long row_begin, row_count;   // rows [row_begin, row_begin + row_count) are processed by this launch
     long long sb, sl, sh;  // output strides in elements
 };
 
@@ -195,6 +197,8 @@ struct dt_ctx {
     double planner_eps_local = 0.0, planner_cache_ratio = 0.0;   // 2 * DT_MAX_P words: composition, planned merge
     void *o_state = nullptr;
     float *lse_state = nullptr;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;   // dt_step_host: H2D and D2H overlap the kernels
+    std::vector<cudaEvent_t> events;                       // created on first use
     uint64_t launches = 0;
     std::string err;
     void *encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime

@@ -122,8 +122,8 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
     uint8_t *src_s = reinterpret_cast<uint8_t *>(abort_flag + 2);                             // [NS] source ids in staging order
     const uint32_t bar = smem_u32(bar_ptr);
 
-    const long long row0 = (long long)blockIdx.x * ROWS;
-    const int valid = (int)min((long long)ROWS, p.R - row0);   // rows of this block that exist
+    const long long row0 = p.row_begin + (long long)blockIdx.x * ROWS;
+    const int valid = (int)min((long long)ROWS, p.row_begin + p.row_count - row0);   // rows of this block that exist
     const uint32_t bytes = (uint32_t)valid * Cf::ROW_BYTES;
 
     // query partition of a cache row (token index l = row mod L); the offsets travel as kernel
@@ -248,7 +248,7 @@ cudaError_t launch_mode(const MergeParams &p, cudaStream_t stream) {
     using Cf = MergeCfg<StateT, D>;
     const int rows = Cf::rows(MODE, p.S);
     const size_t smem = Cf::smem_bytes(MODE, p.S);
-    const long long blocks = (p.R + rows - 1) / rows;
+    const long long blocks = (p.row_count + rows - 1) / rows;
     if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(state_merge_kernel<StateT, D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          MERGE_STAGE_BYTES + MERGE_THREADS * (DT_MAX_P + 1) * (int)sizeof(float) + 128);
