@@ -168,7 +168,7 @@ def aggregate_throughput(units_per_rank: float, seconds_max: float, world: int) 
 
 
 # ------------------------------------------------------------------------------------------ oracle legs
-def oracle_sample(wl, q, k, v, mask, budget_s: float, seed: int = 0):
+def oracle_sample(wl, q, k, v, mask, budget_s: float, seed: int = 0, fp16: bool = False):
     """Time the oracle, as it stands, on a bounded sample: one head, a seeded subset of query rows;
     per row the COMPUTE pair states of its partition (Eq. 1) and the P-way merge (Eq. 2) -- REUSE
     states are taken as already cached (zeros stand in; the arithmetic cost is the same).
@@ -189,7 +189,7 @@ def oracle_sample(wl, q, k, v, mask, budget_s: float, seed: int = 0):
                 continue
             for j in range(wl.P):
                 if mask[i, j]:
-                    o, l = orc.pair_state(qb, kb, vb, wl.scale, 0, 0, rows[sel], int(off[j]), int(off[j + 1]))
+                    o, l = orc.pair_state(qb, kb, vb, wl.scale, 0, 0, rows[sel], int(off[j]), int(off[j + 1]), fp16=fp16)
                     o_st[sel, j], l_st[sel, j] = o, l
         orc.merge(o_st, l_st)
         return time.perf_counter() - t0
@@ -255,13 +255,15 @@ def run_cuda(args, wl):
     state_dtype = binding.DT_STATE_BF16 if args.state_dtype == "bf16" else binding.DT_STATE_FP32
     sbytes = 2 if args.state_dtype == "bf16" else 4
 
-    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale, state_dtype, local, group_size=args.group_size)
+    in_dt = torch.float16 if args.dtype == "fp16" else torch.bfloat16
+    ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale, state_dtype, local, group_size=args.group_size,
+                          input_dtype=binding.DT_INPUT_FP16 if args.dtype == "fp16" else binding.DT_INPUT_BF16)
     S, g = ctx.dt_num_slots()
-    gen = inputs.StepInputs(wl, seed=0, device=dev)
+    gen = inputs.StepInputs(wl, seed=0, device=dev, dtype=in_dt)
     steps_in = [gen.next() for _ in range(wl.steps)]          # resident bf16 inputs of every denoising step
     del gen
     torch.cuda.empty_cache()
-    out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
+    out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=in_dt, device=dev)
     lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
     PP = wl.P * S            # decisions per plan: [P][S] (S = P without grouping)
     masks = [torch.ones(PP, dtype=torch.uint8, device=dev), torch.ones(PP, dtype=torch.uint8, device=dev)]
@@ -395,7 +397,7 @@ def run_cuda(args, wl):
         cfg = ctx.cfg
         ws = torch.empty(binding.dt_step_host_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
         qh, kh, vh = (x.cpu().pin_memory() for x in steps_in[1 % wl.steps])
-        oh = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+        oh = torch.empty(out.shape, dtype=in_dt).pin_memory()
         lh = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
         mh = masks[cur].cpu()
         times = []
@@ -415,7 +417,7 @@ def run_cuda(args, wl):
     # ---- CPU oracle on a bounded sample of the same workload
     cpu = None
     if not args.no_cpu_baseline:
-        eff, secs, desc, cores = oracle_sample(wl, *steps_in[1 % wl.steps], mask_np, budget_s=15.0)
+        eff, secs, desc, cores = oracle_sample(wl, *steps_in[1 % wl.steps], mask_np, budget_s=15.0, fp16=args.dtype == "fp16")
         cpu = {"value": eff, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds": secs}
 
     attn_avg_ms = float(np.mean(attn_ms))
@@ -424,7 +426,7 @@ def run_cuda(args, wl):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+        "dtype": args.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "D": wl.D, "L": wl.L, "P": wl.P,
                    "computed_pairs": n_comp, "computed_pair_fraction": n_comp / (wl.P * wl.P),
                    "group_size": g, "cache_slots": S, "computed_slots": n_slots_comp, "state_dtype": args.state_dtype,
@@ -473,6 +475,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--fraction", type=float, default=None, help="target computed-pair fraction of the plan")
     ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"], help="element type of q, k, v and the output")
     ap.add_argument("--heads", type=int, default=None,
                     help="override the head count (smaller captures under a profiler; not a bench configuration)")
     ap.add_argument("--composed", action="store_true",

@@ -22,7 +22,8 @@
  *     Conditions only the device can see (REUSE of a never-computed pair, a bounded wait
  *     that ran out) are recorded in a device status word that dt_poll reads.
  *   - Natural logarithm everywhere an LSE crosses this boundary.
- *   - Limits: D in {64, 128}; 1 <= P <= 32; bf16 inputs; innermost stride 1.
+ *   - Limits: D in {64, 128}; 1 <= P <= 32; bf16 or fp16 inputs ("bf16" below stands for the configured
+ *     input type); innermost stride 1.
  *
  * Memory layout of the state cache (caller-owned device memory, sized by dt_cache_bytes):
  *   o_state   [S (slot)][B][H][L][D]   fp32 or bf16 (dt_config.state_dtype)
@@ -59,6 +60,7 @@ typedef enum {
 } dt_status;
 
 enum { DT_STATE_FP32 = 0, DT_STATE_BF16 = 1 };
+enum { DT_INPUT_BF16 = 0, DT_INPUT_FP16 = 1 };
 enum { DT_MAX_P = 32 };
 
 typedef struct {
@@ -68,6 +70,9 @@ typedef struct {
     int32_t state_dtype;         /* DT_STATE_FP32 or DT_STATE_BF16: storage type of cached OUT_ij    */
     int32_t device;              /* CUDA device ordinal                                              */
     int32_t group_size;          /* 0 or 1: pair mode; g >= 2: grouped cache with g partitions per group */
+    int32_t input_dtype;         /* DT_INPUT_BF16 or DT_INPUT_FP16: element type of q, k, v and of the attention
+                                    output (Table 1: the Wan models run in FP16); P is rounded to the same type for
+                                    the PV product, accumulation stays fp32 */
 } dt_config;
 
 /* Create / destroy a context.  dt_create makes `device` current, checks it is sm_100, copies the

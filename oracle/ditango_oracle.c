@@ -7,7 +7,7 @@
  * shares no code, header, table or helper with the CUDA path.
  *
  * Everything is fp64, plain loops, no tiling, no online softmax, no fusion.
- * Inputs Q, K, V are bf16 bit patterns (uint16) in layout [B, L, H, D]; they
+ * Inputs Q, K, V are bf16 (or, with in_fp16, IEEE fp16) bit patterns (uint16) in layout [B, L, H, D]; they
  * are widened exactly to double before any arithmetic.
  *
  * Notation (paper, Section 2.2.4 and Section 4):
@@ -41,6 +41,24 @@ static inline double bf16_to_f64(uint16_t bits) {
     return (double)f;
 }
 
+/* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits; subnormals, infinities and NaN included */
+static inline double f16_to_f64(uint16_t bits) {
+    int sign = bits >> 15, e = (bits >> 10) & 0x1F, frac = bits & 0x3FF;
+    double v;
+    if (e == 0) v = ldexp((double)frac, -24);
+    else if (e == 31) v = frac ? NAN : INFINITY;
+    else v = ldexp((double)(1024 + frac), e - 25);
+    return sign ? -v : v;
+}
+
+/* element of q, k or v as a double: the bit pattern is bf16 (in_fp16 == 0) or fp16 */
+static inline double in_to_f64(uint16_t bits, int in_fp16) {
+    return in_fp16 ? f16_to_f64(bits) : bf16_to_f64(bits);
+}
+
+/* exposed for the pins: widening of one bit pattern */
+double orc_widen(uint16_t bits, int in_fp16) { return in_to_f64(bits, in_fp16); }
+
 int orc_num_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();
@@ -65,7 +83,7 @@ static inline size_t idx4(int b, int l, int h, int d, int L, int H, int D) {
 int orc_pair_state(const uint16_t *q, const uint16_t *k, const uint16_t *v,
                    int B, int L, int H, int D, double scale, int b, int h,
                    const int32_t *rows, int nrows, int key_begin, int key_end,
-                   double *out, double *lse) {
+                   double *out, double *lse, int in_fp16) {
     if (b < 0 || b >= B || h < 0 || h >= H || key_begin < 0 || key_end > L || key_begin >= key_end)
         return -1;
     int nk = key_end - key_begin;
@@ -82,7 +100,7 @@ int orc_pair_state(const uint16_t *q, const uint16_t *k, const uint16_t *v,
             for (int c = 0; c < nk; ++c) {
                 const uint16_t *kc = k + idx4(b, key_begin + c, h, 0, L, H, D);
                 double dot = 0.0;
-                for (int d = 0; d < D; ++d) dot += bf16_to_f64(qr[d]) * bf16_to_f64(kc[d]);
+                for (int d = 0; d < D; ++d) dot += in_to_f64(qr[d], in_fp16) * in_to_f64(kc[d], in_fp16);
                 x[c] = scale * dot;
                 if (x[c] > m) m = x[c];
             }
@@ -93,7 +111,7 @@ int orc_pair_state(const uint16_t *q, const uint16_t *k, const uint16_t *v,
             for (int c = 0; c < nk; ++c) {
                 double p = exp(x[c] - m);
                 const uint16_t *vc = v + idx4(b, key_begin + c, h, 0, L, H, D);
-                for (int d = 0; d < D; ++d) o[d] += p * bf16_to_f64(vc[d]);
+                for (int d = 0; d < D; ++d) o[d] += p * in_to_f64(vc[d], in_fp16);
             }
             for (int d = 0; d < D; ++d) o[d] /= ell;
             lse[ri] = m + log(ell);
@@ -112,7 +130,7 @@ int orc_pair_state(const uint16_t *q, const uint16_t *k, const uint16_t *v,
  */
 int orc_full_attention(const uint16_t *q, const uint16_t *k, const uint16_t *v,
                        int B, int L, int H, int D, double scale, int b, int h,
-                       const int32_t *rows, int nrows, double *out, double *lse) {
+                       const int32_t *rows, int nrows, double *out, double *lse, int in_fp16) {
     if (b < 0 || b >= B || h < 0 || h >= H) return -1;
     int bad = 0;
 #pragma omp parallel
@@ -127,7 +145,7 @@ int orc_full_attention(const uint16_t *q, const uint16_t *k, const uint16_t *v,
             for (int c = 0; c < L; ++c) {
                 const uint16_t *kc = k + idx4(b, c, h, 0, L, H, D);
                 double dot = 0.0;
-                for (int d = 0; d < D; ++d) dot += bf16_to_f64(qr[d]) * bf16_to_f64(kc[d]);
+                for (int d = 0; d < D; ++d) dot += in_to_f64(qr[d], in_fp16) * in_to_f64(kc[d], in_fp16);
                 p[c] = scale * dot;
                 if (p[c] > m) m = p[c];
             }
@@ -138,7 +156,7 @@ int orc_full_attention(const uint16_t *q, const uint16_t *k, const uint16_t *v,
             for (int d = 0; d < D; ++d) o[d] = 0.0;
             for (int c = 0; c < L; ++c) {
                 const uint16_t *vc = v + idx4(b, c, h, 0, L, H, D);
-                for (int d = 0; d < D; ++d) o[d] += p[c] * bf16_to_f64(vc[d]);
+                for (int d = 0; d < D; ++d) o[d] += p[c] * in_to_f64(vc[d], in_fp16);
             }
             lse[ri] = m + log(z);
         }

@@ -5,7 +5,7 @@ Eq. 8 and Eq. 13 lives in ditango_oracle.c; this file only moves numpy arrays in
 and keeps the state cache of the selective compute / reuse step (Section 2.2.4, Fig. 6;
 cache timestep t_c of Section 4.2.2; Algorithm 1's t_c bookkeeping).
 
-Q, K, V are numpy uint16 arrays holding bf16 bit patterns in layout [B, L, H, D].
+Q, K, V are numpy uint16 arrays holding bf16 (or, with fp16=True, IEEE fp16) bit patterns in layout [B, L, H, D].
 """
 from __future__ import annotations
 
@@ -27,10 +27,12 @@ def lib():
         L.orc_num_threads.restype = C.c_int
         L.orc_pair_state.restype = C.c_int
         L.orc_pair_state.argtypes = [u16p, u16p, u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
-                                     C.c_int, C.c_int, i32p, C.c_int, C.c_int, C.c_int, f64p, f64p]
+                                     C.c_int, C.c_int, i32p, C.c_int, C.c_int, C.c_int, f64p, f64p, C.c_int]
+        L.orc_widen.restype = C.c_double
+        L.orc_widen.argtypes = [C.c_uint16, C.c_int]
         L.orc_full_attention.restype = C.c_int
         L.orc_full_attention.argtypes = [u16p, u16p, u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
-                                         C.c_int, C.c_int, i32p, C.c_int, f64p, f64p]
+                                         C.c_int, C.c_int, i32p, C.c_int, f64p, f64p, C.c_int]
         L.orc_compose2.restype = None
         L.orc_compose2.argtypes = [f64p, C.c_double, f64p, C.c_double, C.c_int, f64p, f64p]
         L.orc_merge.restype = None
@@ -64,8 +66,14 @@ def _chk_qkv(q, k, v):
     return q.shape
 
 
-def pair_state(q, k, v, scale, b, h, rows, key_begin, key_end):
+def widen(bits, fp16=False):
+    """One 16-bit pattern (bf16, or IEEE fp16) as the double the oracle computes with."""
+    return float(lib().orc_widen(int(bits), 1 if fp16 else 0))
+
+
+def pair_state(q, k, v, scale, b, h, rows, key_begin, key_end, fp16=False):
     """Eq. 1 for the listed query rows of (b, h) against keys [key_begin, key_end).
+    q, k, v hold bf16 bit patterns, or fp16 ones with fp16=True (Table 1: the Wan models run in FP16).
 
     Returns (OUT [nrows, D], LSE [nrows]) in fp64."""
     B, L, H, D = _chk_qkv(q, k, v)
@@ -74,13 +82,13 @@ def pair_state(q, k, v, scale, b, h, rows, key_begin, key_end):
     lse = np.empty((rows.size,), dtype=np.float64)
     rc = lib().orc_pair_state(_p(q, C.c_uint16), _p(k, C.c_uint16), _p(v, C.c_uint16), B, L, H, D,
                               float(scale), int(b), int(h), _p(rows, C.c_int32), rows.size,
-                              int(key_begin), int(key_end), _p(out, C.c_double), _p(lse, C.c_double))
+                              int(key_begin), int(key_end), _p(out, C.c_double), _p(lse, C.c_double), 1 if fp16 else 0)
     if rc != 0:
         raise ValueError("orc_pair_state: bad arguments")
     return out, lse
 
 
-def full_attention(q, k, v, scale, b, h, rows):
+def full_attention(q, k, v, scale, b, h, rows, fp16=False):
     """softmax(scale * q K^T) V over all L keys for the listed rows of (b, h), fp64."""
     B, L, H, D = _chk_qkv(q, k, v)
     rows = np.ascontiguousarray(rows, dtype=np.int32)
@@ -88,7 +96,7 @@ def full_attention(q, k, v, scale, b, h, rows):
     lse = np.empty((rows.size,), dtype=np.float64)
     rc = lib().orc_full_attention(_p(q, C.c_uint16), _p(k, C.c_uint16), _p(v, C.c_uint16), B, L, H, D,
                                   float(scale), int(b), int(h), _p(rows, C.c_int32), rows.size,
-                                  _p(out, C.c_double), _p(lse, C.c_double))
+                                  _p(out, C.c_double), _p(lse, C.c_double), 1 if fp16 else 0)
     if rc != 0:
         raise ValueError("orc_full_attention: bad arguments")
     return out, lse
@@ -180,8 +188,9 @@ class OracleSession:
     which is what lets large workloads be checked on a sample.
     """
 
-    def __init__(self, B, L, H, D, off, scale, rows_by_bh):
+    def __init__(self, B, L, H, D, off, scale, rows_by_bh, fp16=False):
         self.B, self.L, self.H, self.D = B, L, H, D
+        self.fp16 = bool(fp16)
         self.off = np.ascontiguousarray(off, dtype=np.int32)
         self.P = self.off.size - 1
         self.scale = float(scale)
@@ -207,7 +216,7 @@ class OracleSession:
                 for j in range(self.P):
                     if mask[i, j]:
                         o, l = pair_state(q, k, v, self.scale, b, h, rows[sel],
-                                          int(self.off[j]), int(self.off[j + 1]))
+                                          int(self.off[j]), int(self.off[j + 1]), fp16=self.fp16)
                         self.o[bh][sel, j, :] = o
                         self.lse[bh][sel, j] = l
             outs[bh], lses[bh] = merge(self.o[bh], self.lse[bh])
@@ -360,8 +369,9 @@ class GroupedOracleSession:
     recomputed member by member (Eq. 1) and composed (Eq. 2); the output composes all slots that exist.
     compose() is Dynamic Group State Compose with k = 2 (Eq. 15); reset() returns to the original g."""
 
-    def __init__(self, B, L, H, D, off, scale, rows_by_bh, g):
+    def __init__(self, B, L, H, D, off, scale, rows_by_bh, g, fp16=False):
         self.B, self.L, self.H, self.D = B, L, H, D
+        self.fp16 = bool(fp16)
         self.off = np.ascontiguousarray(off, dtype=np.int32)
         self.P = self.off.size - 1
         self.scale = float(scale)
@@ -398,7 +408,7 @@ class GroupedOracleSession:
                     po = np.empty((sel.size, len(mem), self.D)); pl = np.empty((sel.size, len(mem)))
                     for a, j in enumerate(mem):                    # Eq. 1 per member partition
                         po[:, a, :], pl[:, a] = pair_state(q, k, v, self.scale, b, h, rows[sel],
-                                                           int(self.off[j]), int(self.off[j + 1]))
+                                                           int(self.off[j]), int(self.off[j + 1]), fp16=self.fp16)
                     self.o[bh][sel, s, :], self.lse[bh][sel, s] = merge(po, pl)   # Eq. 2: the group state
             outs[bh], lses[bh] = merge(self.o[bh], self.lse[bh])
         for i in range(self.P):

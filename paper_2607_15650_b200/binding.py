@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libditango.so")
 
 DT_OK, DT_ERR_INVALID_ARG, DT_ERR_UNSUPPORTED, DT_ERR_STATE, DT_ERR_CUDA, DT_ERR_TIMEOUT = range(6)
 DT_STATE_FP32, DT_STATE_BF16 = 0, 1
+DT_INPUT_BF16, DT_INPUT_FP16 = 0, 1
 DT_MAX_P = 32
 
 EXPORTS = [
@@ -30,7 +31,8 @@ EXPORTS = [
 class dt_config(C.Structure):
     _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("L", C.c_int32), ("P", C.c_int32),
                 ("part_offsets", C.POINTER(C.c_int32)), ("softmax_scale", C.c_float),
-                ("state_dtype", C.c_int32), ("device", C.c_int32), ("group_size", C.c_int32)]
+                ("state_dtype", C.c_int32), ("device", C.c_int32), ("group_size", C.c_int32),
+                ("input_dtype", C.c_int32)]
 
 
 class dt_planner_config(C.Structure):
@@ -100,10 +102,11 @@ def lib():
     return L
 
 
-def make_config(B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0, group_size=1):
+def make_config(B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0, group_size=1,
+                input_dtype=DT_INPUT_BF16):
     off = np.ascontiguousarray(offsets, dtype=np.int32)
     cfg = dt_config(B, H, D, L, off.size - 1, off.ctypes.data_as(C.POINTER(C.c_int32)), float(softmax_scale),
-                    int(state_dtype), int(device), int(group_size))
+                    int(state_dtype), int(device), int(group_size), int(input_dtype))
     cfg._keepalive = off
     return cfg
 
@@ -166,9 +169,10 @@ class Context:
     """Owns a dt_ctx and (optionally) the state-cache tensors bound to it."""
 
     def __init__(self, B, H, D, L, offsets, softmax_scale, state_dtype=DT_STATE_FP32, device=0, alloc_cache=True,
-                 group_size=1):
+                 group_size=1, input_dtype=DT_INPUT_BF16):
         self._h = C.c_void_p()
-        self.cfg = make_config(B, H, D, L, offsets, softmax_scale, state_dtype, device, group_size)
+        self.cfg = make_config(B, H, D, L, offsets, softmax_scale, state_dtype, device, group_size, input_dtype)
+        self.in_dtype = torch.float16 if input_dtype == DT_INPUT_FP16 else torch.bfloat16
         self.device = torch.device("cuda", device)
         s = lib().dt_create(C.byref(self._h), C.byref(self.cfg))
         if s != DT_OK:
@@ -193,7 +197,7 @@ class Context:
         self.o_state, self.lse_state = o_state, lse_state
 
     def dt_attn_states(self, q, k, v, mask_dev, step, stream=None):
-        assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and q.is_cuda
+        assert q.dtype == k.dtype == v.dtype == self.in_dtype and q.is_cuda
         assert q.stride() == k.stride() == v.stride() and q.shape == k.shape == v.shape
         assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()
         self._check(lib().dt_attn_states(self._h, C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()),
@@ -201,16 +205,16 @@ class Context:
                                          int(step), _stream_ptr(stream)))
 
     def dt_attn_local(self, q, k, v, step, stream=None):
-        assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and q.is_cuda
+        assert q.dtype == k.dtype == v.dtype == self.in_dtype and q.is_cuda
         assert q.stride() == k.stride() == v.stride() and q.shape == k.shape == v.shape
         self._check(lib().dt_attn_local(self._h, C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()),
                                         C.c_void_p(v.data_ptr()), _strides4(q), int(step), _stream_ptr(stream)))
 
     def dt_attn_fused(self, q, k, v, mask_dev, comp_o, comp_lse, out, lse_out=None, stream=None):
-        assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and q.is_cuda
+        assert q.dtype == k.dtype == v.dtype == self.in_dtype and q.is_cuda
         assert q.stride() == k.stride() == v.stride() and q.shape == k.shape == v.shape
         assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()
-        assert out.dtype == torch.bfloat16 and out.is_cuda
+        assert out.dtype == self.in_dtype and out.is_cuda
         opt = lambda t: C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p()
         if comp_o is not None and comp_lse is not None:
             assert comp_o.is_contiguous() and comp_lse.is_contiguous() and comp_o.dtype == self.o_state.dtype
@@ -219,7 +223,7 @@ class Context:
                                         C.c_void_p(out.data_ptr()), _strides4(out), opt(lse_out), _stream_ptr(stream)))
 
     def dt_state_merge(self, out, lse_out=None, stream=None):
-        assert out.dtype == torch.bfloat16 and out.is_cuda
+        assert out.dtype == self.in_dtype and out.is_cuda
         lp = C.c_void_p(lse_out.data_ptr()) if lse_out is not None else C.c_void_p()
         if lse_out is not None:
             assert lse_out.dtype == torch.float32 and lse_out.is_contiguous()
@@ -232,7 +236,7 @@ class Context:
                                            C.c_void_p(comp_lse.data_ptr()), _stream_ptr(stream)))
 
     def dt_state_merge_planned(self, mask_dev, comp_o, comp_lse, out, lse_out=None, stream=None):
-        assert out.dtype == torch.bfloat16 and out.is_cuda
+        assert out.dtype == self.in_dtype and out.is_cuda
         lp = C.c_void_p(lse_out.data_ptr()) if lse_out is not None else C.c_void_p()
         self._check(lib().dt_state_merge_planned(self._h, C.c_void_p(mask_dev.data_ptr()), C.c_void_p(comp_o.data_ptr()),
                                                  C.c_void_p(comp_lse.data_ptr()), C.c_void_p(out.data_ptr()),

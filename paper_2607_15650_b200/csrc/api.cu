@@ -38,6 +38,7 @@ dt_status check_config(const dt_config *c, const char **why) {
         if (c->part_offsets[i + 1] <= c->part_offsets[i]) { *why = "offsets must be strictly increasing"; return DT_ERR_INVALID_ARG; }
     if ((long long)c->B * c->H > 65535) { *why = "B*H exceeds 65535"; return DT_ERR_UNSUPPORTED; }
     if (c->group_size < 0 || c->group_size > c->P) { *why = "group_size must be in [0, P]"; return DT_ERR_INVALID_ARG; }
+    if (c->input_dtype != DT_INPUT_BF16 && c->input_dtype != DT_INPUT_FP16) { *why = "unknown input dtype"; return DT_ERR_UNSUPPORTED; }
     return DT_OK;
 }
 
@@ -108,7 +109,8 @@ dt_status encode_qkv_map(dt_ctx *ctx, CUtensorMap *tm, const void *base, const i
     cuuint32_t box[4] = {64, 1, (cuuint32_t)dt::ATTN_TILE, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
-        tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+        tm, c.input_dtype == DT_INPUT_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+        const_cast<void *>(base), dims, strides, box, estr,
         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -303,6 +305,7 @@ dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const v
     p.lse_state = ctx->lse_state;
     p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P; p.S = ctx->S;
     p.h0 = h0; p.H_launch = hc < 0 ? c.H : hc;
+    p.in_fp16 = c.input_dtype == DT_INPUT_FP16;
     p.qblocks_max = ctx->qblocks_max;
     p.scale_log2 = c.softmax_scale * 1.44269504088896340736f;
     e = dt::launch_attn_states(tq, tk, tv, ts, p, c.D, c.state_dtype, ctx->num_sms, st);
@@ -356,6 +359,7 @@ dt_status dt_attn_fused(dt_ctx *ctx, const void *q_dev, const void *k_dev, const
     p.status = ctx->status_dev;
     p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P; p.S = ctx->S;
     p.h0 = 0; p.H_launch = c.H;
+    p.in_fp16 = c.input_dtype == DT_INPUT_FP16;
     p.qblocks_max = ctx->qblocks_max;
     p.scale_log2 = c.softmax_scale * 1.44269504088896340736f;
     p.tile_tab = ctx->tile_tab_dev;
@@ -406,6 +410,7 @@ dt_status merge_rows(dt_ctx *ctx, void *out_dev, const int64_t out_strides_blhd[
     p.P = c.P; p.S = ctx->S; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
     p.row_begin = row_begin; p.row_count = row_count;
+    p.out_fp16 = c.input_dtype == DT_INPUT_FP16;
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "merge launch");
@@ -466,6 +471,7 @@ dt_status dt_state_merge_planned(dt_ctx *ctx, const uint8_t *mask_dev, const voi
     p.P = c.P; p.S = ctx->S; p.H = c.H; p.L = c.L;
     p.R = (long long)c.B * c.H * c.L;
     p.row_begin = 0; p.row_count = p.R;
+    p.out_fp16 = c.input_dtype == DT_INPUT_FP16;
     p.sb = out_strides_blhd[0]; p.sl = out_strides_blhd[1]; p.sh = out_strides_blhd[2];
     cudaError_t e = dt::launch_state_merge(p, c.D, c.state_dtype, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e, "planned merge launch");

@@ -186,7 +186,7 @@ __device__ __forceinline__ void load_state_chunk(const __nv_bfloat16 *src, float
     }
 }
 
-template <int D, typename StateT, bool FUSED>
+template <int D, typename StateT, bool FUSED, bool FP16>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                    const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_state,
@@ -294,8 +294,8 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
       } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t IDESC_QK = make_idesc_bf16_f32(128, ATTN_TILE, false);
-            constexpr uint32_t IDESC_PV = make_idesc_bf16_f32(128, D, true);
+            constexpr uint32_t IDESC_QK = make_idesc_bf16_f32(128, ATTN_TILE, false, FP16);
+            constexpr uint32_t IDESC_PV = make_idesc_bf16_f32(128, D, true, FP16);
             uint32_t q_phase = 0, p_phase = 0, of_phase = 0;
             RingPos<C::STAGES> ring;
             bool ok = true;
@@ -477,7 +477,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     float2 rs4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
-                        uint32_t pk[32];  // 64 keys as packed bf16 pairs (even key in the low half)
+                        uint32_t pk[32];  // 64 keys as packed 16-bit pairs in the inputs' type (even key in the low half)
 #pragma unroll
                         for (int c = half * 64; c < half * 64 + 64; c += 2) {
                             const float s0 = __uint_as_float(s[c >> 5][c & 31]), s1 = __uint_as_float(s[(c + 1) >> 5][(c + 1) & 31]);
@@ -485,7 +485,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             const float2 pp = (((c >> 1) & 7) < POLY_PER_8) ? exp2_poly2(x)
                                                                             : make_float2(ex2_approx(x.x), ex2_approx(x.y));
                             rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
-                            pk[(c >> 1) & 31] = pack_bf16x2(pp.x, pp.y);
+                            pk[(c >> 1) & 31] = pack_half2<FP16>(pp.x, pp.y);
                         }
                         tmem_st_x32(s_tmem + 32 * half, pk);
                     }
@@ -566,10 +566,10 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 #pragma unroll
                         for (int c = 0; c < 32; c += 8) {
                             uint4 v;
-                            v.x = pack_bf16x2(fmaf(w_f, __uint_as_float(o[c]), w_c * cv[c]), fmaf(w_f, __uint_as_float(o[c + 1]), w_c * cv[c + 1]));
-                            v.y = pack_bf16x2(fmaf(w_f, __uint_as_float(o[c + 2]), w_c * cv[c + 2]), fmaf(w_f, __uint_as_float(o[c + 3]), w_c * cv[c + 3]));
-                            v.z = pack_bf16x2(fmaf(w_f, __uint_as_float(o[c + 4]), w_c * cv[c + 4]), fmaf(w_f, __uint_as_float(o[c + 5]), w_c * cv[c + 5]));
-                            v.w = pack_bf16x2(fmaf(w_f, __uint_as_float(o[c + 6]), w_c * cv[c + 6]), fmaf(w_f, __uint_as_float(o[c + 7]), w_c * cv[c + 7]));
+                            v.x = pack_half2<FP16>(fmaf(w_f, __uint_as_float(o[c]), w_c * cv[c]), fmaf(w_f, __uint_as_float(o[c + 1]), w_c * cv[c + 1]));
+                            v.y = pack_half2<FP16>(fmaf(w_f, __uint_as_float(o[c + 2]), w_c * cv[c + 2]), fmaf(w_f, __uint_as_float(o[c + 3]), w_c * cv[c + 3]));
+                            v.z = pack_half2<FP16>(fmaf(w_f, __uint_as_float(o[c + 4]), w_c * cv[c + 4]), fmaf(w_f, __uint_as_float(o[c + 5]), w_c * cv[c + 5]));
+                            v.w = pack_half2<FP16>(fmaf(w_f, __uint_as_float(o[c + 6]), w_c * cv[c + 6]), fmaf(w_f, __uint_as_float(o[c + 7]), w_c * cv[c + 7]));
                             __stcs(reinterpret_cast<uint4 *>(dst + c0 + c), v);
                         }
                     }
@@ -652,27 +652,37 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp == 0) tmem_dealloc(tmem_base, 512);
 }
 
-template <int D, typename StateT, bool FUSED>
-cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
-                   const AttnParams &p, int num_ctas, cudaStream_t stream) {
-    attn_states_kernel<D, StateT, FUSED><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, ts, p);
+template <int D, typename StateT, bool FUSED, bool FP16>
+cudaError_t launch_one(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
+                       const AttnParams &p, int num_ctas, cudaStream_t stream) {
+    attn_states_kernel<D, StateT, FUSED, FP16><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, ts, p);
     return cudaGetLastError();
 }
 
 template <int D, typename StateT, bool FUSED>
+cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
+                   const AttnParams &p, int num_ctas, cudaStream_t stream) {
+    return p.in_fp16 ? launch_one<D, StateT, FUSED, true>(tq, tk, tv, ts, p, num_ctas, stream)
+                     : launch_one<D, StateT, FUSED, false>(tq, tk, tv, ts, p, num_ctas, stream);
+}
+
+template <int D, typename StateT, bool FUSED, bool FP16>
 cudaError_t configure_one() {
     cudaFuncAttributes attr;
-    cudaError_t e = cudaFuncGetAttributes(&attr, attn_states_kernel<D, StateT, FUSED>);
+    cudaError_t e = cudaFuncGetAttributes(&attr, attn_states_kernel<D, StateT, FUSED, FP16>);
     if (e != cudaSuccess) return e;
     if (attr.numRegs != LAUNCH_REGS) return cudaErrorInvalidConfiguration;   // the register hand-over would not balance
-    return cudaFuncSetAttribute(attn_states_kernel<D, StateT, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(attn_states_kernel<D, StateT, FUSED, FP16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 Cfg<D>::SMEM_BYTES);
 }
 
 template <int D, typename StateT>
 cudaError_t configure() {
-    cudaError_t e = configure_one<D, StateT, false>();
-    return e != cudaSuccess ? e : configure_one<D, StateT, true>();
+    cudaError_t e = configure_one<D, StateT, false, false>();
+    if (e == cudaSuccess) e = configure_one<D, StateT, true, false>();
+    if (e == cudaSuccess) e = configure_one<D, StateT, false, true>();
+    if (e == cudaSuccess) e = configure_one<D, StateT, true, true>();
+    return e;
 }
 
 // Fused mode: per query partition the K/V tiles of one pass over the keys of all its COMPUTE slots.  The slots'

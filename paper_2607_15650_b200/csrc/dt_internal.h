@@ -34,6 +34,7 @@ struct AttnParams {
     void *o_state;            // [S][B][H][L][D]
     float *lse_state;         // [S][B][H][L]
     int B, H, L, P, S;
+    int in_fp16;              // q, k, v (and the fused output) are fp16 instead of bf16
     int h0, H_launch;         // heads [h0, h0 + H_launch) are processed by this launch (the whole range: 0, H)
     int qblocks_max;          // ceil(max_i n_i / (ATTN_NQ * ATTN_TILE))
     float scale_log2;         // softmax_scale * log2(e)
@@ -62,7 +63,8 @@ struct MergeParams {
     float *comp_lse_out;
     const void *o_state;
     const float *lse_state;
-    void *out;       // bf16
+    void *out;       // bf16, or fp16 if out_fp16
+    int out_fp16;
     float *lse_out;  // may be null
     int32_t *status; // device status word
     int P, S, H, L;  // query partitions, cache slots

@@ -48,14 +48,12 @@ struct StateVec<__nv_bfloat16> {
     }
 };
 
+// VEC fp32 values -> 16-bit elements (bf16, or fp16 when `fp16`), one vector store
 template <int VEC>
-__device__ __forceinline__ void store_bf16(__nv_bfloat16 *p, const float (&v)[VEC]) {
+__device__ __forceinline__ void store_bf16(__nv_bfloat16 *p, const float (&v)[VEC], bool fp16 = false) {
     uint32_t w[VEC / 2];
 #pragma unroll
-    for (int i = 0; i < VEC / 2; ++i) {
-        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-        w[i] = *reinterpret_cast<uint32_t *>(&h);
-    }
+    for (int i = 0; i < VEC / 2; ++i) w[i] = fp16 ? pack_f16x2(v[2 * i], v[2 * i + 1]) : pack_bf16x2(v[2 * i], v[2 * i + 1]);
     if constexpr (VEC == 4) {
         __stcs(reinterpret_cast<uint2 *>(p), make_uint2(w[0], w[1]));
     } else {
@@ -239,7 +237,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
     const int l = (int)(row - bh * p.L);
     const int b = (int)(bh / p.H), h = (int)(bh - (long long)b * p.H);
     __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(p.out) + b * p.sb + l * p.sl + h * p.sh + lane * VEC;
-    store_bf16<VEC>(out, acc);
+    store_bf16<VEC>(out, acc, p.out_fp16 != 0);
     if (lane == 0 && p.lse_out != nullptr) p.lse_out[row] = lse_row;
 }
 

@@ -82,10 +82,11 @@ def banded_mask(P: int, width: int = 1) -> np.ndarray:
 
 
 class StepInputs:
-    """Iterates the denoising steps of one workload: (q, k, v) bf16 tensors [B, L, H, D]."""
+    """Iterates the denoising steps of one workload: (q, k, v) bf16 (or fp16) tensors [B, L, H, D]."""
 
-    def __init__(self, wl: Workload, seed: int = 0, device="cpu"):
+    def __init__(self, wl: Workload, seed: int = 0, device="cpu", dtype=torch.bfloat16):
         self.wl, self.seed, self.device = wl, seed, torch.device(device)
+        self.dtype = dtype          # 16-bit type the fp32 masters are rounded to: bfloat16 or float16
         self._masters = None
         self._step = 0
 
@@ -121,11 +122,11 @@ class StepInputs:
                 m.add_(torch.randn(m.shape, generator=g, device=self.device, dtype=torch.float32),
                        alpha=wl.sigma)
         self._step += 1
-        return tuple(m.to(torch.bfloat16) for m in self._masters)
+        return tuple(m.to(self.dtype) for m in self._masters)
 
 
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
-    """bf16 tensor -> C-contiguous numpy uint16 array of its bit patterns (host)."""
+    """bf16 (or fp16) tensor -> C-contiguous numpy uint16 array of its bit patterns (host)."""
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 

@@ -33,18 +33,20 @@ def check_lse(got, ref, what=""):
 class Run:
     """Drives one workload through the C ABI and the oracle side by side."""
 
-    def __init__(self, wl, rows_by_bh=None, state_dtype=binding.DT_STATE_FP32, seed=0, offsets=None):
+    def __init__(self, wl, rows_by_bh=None, state_dtype=binding.DT_STATE_FP32, seed=0, offsets=None, fp16=False):
         self.wl = wl
         self.off = wl.offsets() if offsets is None else np.asarray(offsets, dtype=np.int32)
         self.P = self.off.size - 1
         self.dev = torch.device("cuda", 0)
-        self.ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, self.off, wl.scale, state_dtype, 0)
-        self.gen = inputs.StepInputs(wl, seed=seed, device=self.dev)
+        in_dt = torch.float16 if fp16 else torch.bfloat16
+        self.ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, self.off, wl.scale, state_dtype, 0,
+                                   input_dtype=binding.DT_INPUT_FP16 if fp16 else binding.DT_INPUT_BF16)
+        self.gen = inputs.StepInputs(wl, seed=seed, device=self.dev, dtype=in_dt)
         if rows_by_bh is None:
             rows_by_bh = {(b, h): np.arange(wl.L, dtype=np.int32) for b in range(wl.B) for h in range(wl.H)}
         self.rows = rows_by_bh
-        self.ses = orc.OracleSession(wl.B, wl.L, wl.H, wl.D, self.off, wl.scale, rows_by_bh)
-        self.out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=self.dev)
+        self.ses = orc.OracleSession(wl.B, wl.L, wl.H, wl.D, self.off, wl.scale, rows_by_bh, fp16=fp16)
+        self.out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=in_dt, device=self.dev)
         self.lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=self.dev)
         self.t = 0
 

@@ -506,3 +506,40 @@ def test_uniform_offsets():
     assert off[0] == 0 and off[-1] == 32760
     sizes = np.diff(off)
     assert set(sizes.tolist()) == {2047, 2048} and (sizes == 2047).sum() == 8
+
+
+# ---------------------------------------------------------------- input widening (bf16 / fp16)
+
+def test_widening_of_every_16_bit_pattern_is_exact():
+    """The oracle computes with the exact value of each input element: all 65 536 bit patterns of both input
+    types against numpy / torch conversions (subnormals, infinities and NaN included)."""
+    bits = np.arange(65536, dtype=np.uint16)
+    ref16 = bits.view(np.float16).astype(np.float64)
+    refbf = widen(bits)
+    for b in range(0, 65536, 1):
+        g16, gbf = orc.widen(b, fp16=True), orc.widen(b, fp16=False)
+        assert (math.isnan(g16) and math.isnan(ref16[b])) or g16 == ref16[b], hex(b)
+        assert (math.isnan(gbf) and math.isnan(refbf[b])) or gbf == refbf[b], hex(b)
+        if b % 97:          # the full sweep of the cheap comparison above, the sign check on a subset
+            continue
+        assert math.isnan(g16) or math.copysign(1.0, g16) == math.copysign(1.0, float(ref16[b]))
+
+
+def test_fp16_inputs_full_attention_matches_library_sdpa():
+    """Table 1 (the Wan models run in FP16): the same definitions on fp16 bit patterns."""
+    rng = np.random.default_rng(12)
+    B, L, H, D = 1, 29, 2, 16
+    x = [rng.standard_normal((B, L, H, D)).astype(np.float16) for _ in range(3)]
+    q, k, v = (a.view(np.uint16).copy() for a in x)
+    qt, kt, vt = (torch.from_numpy(a.astype(np.float64)).permute(0, 2, 1, 3) for a in x)
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, scale=0.3).numpy()
+    off = orc.uniform_offsets(L, 3)
+    for h in range(H):
+        o, lse = orc.full_attention(q, k, v, 0.3, 0, h, all_rows(L), fp16=True)
+        np.testing.assert_allclose(o, ref[0, h], rtol=0, atol=1e-13)
+        ses = orc.OracleSession(B, L, H, D, off, 0.3, {(0, h): all_rows(L)}, fp16=True)
+        outs, _ = ses.step(q, k, v, np.ones((3, 3), np.uint8), 0)
+        np.testing.assert_allclose(outs[(0, h)], ref[0, h], rtol=0, atol=1e-13)
+    # the same bits read as bf16 give a different answer: the flag is not ignored
+    o_bf, _ = orc.full_attention(q, k, v, 0.3, 0, 0, all_rows(L), fp16=False)
+    assert np.abs(o_bf - ref[0, 0]).max() > 1e-3
