@@ -73,16 +73,17 @@ struct MergeCfg {
     static constexpr int TPR = D / VEC;                       // threads per row
     static constexpr int MAX_ROWS = MERGE_THREADS / TPR;      // rows the block's threads can cover
     static constexpr int ROW_BYTES = D * (int)sizeof(StateT);
-    // MERGE_ALL stages all P slots at once (64 KB per block, three blocks per SM); the subset modes stage
-    // MERGE_CHUNK sources at a time for the full MAX_ROWS rows (32 KB per block, six blocks per SM), so
-    // that a step which needs few sources per row still keeps many bytes in flight per SM.
+    // MERGE_ALL stages all slots at once (64 KB per block, three blocks per SM) as long as the block can then
+    // cover its full MAX_ROWS rows; with more slots, and in the subset modes, MERGE_CHUNK sources are staged at a
+    // time for MAX_ROWS rows (32 KB per block, six blocks per SM): bulk copies stay at 4 KB instead of shrinking
+    // with the slot count, and a step which needs few sources per row still keeps many bytes in flight per SM.
+    static bool chunked(int mode, int P) { return mode != MERGE_ALL || MERGE_STAGE_BYTES / (P * ROW_BYTES) < MAX_ROWS; }
     static int rows(int mode, int P) {
-        if (mode != MERGE_ALL) return MAX_ROWS;
-        int r = MERGE_STAGE_BYTES / (P * ROW_BYTES);
-        r = r < 1 ? 1 : r;
+        if (chunked(mode, P)) return MAX_ROWS;
+        const int r = MERGE_STAGE_BYTES / (P * ROW_BYTES);
         return r > MAX_ROWS ? MAX_ROWS : r;
     }
-    static int staged(int mode, int P) { return mode == MERGE_ALL ? P : MERGE_CHUNK; }
+    static int staged(int mode, int P) { return chunked(mode, P) ? MERGE_CHUNK : P; }
     static size_t smem_bytes(int mode, int P) {
         return (size_t)staged(mode, P) * rows(mode, P) * ROW_BYTES + (size_t)rows(mode, P) * (DT_MAX_P + 1) * sizeof(float) + 40 + 64;
     }
@@ -103,7 +104,7 @@ __device__ __forceinline__ void store_state(__nv_bfloat16 *p, const float (&v)[V
 //                  state (OUT in the cache's dtype, LSE) written to the composed-state buffers
 //   MERGE_PLANNED  the COMPUTE slots (mask != 0) plus the composed state as one more source
 template <typename StateT, int D, int MODE>
-__global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid_constant__ MergeParams p, int ROWS) {
+__global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid_constant__ MergeParams p, int ROWS, int staged) {
     using Cf = MergeCfg<StateT, D>;
     constexpr int VEC = Cf::VEC, TPR = Cf::TPR;
     constexpr int NS = DT_MAX_P + 1;   // sources per row at most: P slots + the composed state
@@ -111,7 +112,6 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
     const int P = p.S;   // sources in the cache: one per slot
     constexpr int EXTRA = (MODE == MERGE_PLANNED) ? 1 : 0;
     const int nslots = P + EXTRA;
-    const int staged = (MODE == MERGE_ALL) ? P : MERGE_CHUNK;
     StateT *tile = reinterpret_cast<StateT *>(smem);                                         // [staged][ROWS][D]
     float *lse_s = reinterpret_cast<float *>(smem + (size_t)staged * ROWS * Cf::ROW_BYTES);   // [ROWS][NS]
     uint64_t *bar_ptr = reinterpret_cast<uint64_t *>(lse_s + ((ROWS * NS + 1) & ~1));        // 8-byte aligned
@@ -251,7 +251,7 @@ cudaError_t launch_mode(const MergeParams &p, cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(state_merge_kernel<StateT, D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          MERGE_STAGE_BYTES + MERGE_THREADS * (DT_MAX_P + 1) * (int)sizeof(float) + 128);
     if (e != cudaSuccess) return e;
-    state_merge_kernel<StateT, D, MODE><<<(unsigned)blocks, MERGE_THREADS, smem, stream>>>(p, rows);
+    state_merge_kernel<StateT, D, MODE><<<(unsigned)blocks, MERGE_THREADS, smem, stream>>>(p, rows, Cf::staged(MODE, p.S));
     return cudaGetLastError();
 }
 
