@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
     __shared__ double W[DT_MAX_P * DT_MAX_P];
     __shared__ double m_s[DT_MAX_P * DT_MAX_P];
     __shared__ uint8_t size_s[DT_MAX_P * DT_MAX_P];
+    __shared__ uint8_t dist_s[DT_MAX_P * DT_MAX_P];
     __shared__ uint8_t dec_s[DT_MAX_P * DT_MAX_P];
     __shared__ double edge[2];
     const int P = p.P, total = P * P, g = p.group_size;
@@ -114,6 +115,7 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
         dist = uk > gi ? uk - gi : gi - uk;
         m_s[e] = m;
         size_s[e] = (uint8_t)size;
+        dist_s[e] = (uint8_t)dist;
     }
     __syncthreads();
     bool take = false;
@@ -125,11 +127,10 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
         } else {
             rank = 0;
             int cum = size;
-            for (int o = 0; o < nunits; ++o) {
-                if (o == e || size_s[o] == 0) continue;
-                const int oi = o / ng, ok = o - oi * ng, ogi = oi / g;
-                const int od = ok > ogi ? ok - ogi : ogi - ok;
-                if (ranks_before(m_s[o], od, o, m, dist, e)) { ++rank; cum += size_s[o]; }
+            for (int o = 0; o < nunits; ++o) {   // every thread walks the same o: shared-memory broadcasts
+                const int so = size_s[o];
+                if (o == e || so == 0) continue;
+                if (ranks_before(m_s[o], dist_s[o], o, m, dist, e)) { ++rank; cum += so; }
             }
             take = cum <= budget;
         }
@@ -164,7 +165,7 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
 __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int32_t *tc, int32_t *worklist,
                                                         int32_t *status, const SlotRange *slot_tab, int P, int S,
                                                         int group_mode, int step) {
-    __shared__ uint8_t flag[DT_MAX_P * DT_MAX_P];
+    __shared__ int warp_cnt[32];
     const int total = P * S, e = threadIdx.x;
     bool f = false;
     if (e < total) {
@@ -172,20 +173,22 @@ __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int
         const bool exists = slot_tab[e].n1 + slot_tab[e].n2 > 0;
         const int local = group_mode ? 0 : i;
         f = exists && (mask ? (mask[e] != 0) : (s == local));
-        flag[e] = f ? 1 : 0;
         if (f) tc[e] = step;
         else if (exists && mask && tc[e] < 0) atomicOr(status, STATUS_REUSE_EMPTY);
     }
+    // position of a COMPUTE entry = number of COMPUTE entries with a smaller flat index
+    const unsigned bal = __ballot_sync(0xFFFFFFFFu, f);
+    const int lane = e & 31, warp = e >> 5;
+    if (lane == 0) warp_cnt[warp] = __popc(bal);
     __syncthreads();
-    if (e < total) {
-        int pos = 0, cnt = 0;
-        for (int o = 0; o < total; ++o) {
-            cnt += flag[o];
-            if (o < e) pos += flag[o];
-        }
-        if (f) worklist[1 + pos] = (e / S) | ((e % S) << 8);
-        if (e == 0) worklist[0] = cnt;
+    int pos = __popc(bal & ((1u << lane) - 1u)), cnt = 0;
+    for (int w = 0; w < 32; ++w) {
+        const int c = warp_cnt[w];
+        cnt += c;
+        if (w < warp) pos += c;
     }
+    if (f) worklist[1 + pos] = (e / S) | ((e % S) << 8);
+    if (e == 0) worklist[0] = cnt;
 }
 
 // Decisions for a grouped cache (Section 4.2.1 - 4.2.3): W[i][s] from the partial sums; every non-local slot
@@ -195,6 +198,7 @@ __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int
 __global__ void __launch_bounds__(1024) plan_slots_kernel(PlanSlotsParams p) {
     __shared__ double m_s[DT_MAX_P * DT_MAX_P];
     __shared__ uint8_t size_s[DT_MAX_P * DT_MAX_P];
+    __shared__ uint8_t dist_s[DT_MAX_P * DT_MAX_P];
     __shared__ double edge[2];
     const int P = p.P, S = p.S, total = P * S, g = p.group_size;
     const int e = threadIdx.x;
@@ -212,6 +216,7 @@ __global__ void __launch_bounds__(1024) plan_slots_kernel(PlanSlotsParams p) {
         dist = k > gi ? k - gi : gi - k;
         m_s[e] = m;
         size_s[e] = (uint8_t)size;
+        dist_s[e] = (uint8_t)dist;
     }
     if (e < 2) edge[e] = 0.0;
     __syncthreads();
@@ -225,10 +230,9 @@ __global__ void __launch_bounds__(1024) plan_slots_kernel(PlanSlotsParams p) {
             rank = 0;
             int cum = size;
             for (int o = 0; o < total; ++o) {
-                if (o == e || size_s[o] == 0) continue;
-                const int oi = o / S, ok = o - oi * S - 1, ogi = oi / g;
-                const int od = ok > ogi ? ok - ogi : ogi - ok;
-                if (ranks_before(m_s[o], od, o, m, dist, e)) { ++rank; cum += size_s[o]; }
+                const int so = size_s[o];
+                if (o == e || so == 0) continue;
+                if (ranks_before(m_s[o], dist_s[o], o, m, dist, e)) { ++rank; cum += so; }
             }
             take = cum <= budget;
         }
