@@ -130,17 +130,22 @@ def bf16_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-def sample_rows(wl: Workload, n: int, seed: int = 0):
+def sample_rows(wl: Workload, n: int, seed: int = 0, max_heads=None):
     """n seeded (b, h, row) samples, grouped as {(b, h): sorted unique rows}; always includes the
-    first and last row of the sequence and rows next to partition boundaries."""
+    first and last row of the sequence and rows next to partition boundaries.  max_heads: draw the heads
+    from a seeded subset of that many (always containing the first and the last head)."""
     rng = np.random.Generator(np.random.PCG64(seed * 1_000_003 + STREAM_ROWS))
     off = wl.offsets()
     out = {}
+    heads = np.arange(wl.H)
+    if max_heads is not None and max_heads < wl.H:
+        inner = rng.permutation(np.arange(1, wl.H - 1))[:max(0, max_heads - 2)]
+        heads = np.unique(np.concatenate([[0, wl.H - 1], inner]))
     special = [0, wl.L - 1] + [int(o) for o in off[1:-1]] + [int(o) - 1 for o in off[1:-1]]
     for s, r in enumerate(special):
-        out.setdefault((0, s % wl.H), set()).add(r)
+        out.setdefault((0, int(heads[s % heads.size])), set()).add(r)
     bs = rng.integers(0, wl.B, size=n)
-    hs = rng.integers(0, wl.H, size=n)
+    hs = heads[rng.integers(0, heads.size, size=n)]
     rs = rng.integers(0, wl.L, size=n)
     for b, h, r in zip(bs, hs, rs):
         out.setdefault((int(b), int(h)), set()).add(int(r))

@@ -543,3 +543,25 @@ def test_fp16_inputs_full_attention_matches_library_sdpa():
     # the same bits read as bf16 give a different answer: the flag is not ignored
     o_bf, _ = orc.full_attention(q, k, v, 0.3, 0, 0, all_rows(L), fp16=False)
     assert np.abs(o_bf - ref[0, 0]).max() > 1e-3
+
+
+def test_config0_regression_values():
+    """The oracle and the seeded inputs reproduce the committed summary values of the correctness configuration
+    (regression only: written by tests/golden/make_config0_reference.py from the oracle itself)."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("make_config0_reference", os.path.join(GOLDEN, "make_config0_reference.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    want = [l.strip() for l in open(os.path.join(GOLDEN, "config0_reference.txt")) if not l.startswith("#")]
+    got = mod.summarise()
+    assert len(got) == len(want)
+    for g, w in zip(got, want):
+        gt, wt = g.split(), w.split()
+        assert len(gt) == len(wt)
+        for a, b in zip(gt, wt):
+            try:
+                fa, fb = float(a), float(b)
+            except ValueError:
+                assert a == b
+                continue
+            assert fa == pytest.approx(fb, rel=1e-9, abs=1e-12), (g, w)
