@@ -68,6 +68,33 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_partial_kernel(PlanParams p
     }
 }
 
+// Sum over (b*h, chunk) of the stage-1 partial sums of every entry (i, column), all 1024 threads taking part:
+// entry = e % total (consecutive threads read consecutive columns: coalesced), the `tpe` threads of an entry take
+// every tpe-th partial, and the entry's first thread adds their sums in a fixed order.  Result in out_s[entry].
+__device__ __forceinline__ void sum_partials(const float *partials, int P, int S, int BH, int chunks, double *scratch,
+                                             double *out_s) {
+    const int total = P * S, e = threadIdx.x;
+    int tpe = 1;
+    while (tpe * 2 * total <= 1024 && tpe < 16) tpe *= 2;
+    const int ent = e % total, part = e / total;
+    if (part < tpe) {
+        const int i = ent / S, j = ent - i * S, K = BH * chunks;
+        double s = 0.0;
+        for (int k = part; k < K; k += tpe) {
+            const int bh = k / chunks, c = k - bh * chunks;
+            s += (double)partials[(((long long)bh * P + i) * chunks + c) * S + j];
+        }
+        scratch[part * total + ent] = s;
+    }
+    __syncthreads();
+    if (e < total) {
+        double s = 0.0;
+        for (int q = 0; q < tpe; ++q) s += scratch[q * total + e];
+        out_s[e] = s;
+    }
+    __syncthreads();
+}
+
 // Strict total order used to rank decision units: larger measure first, then smaller group distance,
 // then smaller flat index.
 __device__ __forceinline__ bool ranks_before(double ma, int da, int fa, double mb, int db, int fb) {
@@ -90,14 +117,12 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
     const int P = p.P, total = P * P, g = p.group_size;
     const int ng = (P + g - 1) / g, nunits = P * ng;
     const int e = threadIdx.x;
+    sum_partials(p.partials, P, P, p.BH, p.chunks, m_s, W);   // m_s doubles as scratch here
     {
-        const int i = e / P, j = e - i * P;
+        const int i = e / P;
         if (e < total) {
-            double s = 0.0;
-            for (int bh = 0; bh < p.BH; ++bh)
-                for (int c = 0; c < p.chunks; ++c) s += (double)p.partials[(((long long)bh * P + i) * p.chunks + c) * P + j];
             const double cnt = (double)p.BH * (double)(p.off[i + 1] - p.off[i]);
-            W[e] = s / cnt;
+            W[e] = W[e] / cnt;
             if (p.w_out) p.w_out[e] = W[e];
         }
     }
@@ -203,13 +228,12 @@ __global__ void __launch_bounds__(1024) plan_slots_kernel(PlanSlotsParams p) {
     const int P = p.P, S = p.S, total = P * S, g = p.group_size;
     const int e = threadIdx.x;
     const int i = e / S, s = e - i * S;
+    __shared__ double sum_s[DT_MAX_P * DT_MAX_P];
+    sum_partials(p.partials, P, S, p.BH, p.chunks, m_s, sum_s);   // m_s doubles as scratch here
     double m = 0.0;
     int size = 0, dist = 0;
     if (e < total) {
-        double sum = 0.0;
-        for (int bh = 0; bh < p.BH; ++bh)
-            for (int c = 0; c < p.chunks; ++c) sum += (double)p.partials[(((long long)bh * P + i) * p.chunks + c) * S + s];
-        m = sum / ((double)p.BH * (double)(p.off[i + 1] - p.off[i]));
+        m = sum_s[e] / ((double)p.BH * (double)(p.off[i + 1] - p.off[i]));
         if (p.w_out) p.w_out[e] = m;
         size = (s == 0) ? 0 : (int)p.members[e];   // the local slot is no unit: always COMPUTE
         const int gi = i / g, k = s - 1;
