@@ -28,7 +28,7 @@ def _random_case(seed):
     B = int(rng.choice([1, 1, 2]))
     H = int(rng.integers(1, 4))
     P = int(rng.integers(1, 9))
-    grid = (int(rng.integers(1, 4)), int(rng.integers(5, 14)), int(rng.integers(5, 14)))
+    grid = (int(rng.integers(1, 5)), int(rng.integers(5, 21)), int(rng.integers(5, 21)))     # up to 1600 tokens
     n_text = int(rng.choice([0, 0, 3, 17]))
     L = n_text + grid[0] * grid[1] * grid[2]
     P = min(P, L // 2)
