@@ -63,17 +63,22 @@ struct Cfg {
     static constexpr int KV_BYTES = STAGES * TILE_BYTES;
     static constexpr int OUT_STAGE_BYTES = ATTN_TILE * 128;   // epilogue staging per query tile: 128 rows x 128 bytes
     static constexpr int OUT_BYTES = ATTN_NQ * OUT_STAGE_BYTES;
-    static constexpr int NBARS = 2 + 2 * STAGES + 4 * ATTN_NQ;
+    static constexpr int NBARS = 2 + 2 * STAGES + 5 * ATTN_NQ;
     static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + Q_BYTES + KV_BYTES + OUT_BYTES + NBARS * 8 + 64;
-    // TMEM columns
-    static constexpr int S_COL = 0;                           // S tile q: S_COL + q*128
-    static constexpr int O_COL = ATTN_NQ * 128;               // O tile q: O_COL + q*D
+    // TMEM columns.  D = 128 fills all 512 (S0 | S1 | O0 | O1) and P has to live over S.  D = 64 leaves 128 columns:
+    // there P gets its own place (S0 | S1 | P0 | P1 | O0 | O1), so S may be overwritten as soon as the softmax has
+    // read it and the next tile's Q K^T runs while this tile's exponentials are being taken.
+    static constexpr bool PREFETCH = (D == 64);
+    static constexpr int S_COL = 0;                                              // S tile q: S_COL + q*128
+    static constexpr int P_COL = PREFETCH ? ATTN_NQ * 128 : 0;                   // P tile q: P_COL + q*(PREFETCH ? 64 : 128)
+    static constexpr int P_STRIDE = PREFETCH ? 64 : 128;
+    static constexpr int O_COL = PREFETCH ? ATTN_NQ * 128 + ATTN_NQ * 64 : ATTN_NQ * 128;   // O tile q: O_COL + q*D
 };
 
 struct Bars {
     uint32_t q_full, q_empty;
     uint32_t kv_full, kv_empty;   // + 8*stage
-    uint32_t s_full, p_full, o_full, o_free;  // + 8*q
+    uint32_t s_full, p_full, o_full, o_free, pv_done;  // + 8*q
 };
 
 // Position in the K/V ring: stage index and the parity of its current use.
@@ -211,6 +216,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     bars.p_full = bars.s_full + 8 * ATTN_NQ;
     bars.o_full = bars.p_full + 8 * ATTN_NQ;
     bars.o_free = bars.o_full + 8 * ATTN_NQ;
+    bars.pv_done = bars.o_free + 8 * ATTN_NQ;   // D = 64 only: the PV MMAs that read P[q] have completed
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_ptr = &abort_flag;
@@ -225,9 +231,12 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         }
         for (int q = 0; q < ATTN_NQ; ++q) {
             mbar_init(bars.s_full + 8 * q, 1);
-            mbar_init(bars.p_full + 8 * q, 128 + (q == 0 ? 1 : 0));   // tile 0: + the K/V watcher
+            // D = 128: P ready (128 threads), tile 0: + the K/V watcher.  D = 64: "go" = S read + previous P stored
+            // (2 x 128) + the watcher, for both tiles
+            mbar_init(bars.p_full + 8 * q, C::PREFETCH ? 257 : 128 + (q == 0 ? 1 : 0));
             mbar_init(bars.o_full + 8 * q, 1);
             mbar_init(bars.o_free + 8 * q, 128);
+            mbar_init(bars.pv_done + 8 * q, 1);
         }
         fence_mbar_init();
     }
@@ -319,12 +328,71 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             // O[q] (+)= P[q] V for the V tile in ring stage `st`
             auto issue_pv = [&](int q, uint32_t st, bool accumulate) {
                 const uint64_t b0 = vdesc0 + (uint64_t)((st * C::TILE_BYTES) >> 4);
-                const uint32_t d = tmem_base + C::O_COL + q * D, a = tmem_base + C::S_COL + q * 128;
+                const uint32_t d = tmem_base + C::O_COL + q * D, a = tmem_base + C::P_COL + q * C::P_STRIDE;
 #pragma unroll
                 for (int kk = 0; kk < ATTN_TILE / 16; ++kk)
                     mma_ts(d, a + kk * 8, b0 + (uint64_t)((kk * 2048) >> 4), IDESC_PV, (accumulate || kk > 0) ? 1u : 0u);
             };
 
+            if constexpr (C::PREFETCH) {
+                // D = 64.  Per item, "go" phases k = 0 .. tiles for each query tile: phase k is complete when the
+                // softmax has read S_k, stored P_{k-1}, and V_{k-1}, K_{k+1} have landed.  Then O += P_{k-1} V_{k-1}
+                // (commit pv_done: P's place is free again) and S_{k+1} = Q K_{k+1}^T (commit s_full) are issued.
+                // Stage of the n-th K/V tile of the run: (n mod STAGES).
+                uint32_t abs0 = 0, go_phase = 0;   // tiles loaded before this item (K_t = abs0 + 2t, V_t = abs0 + 2t + 1)
+                for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+                    WorkItem it;
+                    if (!decode_work<FUSED>(p, npairs, w, it)) continue;
+                    ok = mbar_wait_bounded(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
+                    if (!ok) break;
+                    q_phase ^= 1u;
+                    {
+                        const uint32_t st = abs0 % C::STAGES, ph = (abs0 / C::STAGES) & 1u;
+                        ok = mbar_wait_bounded(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int q = 0; q < ATTN_NQ; ++q) {
+                            issue_qk(q, st);
+                            tc_commit(bars.s_full + 8 * q);
+                        }
+                        tc_commit(bars.kv_empty + 8 * st);
+                        if (it.tiles == 1) tc_commit(bars.q_empty);
+                    }
+                    for (int k = 0; k <= it.tiles && ok; ++k) {
+                        const uint32_t st_v = (abs0 + 2 * k - 1) % C::STAGES;   // V_{k-1} (k >= 1)
+                        const uint32_t st_k = (abs0 + 2 * k + 2) % C::STAGES;   // K_{k+1}
+                        const bool has_pv = (k >= 1), has_qk = (k + 1 < it.tiles);
+#pragma unroll
+                        for (int q = 0; q < ATTN_NQ; ++q) {
+                            ok = mbar_wait_bounded(bars.p_full + 8 * q, go_phase, abort_ptr, WAIT_LIMIT_NS);
+                            if (!ok) break;
+                            if (k == 1) {  // first PV of the item: the previous item's epilogue must have drained O[q]
+                                ok = mbar_wait_bounded(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                                if (!ok) break;
+                            }
+                            tc_fence_after();
+                            if (has_pv) {
+                                issue_pv(q, st_v, k > 1);
+                                tc_commit(k < it.tiles ? bars.pv_done + 8 * q : bars.o_full + 8 * q);   // P's place is free
+                            }
+                            if (has_qk) {
+                                issue_qk(q, st_k);
+                                tc_commit(bars.s_full + 8 * q);
+                            }
+                        }
+                        if (!ok) break;
+                        if (has_pv) tc_commit(bars.kv_empty + 8 * st_v);
+                        if (has_qk) {
+                            tc_commit(bars.kv_empty + 8 * st_k);
+                            if (k + 2 == it.tiles) tc_commit(bars.q_empty);
+                        }
+                        go_phase ^= 1u;
+                    }
+                    of_phase ^= 1u;
+                    abs0 += 2u * (uint32_t)it.tiles;
+                }
+            } else
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
                 if (!decode_work<FUSED>(p, npairs, w, it)) continue;
@@ -395,6 +463,33 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             RingPos<C::STAGES> ring;
             uint32_t p_phase = 0;
             bool ok = true;
+            if constexpr (C::PREFETCH) {
+                // D = 64: one arrival on each go[q] per phase k, made once V_{k-1} and K_{k+1} are in shared memory
+                uint32_t abs0 = 0;
+                for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+                    WorkItem it;
+                    if (!decode_work<FUSED>(p, npairs, w, it)) continue;
+                    for (int k = 0; k <= it.tiles && ok; ++k) {
+                        if (k >= 1) {
+                            const uint32_t a = abs0 + 2 * k - 1;
+                            ok = mbar_wait_bounded(bars.kv_full + 8 * (a % C::STAGES), (a / C::STAGES) & 1u, abort_ptr, WAIT_LIMIT_NS);
+                        }
+                        if (ok && k + 1 < it.tiles) {
+                            const uint32_t a = abs0 + 2 * k + 2;
+                            ok = mbar_wait_bounded(bars.kv_full + 8 * (a % C::STAGES), (a / C::STAGES) & 1u, abort_ptr, WAIT_LIMIT_NS);
+                        }
+                        if (ok) {
+#pragma unroll
+                            for (int q = 0; q < ATTN_NQ; ++q) mbar_arrive(bars.p_full + 8 * q);
+#pragma unroll
+                            for (int q = 0; q < ATTN_NQ; ++q)
+                                ok = ok && mbar_wait_bounded(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_NS);
+                            p_phase ^= 1u;
+                        }
+                    }
+                    abs0 += 2u * (uint32_t)it.tiles;
+                }
+            } else
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
                 if (!decode_work<FUSED>(p, npairs, w, it)) continue;
@@ -426,8 +521,9 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const int row_in_tile = (warp % 4) * 32 + lane;
         const uint32_t lane_addr = ((uint32_t)((warp % 4) * 32)) << 16;
         const uint32_t s_tmem = tmem_base + lane_addr + C::S_COL + q * 128;
+        const uint32_t p_tmem = tmem_base + lane_addr + C::P_COL + q * C::P_STRIDE;   // D = 128: the same columns as S
         const uint32_t o_tmem = tmem_base + lane_addr + C::O_COL + q * D;
-        uint32_t s_phase = 0, o_phase = 0;
+        uint32_t s_phase = 0, o_phase = 0, pv_phase = 0;
         bool ok = true;
         StateT *o_state = static_cast<StateT *>(p.o_state);
 
@@ -447,6 +543,12 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 tmem_ld_x32(s_tmem + 64, s[2]);
                 tmem_ld_x32(s_tmem + 96, s[3]);
                 tmem_wait_ld();
+                bool p_place_free = !C::PREFETCH || t == 0;   // D = 64: P's columns may still be read by the previous tile's PV
+                if constexpr (C::PREFETCH) {
+                    tc_fence_before();
+                    mbar_arrive(bars.p_full + 8 * q);               // S_t has been read: Q K_{t+1}^T may overwrite it
+                    if (t == 0) mbar_arrive(bars.p_full + 8 * q);   // stands in for "P_{-1} stored"
+                }
                 if (valid < ATTN_TILE) {
 #pragma unroll
                     for (int c = 0; c < 128; ++c)
@@ -487,7 +589,15 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
                             pk[(c >> 1) & 31] = pack_half2<FP16>(pp.x, pp.y);
                         }
-                        tmem_st_x32(s_tmem + 32 * half, pk);
+                        if constexpr (C::PREFETCH) {
+                            if (!p_place_free) {   // PV of tile t-1 is done with P's columns
+                                ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_NS));
+                                pv_phase ^= 1u;
+                                p_place_free = true;
+                                tc_fence_after();
+                            }
+                        }
+                        tmem_st_x32(p_tmem + 32 * half, pk);
                     }
                     const float2 r = __fadd2_rn(__fadd2_rn(rs4[0], rs4[1]), __fadd2_rn(rs4[2], rs4[3]));
                     return r.x + r.y;
@@ -519,8 +629,10 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bars.p_full + 8 * q);
+                if (!ok) break;
             }
             if (!ok) break;
+            if constexpr (C::PREFETCH) mbar_arrive(bars.p_full + 8 * q);   // closes the last phase (no further S to read)
             // epilogue: OUT_ij = O / l, LSE_ij = ln2 * (m + log2 l); rows beyond the partition are dropped
             ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.o_full + 8 * q, o_phase, abort_ptr, WAIT_LIMIT_NS));
             if (!ok) break;
