@@ -360,6 +360,32 @@ def run_cuda(args, wl):
     n_slots_comp = int((masks[cur] != 0).sum().item())
     value = aggregate_throughput(full_flops(wl) / 1e12, ms_per_step / 1e3, world)
 
+    # ---- end to end through the C ABI with host buffers (pinned): H2D of q, k, v, mask; D2H of out, lse
+    e2e = None
+    if not args.no_e2e:
+        cfg = ctx.cfg
+        ws = torch.empty(binding.dt_step_host_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+        qh, kh, vh = (x.cpu().pin_memory() for x in steps_in[1 % wl.steps])
+        oh = torch.empty(out.shape, dtype=in_dt).pin_memory()
+        lh = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+        mh = masks[cur].cpu()
+        times = []
+        for i in range(1 + 3):
+            if world > 1:
+                import torch.distributed as dist
+                dist.barrier()           # every replica runs its end-to-end step at the same time
+            t0 = time.perf_counter()
+            ctx.dt_step_host(qh, kh, vh, mh, t, oh, lh, ws)
+            times.append(time.perf_counter() - t0)
+            t += 1
+        e2e_s = max_over_ranks(float(np.mean(times[1:])), world, dev)
+        h2d = 3 * qh.numel() * 2 + PP
+        d2h = oh.numel() * 2 + lh.numel() * 4
+        e2e = {"value": aggregate_throughput(full_flops(wl) / 1e12, e2e_s, world), "unit": UNIT, "ms_per_step": 1e3 * e2e_s,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "includes": "dt_step_host: H2D q,k,v,mask + dt_attn_states + dt_state_merge + D2H out,lse"}
+        del ws
+
     if rank != 0:
         return
 
@@ -391,32 +417,9 @@ def run_cuda(args, wl):
             dense_ms.append(a.elapsed_time(b))
     dense_ms = float(np.mean(dense_ms))
 
-    # ---- end to end through the C ABI with host buffers (pinned): H2D of q, k, v, mask; D2H of out, lse
-    e2e = None
-    if not args.no_e2e:
-        cfg = ctx.cfg
-        ws = torch.empty(binding.dt_step_host_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
-        qh, kh, vh = (x.cpu().pin_memory() for x in steps_in[1 % wl.steps])
-        oh = torch.empty(out.shape, dtype=in_dt).pin_memory()
-        lh = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
-        mh = masks[cur].cpu()
-        times = []
-        for i in range(1 + 3):
-            t0 = time.perf_counter()
-            ctx.dt_step_host(qh, kh, vh, mh, t, oh, lh, ws)
-            times.append(time.perf_counter() - t0)
-            t += 1
-        e2e_s = float(np.mean(times[1:]))
-        h2d = 3 * qh.numel() * 2 + PP
-        d2h = oh.numel() * 2 + lh.numel() * 4
-        e2e = {"value": full_flops(wl) / 1e12 / e2e_s, "unit": UNIT, "ms_per_step": 1e3 * e2e_s,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "includes": "dt_step_host: H2D q,k,v,mask + dt_attn_states + dt_state_merge + D2H out,lse"}
-        del ws
-
     # ---- CPU oracle on a bounded sample of the same workload
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:
         eff, secs, desc, cores = oracle_sample(wl, *steps_in[1 % wl.steps], mask_np, budget_s=15.0, fp16=args.dtype == "fp16")
         cpu = {"value": eff, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds": secs}
 
