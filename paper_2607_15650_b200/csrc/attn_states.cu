@@ -15,11 +15,18 @@
 //   warp 10          K/V watcher: adds its arrival to p_full[0] once V_t and K_{t+1} have landed
 //   warp 11          idle (completes the producer warpgroup for the register hand-over)
 // TMEM (512 columns): S0 | S1 | O0 | O1.  S_t = Q K_t^T (fp32) lands in S; the softmax warpgroup
-// reads its row, writes P = exp2(s*scale*log2e - m) back over S as packed bf16, and the PV MMA
-// takes P from TMEM as its A operand and V from shared memory (MN-major) as B, accumulating in O.
-// While one query tile is in softmax the tensor core works on the other (ping-pong).
-// The running maximum is only moved (and O, l rescaled) when it grew by more than 2^8: stale
-// maxima cancel exactly in OUT = O / l and LSE = m + log l.
+// reads its row, writes P = exp2(s*scale*log2e - m) back over S as packed bf16 (fp16 for fp16 inputs),
+// and the PV MMA takes P from TMEM as its A operand and V from shared memory (MN-major) as B,
+// accumulating in O.  While one query tile is in softmax the tensor core works on the other
+// (ping-pong).  With D = 64 there is room for S0 | S1 | P0 | P1 | O0 | O1: P has columns of its own and
+// the next tile's Q K^T is issued as soon as the softmax has read S (see Cfg::PREFETCH).
+// P is computed against the reference maximum of the earlier tiles; only when a row sum of P reaches
+// ROWSUM_TRIGGER is the tile's own maximum taken and, if it lies more than 2^RESCALE_THRESHOLD above the
+// reference, the reference moved and O, l rescaled: stale references cancel exactly in OUT = O / l and
+// LSE = m + log l.
+// Epilogue: a query tile that lies wholly inside its partition leaves through shared memory as tiled
+// bulk stores; the fused mode (dt_attn_fused) composes the fresh state with the composed reuse state in
+// registers and stores the attention output itself.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA records STATUS_WAIT_TIMEOUT, leaves
 // its loops, frees TMEM and returns.
