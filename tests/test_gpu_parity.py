@@ -517,3 +517,49 @@ def test_algorithm1_planner_over_denoising_steps():
             selective += 1
             assert 0 < got_mask.sum() < P * P
     assert anchors >= 2 and selective >= 1
+
+
+@pytest.mark.parametrize("D,fp16", [(128, False), (64, False), (128, True)])
+def test_growing_logits_move_the_reference_maximum(D, fp16):
+    """Logits that grow along the key axis by far more than the rescale threshold (and by more than fp32's exponent
+    range in total), plus rows whose largest logit sits in the first tile: the stale-reference softmax has to move
+    its reference (and rescale O and l) again and again, and must never overflow."""
+    B, H, L, P = 1, 2, 1100, 2
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(17)
+    dt = torch.float16 if fp16 else torch.bfloat16
+    q = rng.standard_normal((B, L, H, D)).astype(np.float32)
+    k = rng.standard_normal((B, L, H, D)).astype(np.float32) * 0.1
+    v = rng.standard_normal((B, L, H, D)).astype(np.float32)
+    ramp = np.linspace(0.0, 1.0, L, dtype=np.float32)
+    # head 0: k aligned with a fixed direction u with a coefficient that rises along the keys; q rows aligned with +u
+    # (logits rise to about +300 in natural units at the last key) or -u (largest logit at the first key)
+    u = np.zeros(D, np.float32); u[:8] = 1.0 / np.sqrt(8.0)
+    k[0, :, 0, :] += np.outer(ramp * 30.0, u)
+    sign = np.where(np.arange(L) % 3 == 0, -1.0, 1.0).astype(np.float32)
+    q[0, :, 0, :] = np.outer(sign * 10.0, u) + 0.1 * q[0, :, 0, :]
+    qt, kt, vt = (torch.from_numpy(x).to(dt).to(dev) for x in (q, k, v))
+    scale = 1.0
+    off = np.array([0, 500, L], dtype=np.int32)
+    ctx = binding.Context(B, H, D, L, off, scale, input_dtype=binding.DT_INPUT_FP16 if fp16 else binding.DT_INPUT_BF16)
+    out = torch.empty((B, L, H, D), dtype=dt, device=dev)
+    lse = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+    ctx.dt_attn_states(qt, kt, vt, torch.ones(P * P, dtype=torch.uint8, device=dev), 0)
+    ctx.dt_state_merge(out, lse)
+    torch.cuda.synchronize()
+    ctx.dt_poll()
+    qb, kb, vb = (inputs.bf16_bits(x) for x in (qt, kt, vt))
+    rows = np.arange(L, dtype=np.int32)
+    lse_max = -np.inf
+    for h in range(H):
+        ro, rl = orc.full_attention(qb, kb, vb, scale, 0, h, rows, fp16=fp16)
+        lse_max = max(lse_max, rl.max())
+        assert np.isfinite(lse[0, h].cpu().numpy()).all() and torch.isfinite(out[0, :, h].float()).all()
+        check_o(out[0, :, h].float().cpu().numpy(), ro, f"growing logits head {h}")
+        # LSE values reach a few hundred here: the absolute tolerance is kept, relative to that it is 1e-5
+        check_lse(lse[0, h].cpu().numpy(), rl, f"growing logits head {h}")
+        for j in range(P):
+            so, sl = orc.pair_state(qb, kb, vb, scale, 0, h, rows, int(off[j]), int(off[j + 1]), fp16=fp16)
+            check_o(ctx.o_state[j, 0, h].float().cpu().numpy(), so, f"growing logits state {j}")
+            check_lse(ctx.lse_state[j, 0, h].cpu().numpy(), sl, f"growing logits state {j}")
+    assert lse_max > 150.0      # the case really is extreme
