@@ -69,6 +69,8 @@ def test_random_configuration(seed):
     if g > 1 and seed % 2 == 0 and run.S - 1 >= 2:
         run.ctx.dt_group_compose()
         run.ses.compose()
+        if state_dtype == binding.DT_STATE_BF16:
+            run.tol_scale = 2.0          # composed states have been rounded to bf16 twice
         run.check_layout()
         torch.cuda.synchronize()
         run.check_states("after compose")

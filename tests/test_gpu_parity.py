@@ -19,10 +19,12 @@ def _built():
     binding.lib()
 
 
-def check_o(got, ref, what=""):
+def check_o(got, ref, what="", scale=1.0):
+    """scale > 1 only where a bf16 state cache has been composed in place: every composition rounds the state to
+    bf16 once more (relative 2^-9 of values up to about 4), on top of the rounding of the stored states."""
     err = np.abs(np.asarray(got, dtype=np.float64) - ref)
-    assert err.max() <= O_MAX, f"{what}: O max abs err {err.max():.3e}"
-    assert err.mean() <= O_MEAN, f"{what}: O mean abs err {err.mean():.3e}"
+    assert err.max() <= scale * O_MAX, f"{what}: O max abs err {err.max():.3e}"
+    assert err.mean() <= scale * O_MEAN, f"{what}: O mean abs err {err.mean():.3e}"
 
 
 def check_lse(got, ref, what=""):
