@@ -21,6 +21,10 @@
  *   - Every function returns a dt_status.  Argument errors are detected before any launch.
  *     Conditions only the device can see (REUSE of a never-computed pair, a bounded wait
  *     that ran out) are recorded in a device status word that dt_poll reads.
+ *   - A context is not thread-safe: issue the calls on one context from one thread at a time.  Its device
+ *     scratch (work list, tile table, partial sums, selection bits) is shared by its calls, so calls on one
+ *     context must also be ordered on the device -- use one stream per context, or order streams with events.
+ *     Different contexts are independent.
  *   - Natural logarithm everywhere an LSE crosses this boundary.
  *   - Limits: D in {64, 128}; 1 <= P <= 32; bf16 or fp16 inputs ("bf16" below stands for the configured
  *     input type); innermost stride 1.
