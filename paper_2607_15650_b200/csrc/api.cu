@@ -122,29 +122,6 @@ dt_status encode_qkv_map(dt_ctx *ctx, CUtensorMap *tm, const void *base, const i
     return DT_OK;
 }
 
-// State cache viewed as a 2-D tensor map (d, slot*b*h*l row) for the attention epilogue's tiled stores:
-// box = 128 bytes of a row x 128 rows, 128-byte swizzle.
-dt_status encode_state_map(dt_ctx *ctx, CUtensorMap *tm) {
-    const dt_config &c = ctx->cfg;
-    const bool f32 = c.state_dtype == DT_STATE_FP32;
-    const size_t esz = f32 ? 4 : 2;
-    cuuint64_t dims[2] = {(cuuint64_t)c.D, (cuuint64_t)ctx->S0 * c.B * c.H * c.L};
-    cuuint64_t strides[1] = {(cuuint64_t)c.D * esz};
-    cuuint32_t box[2] = {(cuuint32_t)(128 / esz), (cuuint32_t)dt::ATTN_TILE};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
-        tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->o_state, dims, strides, box, estr,
-        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        char buf[96];
-        snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled (state cache) failed with CUresult %d", (int)r);
-        ctx->err = buf;
-        return DT_ERR_CUDA;
-    }
-    return DT_OK;
-}
-
 }  // namespace
 
 extern "C" {
@@ -285,12 +262,11 @@ dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const v
         dt_status s = check_strides(strides_blhd, t, &why);
         if (s != DT_OK) return fail(ctx, s, why);
     }
-    CUtensorMap tq, tk, tv, ts;
+    CUtensorMap tq, tk, tv;
     dt_status s;
     if ((s = encode_qkv_map(ctx, &tq, q_dev, strides_blhd)) != DT_OK) return s;
     if ((s = encode_qkv_map(ctx, &tk, k_dev, strides_blhd)) != DT_OK) return s;
     if ((s = encode_qkv_map(ctx, &tv, v_dev, strides_blhd)) != DT_OK) return s;
-    if ((s = encode_state_map(ctx, &ts)) != DT_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dt_config &c = ctx->cfg;
     cudaError_t e = dt::launch_worklist(mask_dev, ctx->tc_dev, ctx->worklist_dev, ctx->status_dev, ctx->slot_tab_dev, c.P,
@@ -308,7 +284,7 @@ dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const v
     p.in_fp16 = c.input_dtype == DT_INPUT_FP16;
     p.qblocks_max = ctx->qblocks_max;
     p.scale_log2 = c.softmax_scale * 1.44269504088896340736f;
-    e = dt::launch_attn_states(tq, tk, tv, ts, p, c.D, c.state_dtype, ctx->num_sms, st);
+    e = dt::launch_attn_states(tq, tk, tv, p, c.D, c.state_dtype, ctx->num_sms, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "attention launch");
     ctx->launches += 2;
     return DT_OK;

@@ -24,8 +24,8 @@
 // ROWSUM_TRIGGER is the tile's own maximum taken and, if it lies more than 2^RESCALE_THRESHOLD above the
 // reference, the reference moved and O, l rescaled: stale references cancel exactly in OUT = O / l and
 // LSE = m + log l.
-// Epilogue: a query tile that lies wholly inside its partition leaves through shared memory as tiled
-// bulk stores; the fused mode (dt_attn_fused) composes the fresh state with the composed reuse state in
+// Epilogue: the rows leave through warp-private shared-memory tiles so that the cache is written in whole
+// 128-byte lines; the fused mode (dt_attn_fused) composes the fresh state with the composed reuse state in
 // registers and stores the attention output itself.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA records STATUS_WAIT_TIMEOUT, leaves
@@ -68,7 +68,7 @@ struct Cfg {
     static constexpr int STAGES = (D == 128) ? 4 : 8;         // K/V ring depth
     static constexpr int Q_BYTES = ATTN_NQ * TILE_BYTES;
     static constexpr int KV_BYTES = STAGES * TILE_BYTES;
-    static constexpr int OUT_STAGE_BYTES = ATTN_TILE * 128;   // epilogue staging per query tile: 128 rows x 128 bytes
+    static constexpr int OUT_STAGE_BYTES = ATTN_TILE * 128;   // epilogue staging per query tile: 4 warps x [32 rows x 128 bytes]
     static constexpr int OUT_BYTES = ATTN_NQ * OUT_STAGE_BYTES;
     static constexpr int NBARS = 2 + 2 * STAGES + 5 * ATTN_NQ;
     static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + Q_BYTES + KV_BYTES + OUT_BYTES + NBARS * 8 + 64;
@@ -152,31 +152,6 @@ __device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, lon
     return it.n_q > 0;
 }
 
-template <typename StateT>
-__device__ __forceinline__ void store_state_chunk(StateT *dst, const uint32_t (&r)[32], float inv_l);
-
-template <>
-__device__ __forceinline__ void store_state_chunk<float>(float *dst, const uint32_t (&r)[32], float inv_l) {
-#pragma unroll
-    for (int c = 0; c < 32; c += 4) {
-        float4 v = make_float4(__uint_as_float(r[c]) * inv_l, __uint_as_float(r[c + 1]) * inv_l,
-                               __uint_as_float(r[c + 2]) * inv_l, __uint_as_float(r[c + 3]) * inv_l);
-        __stcs(reinterpret_cast<float4 *>(dst + c), v);
-    }
-}
-template <>
-__device__ __forceinline__ void store_state_chunk<__nv_bfloat16>(__nv_bfloat16 *dst, const uint32_t (&r)[32], float inv_l) {
-#pragma unroll
-    for (int c = 0; c < 32; c += 8) {
-        uint4 v;
-        v.x = pack_bf16x2(__uint_as_float(r[c]) * inv_l, __uint_as_float(r[c + 1]) * inv_l);
-        v.y = pack_bf16x2(__uint_as_float(r[c + 2]) * inv_l, __uint_as_float(r[c + 3]) * inv_l);
-        v.z = pack_bf16x2(__uint_as_float(r[c + 4]) * inv_l, __uint_as_float(r[c + 5]) * inv_l);
-        v.w = pack_bf16x2(__uint_as_float(r[c + 6]) * inv_l, __uint_as_float(r[c + 7]) * inv_l);
-        __stcs(reinterpret_cast<uint4 *>(dst + c), v);
-    }
-}
-
 // 32 consecutive elements of a cached state row as fp32
 __device__ __forceinline__ void load_state_chunk(const float *src, float (&v)[32]) {
 #pragma unroll
@@ -201,8 +176,7 @@ __device__ __forceinline__ void load_state_chunk(const __nv_bfloat16 *src, float
 template <int D, typename StateT, bool FUSED, bool FP16>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                   const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_state,
-                   const AttnParams p) {
+                   const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_slot;
@@ -696,64 +670,57 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 if (row_valid && p.lse_out != nullptr) p.lse_out[crow] = lse_row;
             } else {
                 const long long srow = ((long long)it.slot * p.B * p.H + it.bh) * p.L + it.q_row0 + row_in_block;
-                if (it.n_q >= (q + 1) * ATTN_TILE) {
-                    // Whole query tile inside the partition: rows go through shared memory (128 bytes of every row
-                    // at a time, 128-byte swizzle) and leave as one tiled bulk store per chunk -- whole lines instead
-                    // of 16 bytes per lane at a 512-byte stride.
-                    constexpr int CH = 128 / (int)sizeof(StateT);          // state elements per 128-byte chunk
-                    const uint32_t stage = out_smem + q * C::OUT_STAGE_BYTES;
-                    const uint32_t my_row = stage + row_in_tile * 128;
-                    const bool issuer = ((warp % 4) == 0 && lane == 0);
+                // Rows leave through shared memory, warp by warp: each thread writes 128 bytes of its row (swizzled,
+                // so the 32 lanes hit different banks), then the warp reads the 4 KB back so that 8 lanes hold the
+                // 128 contiguous bytes of one row and stores them -- whole lines to the cache instead of 16 bytes per
+                // lane at a 512-byte stride.  The staging area is private to the warp: only __syncwarp() is needed,
+                // and no store has to be waited for.  Rows beyond the partition are skipped row by row.
+                constexpr int CH = 128 / (int)sizeof(StateT);          // state elements per 128-byte chunk
+                const uint32_t stage = out_smem + warp * 4096;          // [32 rows][128 bytes]
+                const uint32_t my_row = stage + lane * 128;
+                const int rows_left = it.n_q - (row_in_block - lane);   // valid rows of this warp's 32
+                uint8_t *gbase = reinterpret_cast<uint8_t *>(o_state + (srow - lane) * D);   // row 0 of this warp
 #pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += CH) {
-                        uint32_t o[CH / 32][32];
+                for (int c0 = 0; c0 < D; c0 += CH) {
+                    uint32_t o[CH / 32][32];
 #pragma unroll
-                        for (int u = 0; u < CH / 32; ++u) tmem_ld_x32(o_tmem + c0 + 32 * u, o[u]);
-                        tmem_wait_ld();
-                        if (c0 + CH >= D) {  // O[q] fully read: the next item's first PV may overwrite it
-                            tc_fence_before();
-                            mbar_arrive(bars.o_free + 8 * q);
-                        }
-                        if (issuer) bulk_wait_group_read0();   // the previous chunk's store has read the staging tile
-                        named_bar_sync(1 + q, 128);
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {   // 16-byte piece c of this row's 128 bytes
-                            uint4 v;
-                            if constexpr (sizeof(StateT) == 4) {
-                                v.x = __float_as_uint(__uint_as_float(o[0][4 * c]) * inv_l);
-                                v.y = __float_as_uint(__uint_as_float(o[0][4 * c + 1]) * inv_l);
-                                v.z = __float_as_uint(__uint_as_float(o[0][4 * c + 2]) * inv_l);
-                                v.w = __float_as_uint(__uint_as_float(o[0][4 * c + 3]) * inv_l);
-                            } else {
-                                const uint32_t(&oo)[32] = o[(8 * c) / 32];
-                                const int b0 = (8 * c) % 32;
-                                v.x = pack_bf16x2(__uint_as_float(oo[b0]) * inv_l, __uint_as_float(oo[b0 + 1]) * inv_l);
-                                v.y = pack_bf16x2(__uint_as_float(oo[b0 + 2]) * inv_l, __uint_as_float(oo[b0 + 3]) * inv_l);
-                                v.z = pack_bf16x2(__uint_as_float(oo[b0 + 4]) * inv_l, __uint_as_float(oo[b0 + 5]) * inv_l);
-                                v.w = pack_bf16x2(__uint_as_float(oo[b0 + 6]) * inv_l, __uint_as_float(oo[b0 + 7]) * inv_l);
-                            }
-                            const uint32_t dst = my_row + (uint32_t)((c ^ (row_in_tile & 7)) << 4);
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-                        }
-                        fence_proxy_async_smem();
-                        named_bar_sync(1 + q, 128);
-                        if (issuer) {
-                            tma_store_2d(&tmap_state, stage, c0, (int)(srow - row_in_tile));
-                            bulk_commit_group();
-                        }
+                    for (int u = 0; u < CH / 32; ++u) tmem_ld_x32(o_tmem + c0 + 32 * u, o[u]);
+                    tmem_wait_ld();
+                    if (c0 + CH >= D) {  // O[q] fully read: the next item's first PV may overwrite it
+                        tc_fence_before();
+                        mbar_arrive(bars.o_free + 8 * q);
                     }
-                } else {
 #pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += 32) {
-                        uint32_t o[32];
-                        tmem_ld_x32(o_tmem + c0, o);
-                        tmem_wait_ld();
-                        if (c0 + 32 >= D) {  // O[q] fully read: the next item's first PV may overwrite it
-                            tc_fence_before();
-                            mbar_arrive(bars.o_free + 8 * q);
+                    for (int c = 0; c < 8; ++c) {   // 16-byte piece c of this row's 128 bytes
+                        uint4 v;
+                        if constexpr (sizeof(StateT) == 4) {
+                            v.x = __float_as_uint(__uint_as_float(o[0][4 * c]) * inv_l);
+                            v.y = __float_as_uint(__uint_as_float(o[0][4 * c + 1]) * inv_l);
+                            v.z = __float_as_uint(__uint_as_float(o[0][4 * c + 2]) * inv_l);
+                            v.w = __float_as_uint(__uint_as_float(o[0][4 * c + 3]) * inv_l);
+                        } else {
+                            const uint32_t(&oo)[32] = o[(8 * c) / 32];
+                            const int b0 = (8 * c) % 32;
+                            v.x = pack_bf16x2(__uint_as_float(oo[b0]) * inv_l, __uint_as_float(oo[b0 + 1]) * inv_l);
+                            v.y = pack_bf16x2(__uint_as_float(oo[b0 + 2]) * inv_l, __uint_as_float(oo[b0 + 3]) * inv_l);
+                            v.z = pack_bf16x2(__uint_as_float(oo[b0 + 4]) * inv_l, __uint_as_float(oo[b0 + 5]) * inv_l);
+                            v.w = pack_bf16x2(__uint_as_float(oo[b0 + 6]) * inv_l, __uint_as_float(oo[b0 + 7]) * inv_l);
                         }
-                        if (row_valid) store_state_chunk<StateT>(o_state + srow * D + c0, o, inv_l);
+                        const uint32_t dst = my_row + (uint32_t)((c ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
                     }
+                    __syncwarp();
+                    const int piece = lane & 7;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {   // 4 rows per pass: lane -> (row, 16-byte piece)
+                        const int r = i * 4 + (lane >> 3);
+                        uint4 v;
+                        const uint32_t src = stage + r * 128 + (uint32_t)((piece ^ (r & 7)) << 4);
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(src) : "memory");
+                        if (r < rows_left)
+                            __stcs(reinterpret_cast<uint4 *>(gbase + (size_t)r * D * sizeof(StateT) + (size_t)c0 * sizeof(StateT) + piece * 16), v);
+                    }
+                    __syncwarp();
                 }
                 if (row_valid) p.lse_state[srow] = lse_fresh;
             }
@@ -762,7 +729,6 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             if (!*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
             *abort_ptr = 1;
         }
-        if ((warp % 4) == 0 && lane == 0) bulk_wait_group0();   // this thread's state stores have left shared memory
     }
 
     tc_fence_before();
@@ -772,17 +738,17 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 }
 
 template <int D, typename StateT, bool FUSED, bool FP16>
-cudaError_t launch_one(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
-                       const AttnParams &p, int num_ctas, cudaStream_t stream) {
-    attn_states_kernel<D, StateT, FUSED, FP16><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, ts, p);
+cudaError_t launch_one(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const AttnParams &p,
+                       int num_ctas, cudaStream_t stream) {
+    attn_states_kernel<D, StateT, FUSED, FP16><<<num_ctas, ATTN_THREADS, Cfg<D>::SMEM_BYTES, stream>>>(tq, tk, tv, p);
     return cudaGetLastError();
 }
 
 template <int D, typename StateT, bool FUSED>
-cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
-                   const AttnParams &p, int num_ctas, cudaStream_t stream) {
-    return p.in_fp16 ? launch_one<D, StateT, FUSED, true>(tq, tk, tv, ts, p, num_ctas, stream)
-                     : launch_one<D, StateT, FUSED, false>(tq, tk, tv, ts, p, num_ctas, stream);
+cudaError_t launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const AttnParams &p,
+                   int num_ctas, cudaStream_t stream) {
+    return p.in_fp16 ? launch_one<D, StateT, FUSED, true>(tq, tk, tv, p, num_ctas, stream)
+                     : launch_one<D, StateT, FUSED, false>(tq, tk, tv, p, num_ctas, stream);
 }
 
 template <int D, typename StateT, bool FUSED, bool FP16>
@@ -845,25 +811,24 @@ cudaError_t attn_states_configure() {
     return configure<128, __nv_bfloat16>();
 }
 
-cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
+cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                                const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream) {
     if (state_dtype == DT_STATE_FP32) {
-        return D == 64 ? launch<64, float, false>(tq, tk, tv, ts, p, num_ctas, stream)
-                       : launch<128, float, false>(tq, tk, tv, ts, p, num_ctas, stream);
+        return D == 64 ? launch<64, float, false>(tq, tk, tv, p, num_ctas, stream)
+                       : launch<128, float, false>(tq, tk, tv, p, num_ctas, stream);
     }
-    return D == 64 ? launch<64, __nv_bfloat16, false>(tq, tk, tv, ts, p, num_ctas, stream)
-                   : launch<128, __nv_bfloat16, false>(tq, tk, tv, ts, p, num_ctas, stream);
+    return D == 64 ? launch<64, __nv_bfloat16, false>(tq, tk, tv, p, num_ctas, stream)
+                   : launch<128, __nv_bfloat16, false>(tq, tk, tv, p, num_ctas, stream);
 }
 
 cudaError_t launch_attn_fused(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                               const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream) {
-    // the fused epilogue stores the attention output itself: the state map is not used (any valid map will do)
     if (state_dtype == DT_STATE_FP32) {
-        return D == 64 ? launch<64, float, true>(tq, tk, tv, tq, p, num_ctas, stream)
-                       : launch<128, float, true>(tq, tk, tv, tq, p, num_ctas, stream);
+        return D == 64 ? launch<64, float, true>(tq, tk, tv, p, num_ctas, stream)
+                       : launch<128, float, true>(tq, tk, tv, p, num_ctas, stream);
     }
-    return D == 64 ? launch<64, __nv_bfloat16, true>(tq, tk, tv, tq, p, num_ctas, stream)
-                   : launch<128, __nv_bfloat16, true>(tq, tk, tv, tq, p, num_ctas, stream);
+    return D == 64 ? launch<64, __nv_bfloat16, true>(tq, tk, tv, p, num_ctas, stream)
+                   : launch<128, __nv_bfloat16, true>(tq, tk, tv, p, num_ctas, stream);
 }
 
 cudaError_t launch_fused_tiles(const uint8_t *mask, const SlotRange *slot_tab, int P, int S, int max_tiles, int2 *tile_tab,

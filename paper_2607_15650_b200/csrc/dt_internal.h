@@ -147,7 +147,7 @@ cudaError_t launch_planner_commit(const PlannerParams &p, int state_dtype, cudaS
 
 cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, const SlotRange *slot_tab,
                             int P, int S, int group_mode, int step, cudaStream_t stream);
-cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &ts,
+cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                                const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream);
 cudaError_t launch_attn_fused(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                               const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream);

@@ -73,19 +73,6 @@ __device__ __forceinline__ void tma_load_4d(uint32_t smem_dst, const CUtensorMap
         : "memory");
 }
 
-// 2-D tiled store shared -> global (bulk async-group completion).  The innermost coordinate times the element
-// size must be a multiple of 16 bytes; the shared-memory tile is laid out as the tensor map's swizzle says.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *tm, uint32_t smem_src, int c0, int c1) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(smem_src), "r"(c0), "r"(c1)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// all earlier bulk groups of this thread have finished READING their shared-memory source
-__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-// all earlier bulk groups of this thread are complete
-__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
 // Untiled bulk copy global -> shared (both addresses 16-byte aligned, size a multiple of 16 bytes),
 // completion counted in bytes on an mbarrier.
 __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void *gmem_src, uint32_t bytes, uint32_t bar) {
