@@ -10,12 +10,16 @@ region an anchor step computes every pair and the first plan is derived from it.
 Q, K, V of every denoising step of the workload) are resident in HBM; they and the state cache
 are far larger than L2, so no explicit flush is needed.
 
+With N > 1 ranks each runs an independent replica of the layer (no collective); `--shard-heads` instead
+spreads the heads of one layer over the ranks, with one all-reduce of the plan's P x S sums per step.
+
 Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead, on a
 bounded sample of the same workload.
 """
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -241,11 +245,15 @@ def run_reference(args, wl):
 
 # ------------------------------------------------------------------------------------------ CUDA arm
 def run_cuda(args, wl):
-    from paper_2607_15650_b200 import binding, build
+    from paper_2607_15650_b200 import binding, build, sharding
     world, rank, local = dist_info()
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl_total = wl
+    if args.shard_heads:     # one layer over all ranks: this rank keeps a contiguous share of the heads
+        h0, h1 = sharding.head_range(wl.H, world, rank)
+        wl = dataclasses.replace(wl, H=h1 - h0)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     build.build()
@@ -259,7 +267,7 @@ def run_cuda(args, wl):
     ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale, state_dtype, local, group_size=args.group_size,
                           input_dtype=binding.DT_INPUT_FP16 if args.dtype == "fp16" else binding.DT_INPUT_BF16)
     S, g = ctx.dt_num_slots()
-    gen = inputs.StepInputs(wl, seed=0, device=dev, dtype=in_dt)
+    gen = inputs.StepInputs(wl, seed=rank if args.shard_heads else 0, device=dev, dtype=in_dt)
     steps_in = [gen.next() for _ in range(wl.steps)]          # resident bf16 inputs of every denoising step
     del gen
     torch.cuda.empty_cache()
@@ -269,8 +277,15 @@ def run_cuda(args, wl):
     masks = [torch.ones(PP, dtype=torch.uint8, device=dev), torch.ones(PP, dtype=torch.uint8, device=dev)]
     ones = torch.ones(PP, dtype=torch.uint8, device=dev)
     W = torch.empty(PP, dtype=torch.float64, device=dev)
+    sums = torch.empty(PP, dtype=torch.float64, device=dev)
     frac = args.fraction if args.fraction is not None else wl.fractions[-1]
     stream = torch.cuda.current_stream()
+
+    def plan(mask_buf):
+        if args.shard_heads:   # local sums -> all-reduce of P*S doubles -> the same plan on every rank
+            sharding.plan_sharded(ctx, wl_total.B * wl_total.H, mask_buf, sums, target_fraction=frac, w_dev=W)
+        else:
+            ctx.dt_plan(mask_buf, target_fraction=frac, w_dev=W)
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
@@ -297,7 +312,7 @@ def run_cuda(args, wl):
             ctx.dt_state_merge(out, lse)
         if timers is not None:
             e[2].record(stream)
-        ctx.dt_plan(masks[cur ^ 1], target_fraction=frac, w_dev=W)
+        plan(masks[cur ^ 1])
         if timers is not None:
             e[3].record(stream)
             timers.append(e)
@@ -307,7 +322,7 @@ def run_cuda(args, wl):
     q, k, v = steps_in[0]
     ctx.dt_attn_states(q, k, v, ones, 0)
     ctx.dt_state_merge(out, lse)
-    ctx.dt_plan(masks[0], target_fraction=frac, w_dev=W)
+    plan(masks[0])
     comp_o = comp_l = None
     compose_ms = None
     if args.composed or args.fused:
@@ -358,7 +373,12 @@ def run_cuda(args, wl):
     comp_fl = computed_flops(wl, mask_np)           # pair count is fixed by the target fraction
     n_comp = int((mask_np != 0).sum())
     n_slots_comp = int((masks[cur] != 0).sum().item())
-    value = aggregate_throughput(full_flops(wl) / 1e12, ms_per_step / 1e3, world)
+    def job_throughput(seconds):   # whole job: N replicas of the layer, or one layer whose heads the ranks share
+        if args.shard_heads:
+            return full_flops(wl_total) / 1e12 / seconds
+        return aggregate_throughput(full_flops(wl) / 1e12, seconds, world)
+
+    value = job_throughput(ms_per_step / 1e3)
 
     # ---- end to end through the C ABI with host buffers (pinned): H2D of q, k, v, mask; D2H of out, lse
     e2e = None
@@ -381,7 +401,7 @@ def run_cuda(args, wl):
         e2e_s = max_over_ranks(float(np.mean(times[1:])), world, dev)
         h2d = 3 * qh.numel() * 2 + PP
         d2h = oh.numel() * 2 + lh.numel() * 4
-        e2e = {"value": aggregate_throughput(full_flops(wl) / 1e12, e2e_s, world), "unit": UNIT, "ms_per_step": 1e3 * e2e_s,
+        e2e = {"value": job_throughput(e2e_s), "unit": UNIT, "ms_per_step": 1e3 * e2e_s,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "includes": "dt_step_host: H2D q,k,v,mask + dt_attn_states + dt_state_merge + D2H out,lse"}
         del ws
@@ -428,15 +448,17 @@ def run_cuda(args, wl):
     peak = peaks["bf16_tflops_sustained"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if args.shard_heads else "weak",
+        "vs_baseline": None,
         "dtype": args.dtype, "data": "synthetic",
-        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "D": wl.D, "L": wl.L, "P": wl.P,
+        "config": {"workload": wl.name, "B": wl.B, "H": wl_total.H, "heads_per_rank": wl.H, "D": wl.D, "L": wl.L, "P": wl.P,
                    "computed_pairs": n_comp, "computed_pair_fraction": n_comp / (wl.P * wl.P),
                    "group_size": g, "cache_slots": S, "computed_slots": n_slots_comp, "state_dtype": args.state_dtype,
                    "cache_gb": S * wl.B * wl.H * wl.L * (wl.D * sbytes + 4) / 1e9,
                    "step": ("dt_attn_fused (COMPUTE slots in one pass + composed reuse state in the epilogue)" if args.fused
                             else "dt_attn_states + dt_state_merge_planned + dt_plan" if args.composed
-                            else "dt_attn_states + dt_state_merge + dt_plan"), "multi_gpu": "independent replicas",
+                            else "dt_attn_states + dt_state_merge + dt_plan"), "multi_gpu": ("heads sharded over the ranks; one all-reduce of P*S plan sums per step" if args.shard_heads
+                                  else "independent replicas"),
                    "l2": "inputs (%.1f GB) and state cache larger than L2; no flush" %
                          ((3 * wl.L * wl.H * wl.D * 2) / 1e9)},
         "clocks": clocks,
@@ -489,13 +511,15 @@ def main():
                          "composed reuse state in the epilogue; no state-cache round trip, the plan stays fixed)")
     ap.add_argument("--group-size", type=int, default=1,
                     help="g >= 2: grouped state cache (ceil(P/g) + 1 slots per row; group states computed in one pass)")
+    ap.add_argument("--shard-heads", action="store_true",
+                    help="N > 1: the ranks share the heads of ONE layer (strong scaling; the plan's sums are all-reduced) "
+                         "instead of running N independent replicas")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     wl = inputs.WORKLOADS[args.workload]
     if args.heads is not None:
-        import dataclasses
         wl = dataclasses.replace(wl, H=args.heads, name=f"{wl.name}_h{args.heads}")
     if args.impl == "reference":
         run_reference(args, wl)

@@ -164,6 +164,23 @@ dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask
 dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32_t group_size, uint8_t *mask_dev,
                           double *w_dev, double *eps_out_dev, void *stream);
 
+/* Head-sharded planning.  The (batch, head) slices of a layer are independent in dt_attn_states and
+ * dt_state_merge, so the heads of one layer may be spread over several contexts (one per GPU) with no
+ * exchange there.  Only the plan needs one: W of Eq. 8 is a mean over all heads, and every shard must
+ * arrive at the same mask (Section 4.3: the compute / reuse strategy is the same on all devices).  The
+ * two halves of dt_plan, with the exchange left to the caller:
+ *   dt_plan_sums       sums_dev (device, double [P*S], written) = sum over this context's batch, heads and
+ *                      the rows of partition i of the per-row weights w (Eq. 8), not yet divided by a count
+ *   (caller)           adds the shards' sums element by element, e.g. one all-reduce of P*S doubles
+ *   dt_plan_from_sums  the plan as dt_plan / dt_plan_grouped would take it, from sums that cover total_bh
+ *                      (batch, head) slices: W[i][s] = sums[i][s] / (total_bh * n_i); then the threshold or
+ *                      the target fraction as there.  total_bh >= this context's B * H.
+ * With one shard (total_bh = B * H) the result is bit-identical to dt_plan_grouped.  Sums of different
+ * shards are added in whatever order the caller's reduction uses; W then agrees to rounding of doubles. */
+dt_status dt_plan_sums(dt_ctx *ctx, double *sums_dev, void *stream);
+dt_status dt_plan_from_sums(dt_ctx *ctx, const double *sums_dev, int64_t total_bh, double eps, double target_fraction,
+                            int32_t group_size, uint8_t *mask_dev, double *w_dev, double *eps_out_dev, void *stream);
+
 /* Anchor-guided selection planning, Algorithm 1 (Section 4), with its state on the device.
  *   partition importance  w(i,j)      Eq. 8, refreshed at anchors from the cached LSEs
  *   scale ratio           alpha(i,j)  Eq. 9: ||AS_ta(i,j)||_2 / ||AS_ta(i,i)||_2, the state being OUT and LSE

@@ -25,6 +25,7 @@ EXPORTS = [
     "dt_plan_static", "dt_step_host_workspace_bytes", "dt_step_host", "dt_get_tc", "dt_set_tc",
     "dt_launch_count", "dt_selftest_wait_timeout", "dt_poll", "dt_status_str", "dt_last_error",
     "dt_attn_fused", "dt_num_slots", "dt_slot_ranges", "dt_group_compose", "dt_group_fit", "dt_group_reset",
+    "dt_plan_sums", "dt_plan_from_sums",
 ]
 
 
@@ -73,6 +74,8 @@ def lib():
         "dt_state_merge_planned": (C.c_int, [vp, u8p, vp, f32p, vp, i64p, f32p, vp]),
         "dt_plan": (C.c_int, [vp, C.c_double, C.c_double, u8p, f64p, f64p, vp]),
         "dt_plan_grouped": (C.c_int, [vp, C.c_double, C.c_double, C.c_int32, u8p, f64p, f64p, vp]),
+        "dt_plan_sums": (C.c_int, [vp, f64p, vp]),
+        "dt_plan_from_sums": (C.c_int, [vp, f64p, C.c_int64, C.c_double, C.c_double, C.c_int32, u8p, f64p, f64p, vp]),
         "dt_planner_init": (C.c_int, [vp, C.POINTER(dt_planner_config), vp, f32p, C.c_size_t, C.c_size_t, vp]),
         "dt_planner_step": (C.c_int, [vp, u8p, vp, f64p, f64p, vp]),
         "dt_planner_commit": (C.c_int, [vp, vp]),
@@ -272,6 +275,20 @@ class Context:
         ep = C.c_void_p(eps_out_dev.data_ptr()) if eps_out_dev is not None else C.c_void_p()
         self._check(lib().dt_plan_grouped(self._h, float(eps), float(target_fraction), int(group_size),
                                           C.c_void_p(mask_dev.data_ptr()), wp, ep, _stream_ptr(stream)))
+
+    def dt_plan_sums(self, sums_dev, stream=None):
+        assert sums_dev.dtype == torch.float64 and sums_dev.is_cuda and sums_dev.is_contiguous()
+        self._check(lib().dt_plan_sums(self._h, C.c_void_p(sums_dev.data_ptr()), _stream_ptr(stream)))
+
+    def dt_plan_from_sums(self, sums_dev, total_bh, mask_dev, eps=0.0, target_fraction=-1.0, group_size=1, w_dev=None,
+                          eps_out_dev=None, stream=None):
+        assert sums_dev.dtype == torch.float64 and sums_dev.is_cuda and sums_dev.is_contiguous()
+        assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()
+        wp = C.c_void_p(w_dev.data_ptr()) if w_dev is not None else C.c_void_p()
+        ep = C.c_void_p(eps_out_dev.data_ptr()) if eps_out_dev is not None else C.c_void_p()
+        self._check(lib().dt_plan_from_sums(self._h, C.c_void_p(sums_dev.data_ptr()), int(total_bh), float(eps),
+                                            float(target_fraction), int(group_size), C.c_void_p(mask_dev.data_ptr()),
+                                            wp, ep, _stream_ptr(stream)))
 
     def dt_plan(self, mask_dev, eps=0.0, target_fraction=-1.0, w_dev=None, eps_out_dev=None, stream=None):
         assert mask_dev.dtype == torch.uint8 and mask_dev.is_cuda and mask_dev.is_contiguous()

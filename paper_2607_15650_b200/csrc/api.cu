@@ -460,13 +460,16 @@ dt_status dt_plan(dt_ctx *ctx, double eps, double target_fraction, uint8_t *mask
     return dt_plan_grouped(ctx, eps, target_fraction, 1, mask_dev, w_dev, eps_out_dev, stream);
 }
 
-dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32_t group_size, uint8_t *mask_dev,
-                          double *w_dev, double *eps_out_dev, void *stream) {
-    if (!ctx) return DT_ERR_INVALID_ARG;
+// The plan computation behind dt_plan, dt_plan_grouped and the two halves of a head-sharded plan:
+//   sums_out != null : stage 1 and the fixed-order sums of this context only, written to sums_out
+//   sums_in  != null : no stage 1; the plan from sums over `total_bh` (batch, head) slices
+static dt_status plan_impl(dt_ctx *ctx, double eps, double target_fraction, int32_t group_size, uint8_t *mask_dev,
+                           double *w_dev, double *eps_out_dev, void *stream, const double *sums_in, double *sums_out,
+                           long long total_bh) {
     if (group_size < 1 || group_size > ctx->cfg.P) return fail(ctx, DT_ERR_INVALID_ARG, "group_size must be in [1, P]");
     if (ctx->group_size0 > 1 && group_size != 1)
         return fail(ctx, DT_ERR_UNSUPPORTED, "a grouped cache decides per slot: group_size must be 1 here");
-    if (!mask_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null mask pointer");
+    if (!mask_dev && !sums_out) return fail(ctx, DT_ERR_INVALID_ARG, "null mask pointer");
     if (!ctx->lse_state) return fail(ctx, DT_ERR_STATE, "state cache not bound");
     if (target_fraction < 0 && !std::isfinite(eps)) return fail(ctx, DT_ERR_INVALID_ARG, "eps must be finite");
     if (target_fraction > 1.0 || std::isnan(target_fraction)) return fail(ctx, DT_ERR_INVALID_ARG, "target_fraction must be <= 1");
@@ -479,8 +482,12 @@ dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32
     pp.nonempty = ctx->group_size0 > 1 ? ctx->nonempty_dev : nullptr;
     pp.P = c.P; pp.S = ctx->S; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
     pp.R = (long long)c.B * c.H * c.L;
-    cudaError_t e = dt::launch_plan_partial(pp, st);
-    if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
+    cudaError_t e = cudaSuccess;
+    if (!sums_in) {
+        e = dt::launch_plan_partial(pp, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
+        ctx->launches += 1;
+    }
     if (ctx->group_size0 > 1) {
         dt::PlanSlotsParams ps;
         ps.partials = ctx->plan_partials_dev;
@@ -495,9 +502,10 @@ dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32
         ps.mask = mask_dev;
         ps.w_out = w_dev;
         ps.eps_out = eps_out_dev;
+        ps.sums_in = sums_in; ps.sums_out = sums_out; ps.count_bh = sums_in ? total_bh : pp.BH;
         e = dt::launch_plan_slots(ps, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e, "plan finalise launch");
-        ctx->launches += 2;
+        ctx->launches += 1;
         return DT_OK;
     }
     dt::PlanFinalParams pf;
@@ -514,10 +522,31 @@ dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32
     pf.mask = mask_dev;
     pf.w_out = w_dev;
     pf.eps_out = eps_out_dev;
+    pf.sums_in = sums_in; pf.sums_out = sums_out; pf.count_bh = sums_in ? total_bh : pp.BH;
     e = dt::launch_plan_final(pf, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "plan finalise launch");
-    ctx->launches += 2;
+    ctx->launches += 1;
     return DT_OK;
+}
+
+dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32_t group_size, uint8_t *mask_dev,
+                          double *w_dev, double *eps_out_dev, void *stream) {
+    return plan_impl(ctx, eps, target_fraction, group_size, mask_dev, w_dev, eps_out_dev, stream, nullptr, nullptr, 0);
+}
+
+dt_status dt_plan_sums(dt_ctx *ctx, double *sums_dev, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!sums_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null sums pointer");
+    return plan_impl(ctx, 0.0, -1.0, 1, nullptr, nullptr, nullptr, stream, nullptr, sums_dev, 0);
+}
+
+dt_status dt_plan_from_sums(dt_ctx *ctx, const double *sums_dev, int64_t total_bh, double eps, double target_fraction,
+                            int32_t group_size, uint8_t *mask_dev, double *w_dev, double *eps_out_dev, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
+    if (!sums_dev) return fail(ctx, DT_ERR_INVALID_ARG, "null sums pointer");
+    if (total_bh < (int64_t)ctx->cfg.B * ctx->cfg.H)
+        return fail(ctx, DT_ERR_INVALID_ARG, "total_bh is smaller than this context's own B * H");
+    return plan_impl(ctx, eps, target_fraction, group_size, mask_dev, w_dev, eps_out_dev, stream, sums_dev, nullptr, total_bh);
 }
 
 dt_status dt_step_host_workspace_bytes(const dt_config *cfg, size_t *bytes) {

@@ -94,6 +94,9 @@ struct PlanSlotsParams {
     uint8_t *mask;           // out, [P][S]
     double *w_out;           // out, [P][S], may be null
     double *eps_out;         // may be null
+    const double *sums_in;   // head-sharded planning: sums over all shards, [P][S]; null = sum this context's partials
+    double *sums_out;        // head-sharded planning: write this context's sums [P][S] and stop; null otherwise
+    long long count_bh;      // (batch, head) slices the sums cover: BH, or the total over all shards with sums_in
 };
 
 struct PlanFinalParams {
@@ -107,6 +110,9 @@ struct PlanFinalParams {
     uint8_t *mask;
     double *w_out;     // may be null
     double *eps_out;   // may be null
+    const double *sums_in;   // as in PlanSlotsParams
+    double *sums_out;
+    long long count_bh;
 };
 
 // Planner state of Algorithm 1, resident on the device.

@@ -95,6 +95,18 @@ __device__ __forceinline__ void sum_partials(const float *partials, int P, int S
     __syncthreads();
 }
 
+// Un-normalised sums of the per-row weights, one per (query partition, slot): this context's own (from its stage-1
+// partials) or, for head-sharded planning, the sums the caller added over all shards.
+__device__ __forceinline__ void load_sums(const double *sums_in, const float *partials, int P, int S, int BH, int chunks,
+                                          double *scratch, double *out_s) {
+    if (sums_in == nullptr) {
+        sum_partials(partials, P, S, BH, chunks, scratch, out_s);
+    } else {
+        if ((int)threadIdx.x < P * S) out_s[threadIdx.x] = sums_in[threadIdx.x];
+        __syncthreads();
+    }
+}
+
 // Strict total order used to rank decision units: larger measure first, then smaller group distance,
 // then smaller flat index.
 __device__ __forceinline__ bool ranks_before(double ma, int da, int fa, double mb, int db, int fb) {
@@ -117,11 +129,15 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
     const int P = p.P, total = P * P, g = p.group_size;
     const int ng = (P + g - 1) / g, nunits = P * ng;
     const int e = threadIdx.x;
-    sum_partials(p.partials, P, P, p.BH, p.chunks, m_s, W);   // m_s doubles as scratch here
+    load_sums(p.sums_in, p.partials, P, P, p.BH, p.chunks, m_s, W);   // m_s doubles as scratch here
+    if (p.sums_out) {   // first half of a head-sharded plan: the caller adds the shards' sums
+        if (e < total) p.sums_out[e] = W[e];
+        return;
+    }
     {
         const int i = e / P;
         if (e < total) {
-            const double cnt = (double)p.BH * (double)(p.off[i + 1] - p.off[i]);
+            const double cnt = (double)p.count_bh * (double)(p.off[i + 1] - p.off[i]);
             W[e] = W[e] / cnt;
             if (p.w_out) p.w_out[e] = W[e];
         }
@@ -229,11 +245,15 @@ __global__ void __launch_bounds__(1024) plan_slots_kernel(PlanSlotsParams p) {
     const int e = threadIdx.x;
     const int i = e / S, s = e - i * S;
     __shared__ double sum_s[DT_MAX_P * DT_MAX_P];
-    sum_partials(p.partials, P, S, p.BH, p.chunks, m_s, sum_s);   // m_s doubles as scratch here
+    load_sums(p.sums_in, p.partials, P, S, p.BH, p.chunks, m_s, sum_s);   // m_s doubles as scratch here
+    if (p.sums_out) {
+        if (e < total) p.sums_out[e] = sum_s[e];
+        return;
+    }
     double m = 0.0;
     int size = 0, dist = 0;
     if (e < total) {
-        m = sum_s[e] / ((double)p.BH * (double)(p.off[i + 1] - p.off[i]));
+        m = sum_s[e] / ((double)p.count_bh * (double)(p.off[i + 1] - p.off[i]));
         if (p.w_out) p.w_out[e] = m;
         size = (s == 0) ? 0 : (int)p.members[e];   // the local slot is no unit: always COMPUTE
         const int gi = i / g, k = s - 1;
@@ -433,6 +453,7 @@ extern "C" dt_status dt_plan_static(const float *lse_state_dev, const int32_t *p
     pf.mask = mask_dev;
     pf.w_out = w_dev;
     pf.eps_out = eps_out_dev;
+    pf.sums_in = nullptr; pf.sums_out = nullptr; pf.count_bh = pp.BH;
     if (dt::launch_plan_final(pf, st) != cudaSuccess) return DT_ERR_CUDA;
     return DT_OK;
 }
