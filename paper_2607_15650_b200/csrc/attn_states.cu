@@ -287,6 +287,11 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         // ------------------------------------------------------------ MMA issuer
         {
             const bool leader = (lane == 0);
+            // Every wait ends in a vote, so that no lane runs ahead of the issuing one: a lane that polled a barrier
+            // two phases late would read the parity of the wrong phase and never see it complete.
+            auto wait_all = [&](uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit) -> bool {
+                return __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, parity, abort_flag, limit)) != 0;
+            };
             constexpr uint32_t IDESC_QK = make_idesc_bf16_f32(128, ATTN_TILE, false, FP16);
             constexpr uint32_t IDESC_PV = make_idesc_bf16_f32(128, D, true, FP16);
             uint32_t q_phase = 0, p_phase = 0, of_phase = 0;
@@ -327,12 +332,12 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                     WorkItem it;
                     if (!decode_work<FUSED>(p, npairs, w, it)) continue;
-                    ok = mbar_wait_bounded(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
+                    ok = wait_all(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
                     if (!ok) break;
                     q_phase ^= 1u;
                     {
                         const uint32_t st = abs0 % C::STAGES, ph = (abs0 / C::STAGES) & 1u;
-                        ok = mbar_wait_bounded(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
+                        ok = wait_all(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
                         if (!ok) break;
                         tc_fence_after();
 #pragma unroll
@@ -349,10 +354,10 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         const bool has_pv = (k >= 1), has_qk = (k + 1 < it.tiles);
 #pragma unroll
                         for (int q = 0; q < ATTN_NQ; ++q) {
-                            ok = mbar_wait_bounded(bars.p_full + 8 * q, go_phase, abort_ptr, WAIT_LIMIT_NS);
+                            ok = wait_all(bars.p_full + 8 * q, go_phase, abort_ptr, WAIT_LIMIT_NS);
                             if (!ok) break;
                             if (k == 1) {  // first PV of the item: the previous item's epilogue must have drained O[q]
-                                ok = mbar_wait_bounded(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                                ok = wait_all(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
                                 if (!ok) break;
                             }
                             tc_fence_after();
@@ -380,13 +385,13 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
                 if (!decode_work<FUSED>(p, npairs, w, it)) continue;
-                ok = mbar_wait_bounded(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
+                ok = wait_all(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
                 if (!ok) break;
                 q_phase ^= 1u;
                 // first K tile
                 {
                     const uint32_t st = ring.st, ph = ring.ph;
-                    ok = mbar_wait_bounded(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
+                    ok = wait_all(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
@@ -406,10 +411,10 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     const bool more = (t + 1 < it.tiles);
 #pragma unroll
                     for (int q = 0; q < ATTN_NQ; ++q) {
-                        ok = mbar_wait_bounded(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_NS);
+                        ok = wait_all(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_NS);
                         if (!ok) break;
                         if (t == 0) {  // the previous item's epilogue must have drained O[q]
-                            ok = mbar_wait_bounded(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                            ok = wait_all(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
                             if (!ok) break;
                         }
                         tc_fence_after();
@@ -522,6 +527,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const uint32_t p_tmem = tmem_base + lane_addr + C::P_COL + q * C::P_STRIDE;   // D = 128: the same columns as S
         const uint32_t o_tmem = tmem_base + lane_addr + C::O_COL + q * D;
         uint32_t s_phase = 0, o_phase = 0, pv_phase = 0;
+        [[maybe_unused]] uint32_t go0_phase = 0;   // D = 64: parity of the current item's first phase of go[q]
         bool ok = true;
         StateT *o_state = static_cast<StateT *>(p.o_state);
 
@@ -626,11 +632,23 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 l_sum += rs;
                 tmem_wait_st();
                 tc_fence_before();
+                if constexpr (C::PREFETCH) {
+                    // "P_0 stored" belongs to phase 1 of go[q].  From tile 1 on, the wait for pv_done keeps a thread from
+                    // getting here before phase t has closed; at tile 0 nothing does, and an arrival made while phase 0
+                    // is still open would be counted in place of a slower thread's "S_0 read" or of the watcher's.
+                    if (t == 0) {
+                        ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.p_full + 8 * q, go0_phase, abort_ptr, WAIT_LIMIT_NS));
+                        if (!ok) break;
+                    }
+                }
                 mbar_arrive(bars.p_full + 8 * q);
                 if (!ok) break;
             }
             if (!ok) break;
-            if constexpr (C::PREFETCH) mbar_arrive(bars.p_full + 8 * q);   // closes the last phase (no further S to read)
+            if constexpr (C::PREFETCH) {
+                mbar_arrive(bars.p_full + 8 * q);   // closes the last phase (no further S to read)
+                go0_phase ^= (uint32_t)(it.tiles + 1) & 1u;   // the item took tiles + 1 phases of go[q]
+            }
             // epilogue: OUT_ij = O / l, LSE_ij = ln2 * (m + log2 l); rows beyond the partition are dropped
             ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.o_full + 8 * q, o_phase, abort_ptr, WAIT_LIMIT_NS));
             if (!ok) break;
