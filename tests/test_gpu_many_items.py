@@ -19,14 +19,19 @@ def _built():
     binding.lib()
 
 
-@pytest.mark.parametrize("D,P,state_dtype", [
-    (64, 6, binding.DT_STATE_FP32),      # two K/V tiles per item
-    (64, 12, binding.DT_STATE_BF16),     # one K/V tile per item: nothing but item starts and ends
-    (128, 6, binding.DT_STATE_FP32),
-    (128, 12, binding.DT_STATE_FP32),
+@pytest.mark.parametrize("D,P,state_dtype,shape", [
+    (64, 6, binding.DT_STATE_FP32, "short"),      # two K/V tiles per item
+    (64, 12, binding.DT_STATE_BF16, "short"),     # one K/V tile per item: nothing but item starts and ends
+    (128, 6, binding.DT_STATE_FP32, "short"),
+    (128, 12, binding.DT_STATE_FP32, "short"),
+    (64, 4, binding.DT_STATE_FP32, "wide"),       # Q, K, V larger than L2: operand loads land late
+    (128, 4, binding.DT_STATE_FP32, "wide"),
 ])
-def test_many_short_items_repeat_bit_for_bit(D, P, state_dtype):
-    wl = inputs.tiny_workload("many_items", B=2, H=24, D=D, grid=(4, 16, 20), n_text=13, P=P)
+def test_many_short_items_repeat_bit_for_bit(D, P, state_dtype, shape):
+    if shape == "short":
+        wl = inputs.tiny_workload("many_items", B=2, H=24, D=D, grid=(4, 16, 20), n_text=13, P=P)
+    else:
+        wl = inputs.tiny_workload("many_items_wide", B=1, H=48 if D == 64 else 24, D=D, grid=(10, 30, 30), n_text=0, P=P)
     dev = torch.device("cuda", 0)
     off = wl.offsets()
     ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, off, wl.scale, state_dtype)
@@ -42,7 +47,7 @@ def test_many_short_items_repeat_bit_for_bit(D, P, state_dtype):
     qb, kb, vb = (inputs.bf16_bits(x) for x in (q, k, v))
     out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
     lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
-    n_items = P * P * wl.B * wl.H
+    n_items = P * P * wl.B * wl.H * (-(-int(np.diff(off).max()) // 256))
     assert n_items > 8 * 148                          # several items per CTA
     for t, m in enumerate(masks):
         m_dev = torch.from_numpy(m.reshape(-1)).to(dev)
