@@ -18,9 +18,18 @@ namespace dt {
 namespace {
 
 constexpr int PLAN_THREADS = 256;
+// Resident blocks per SM the stage-1 kernel is compiled for.  Left to itself the compiler keeps the PMAX row
+// pointers live and takes 141 registers at PMAX = 32: one block of 8 warps per SM, far too few loads in flight.
+#ifndef DT_PLAN_BLOCKS32
+#define DT_PLAN_BLOCKS32 3
+#endif
+#ifndef DT_PLAN_BLOCKS16
+#define DT_PLAN_BLOCKS16 4
+#endif
+#define PLAN_MIN_BLOCKS(PMAX) ((PMAX) == 32 ? DT_PLAN_BLOCKS32 : ((PMAX) == 16 ? DT_PLAN_BLOCKS16 : 6))
 
 template <int PMAX>
-__global__ void __launch_bounds__(PLAN_THREADS) plan_partial_kernel(PlanParams p) {
+__global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS(PMAX)) plan_partial_kernel(PlanParams p) {
     const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z;
     const int P = p.S;   // columns: cache slots (pair mode: one per KV partition)
     const uint32_t have = p.nonempty ? p.nonempty[i] : 0xFFFFFFFFu;   // slots that exist for this query partition
@@ -42,22 +51,38 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_partial_kernel(PlanParams p
         float Z = 0.f;
 #pragma unroll
         for (int j = 0; j < PMAX; ++j) {
-            x[j] = expf(x[j] - M);
+            x[j] = __expf(x[j] - M);   // ex2.approx of a scaled argument: relative error ~1e-6, like the fp32 sums
             Z += x[j];
         }
         const float inv = 1.f / Z;
 #pragma unroll
         for (int j = 0; j < PMAX; ++j) acc[j] = fmaf(x[j], inv, acc[j]);
     }
-    // block reduction in a fixed order: xor-shuffle tree inside a warp, then warp 0 adds the 8 warps
+    // Block reduction in a fixed order.  Inside a warp the PMAX sums of the 32 lanes are reduced together: at each
+    // step a lane keeps one half of its values and adds its partner's copies of them (lanes that differ in the
+    // step's bit hold the two halves), so PMAX - 1 shuffles (plus log2(32 / PMAX) full rounds for PMAX < 32) do the
+    // work of 5 * PMAX and every value is still summed by the same xor tree, 16, 8, 4, 2, 1.  Lane l ends with the
+    // warp's sum of column l % PMAX.  Then the first P threads add the 8 warps.
     __shared__ float red[PLAN_THREADS / 32][PMAX];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    {
+        int ofs = 16;
 #pragma unroll
-    for (int j = 0; j < PMAX; ++j) {
-        float v = acc[j];
+        for (int full = 32; full > PMAX; full >>= 1, ofs >>= 1) {   // more lanes than columns: plain rounds first
 #pragma unroll
-        for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, s);
-        if (lane == 0) red[warp][j] = v;
+            for (int j = 0; j < PMAX; ++j) acc[j] += __shfl_xor_sync(0xFFFFFFFFu, acc[j], ofs);
+        }
+#pragma unroll
+        for (int half = PMAX / 2; half >= 1; half >>= 1, ofs >>= 1) {
+            const bool upper = (lane & ofs) != 0;
+#pragma unroll
+            for (int j = 0; j < half; ++j) {
+                const float send = upper ? acc[j] : acc[j + half];
+                const float keep = upper ? acc[j + half] : acc[j];
+                acc[j] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, ofs);
+            }
+        }
+        red[warp][lane & (PMAX - 1)] = acc[0];   // for PMAX < 32 several lanes hold (and write) the same sum
     }
     __syncthreads();
     if (threadIdx.x < P) {
@@ -107,12 +132,76 @@ __device__ __forceinline__ void load_sums(const double *sums_in, const float *pa
     }
 }
 
-// Strict total order used to rank decision units: larger measure first, then smaller group distance,
-// then smaller flat index.
-__device__ __forceinline__ bool ranks_before(double ma, int da, int fa, double mb, int db, int fb) {
-    if (ma != mb) return ma > mb;
-    if (da != db) return da < db;
-    return fa < fb;
+// Ranking of the decision units for a target pair count.  Strict total order: larger measure first, then smaller
+// group distance, then smaller flat index.  The units are sorted by a key that encodes that order (bitonic network
+// in shared memory, one element per thread), an inclusive scan over the sorted sizes gives every unit the number of
+// pairs it and all units before it stand for, and a unit is taken iff that total fits the budget -- the same
+// decisions as counting, per unit, the units that rank before it, in O(n log^2 n) instead of O(n^2) steps.
+__device__ __forceinline__ unsigned long long descending_key(double m) {   // ascending key order = descending m
+    unsigned long long u = (unsigned long long)__double_as_longlong(m);
+    u = (u >> 63) ? ~u : (u | (1ull << 63));
+    return ~u;
+}
+__device__ __forceinline__ double key_measure(unsigned long long k) {
+    unsigned long long u = ~k;
+    u = (u >> 63) ? (u & ~(1ull << 63)) : ~u;
+    return __longlong_as_double((long long)u);
+}
+struct RankScratch {
+    unsigned long long k1[DT_MAX_P * DT_MAX_P];   // descending_key(measure); all ones: no unit
+    uint32_t k2[DT_MAX_P * DT_MAX_P];             // distance << 20 | flat index << 8 | size
+    int warp_sum[32];
+    uint8_t dec[DT_MAX_P * DT_MAX_P];             // decision of unit e
+};
+// All 1024 threads call this.  Thread e < nunits brings its unit (size 0: none).  Returns the number of units taken;
+// sc.dec[e] holds the decisions, edge[0] / edge[1] the measures of the last unit taken and of the first one not
+// taken (left alone where there is none), *n_units the number of units.
+__device__ __forceinline__ int take_by_rank(RankScratch &sc, double m, int size, int dist, int nunits, int budget,
+                                            double *edge, int *n_units) {
+    const int e = threadIdx.x;
+    const bool unit = e < nunits && size > 0;
+    sc.k1[e] = unit ? descending_key(m) : ~0ull;
+    sc.k2[e] = unit ? ((uint32_t)dist << 20 | (uint32_t)e << 8 | (uint32_t)size) : 0xFFFFFF00u;
+    sc.dec[e] = 0;
+    int n = 32;
+    while (n < nunits) n <<= 1;          // sorted length: a power of two that covers the units
+    for (int k = 2; k <= n; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            __syncthreads();
+            const int x = e ^ j;
+            if (e < n && x > e) {
+                const unsigned long long a1 = sc.k1[e], b1 = sc.k1[x];
+                const uint32_t a2 = sc.k2[e], b2 = sc.k2[x];
+                const bool gt = a1 > b1 || (a1 == b1 && (a2 >> 8) > (b2 >> 8));
+                if (gt == ((e & k) == 0)) {
+                    sc.k1[e] = b1; sc.k1[x] = a1;
+                    sc.k2[e] = b2; sc.k2[x] = a2;
+                }
+            }
+        }
+    __syncthreads();
+    // inclusive scan of the sizes in rank order
+    const int lane = e & 31, warp = e >> 5;
+    const uint32_t mine2 = sc.k2[e];
+    const int sz = (e < n) ? (int)(mine2 & 0xFFu) : 0;
+    int cum = sz;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int up = __shfl_up_sync(0xFFFFFFFFu, cum, d);
+        if (lane >= d) cum += up;
+    }
+    if (lane == 31) sc.warp_sum[warp] = cum;
+    __syncthreads();
+    for (int w = 0; w < warp; ++w) cum += sc.warp_sum[w];
+    const bool take = sz > 0 && cum <= budget;
+    if (sz > 0) sc.dec[(mine2 >> 8) & 0xFFFu] = take ? 1 : 0;
+    const int taken = __syncthreads_count(take);
+    const int units = __syncthreads_count(sz > 0);
+    if (sz > 0 && e == taken - 1) edge[0] = key_measure(sc.k1[e]);
+    if (sz > 0 && e == taken) edge[1] = key_measure(sc.k1[e]);
+    if (e == 0) *n_units = units;
+    __syncthreads();
+    return taken;
 }
 
 // Stage 2.  W[i][j] from the partial sums, then one decision per unit (i, k): query partition i and the
@@ -121,15 +210,13 @@ __device__ __forceinline__ bool ranks_before(double ma, int da, int fa, double m
 // largest measure taken in rank order while their members fit into K - P pairs.
 __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
     __shared__ double W[DT_MAX_P * DT_MAX_P];
-    __shared__ double m_s[DT_MAX_P * DT_MAX_P];
-    __shared__ uint8_t size_s[DT_MAX_P * DT_MAX_P];
-    __shared__ uint8_t dist_s[DT_MAX_P * DT_MAX_P];
-    __shared__ uint8_t dec_s[DT_MAX_P * DT_MAX_P];
+    __shared__ RankScratch sc;
     __shared__ double edge[2];
+    __shared__ int n_units;
     const int P = p.P, total = P * P, g = p.group_size;
     const int ng = (P + g - 1) / g, nunits = P * ng;
     const int e = threadIdx.x;
-    load_sums(p.sums_in, p.partials, P, P, p.BH, p.chunks, m_s, W);   // m_s doubles as scratch here
+    load_sums(p.sums_in, p.partials, P, P, p.BH, p.chunks, reinterpret_cast<double *>(sc.k1), W);   // sc.k1 is scratch here
     if (p.sums_out) {   // first half of a head-sharded plan: the caller adds the shards' sums
         if (e < total) p.sums_out[e] = W[e];
         return;
@@ -154,45 +241,22 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
             if (j != ui) { m += W[ui * P + j]; ++size; }
         const int gi = ui / g;
         dist = uk > gi ? uk - gi : gi - uk;
-        m_s[e] = m;
-        size_s[e] = (uint8_t)size;
-        dist_s[e] = (uint8_t)dist;
     }
-    __syncthreads();
-    bool take = false;
-    int rank = -1;
-    const int budget = p.K - P;
-    if (e < nunits && size > 0) {
-        if (!p.mode_target) {
-            take = m > p.eps;
-        } else {
-            rank = 0;
-            int cum = size;
-            for (int o = 0; o < nunits; ++o) {   // every thread walks the same o: shared-memory broadcasts
-                const int so = size_s[o];
-                if (o == e || so == 0) continue;
-                if (ranks_before(m_s[o], dist_s[o], o, m, dist, e)) { ++rank; cum += so; }
-            }
-            take = cum <= budget;
-        }
-    }
-    if (e < nunits) dec_s[e] = take ? 1 : 0;
-    const int taken = __syncthreads_count(take);
-    if (p.mode_target && rank >= 0) {
-        if (rank == taken - 1) edge[0] = m;
-        if (rank == taken) edge[1] = m;
+    int taken = 0;
+    if (p.mode_target) {
+        taken = take_by_rank(sc, m, size, dist, nunits, p.K - P, edge, &n_units);
+    } else {
+        sc.dec[e] = (e < nunits && size > 0 && m > p.eps) ? 1 : 0;
+        __syncthreads();
     }
     if (e < total) {
         const int i = e / P, j = e - i * P;
-        p.mask[e] = (i == j || dec_s[i * ng + j / g]) ? 1 : 0;
+        p.mask[e] = (i == j || sc.dec[i * ng + j / g]) ? 1 : 0;
     }
-    __syncthreads();
     if (e == 0 && p.eps_out) {
         double eps = p.eps;
         if (p.mode_target) {
-            int n = 0;
-            for (int o = 0; o < nunits; ++o) n += size_s[o] > 0;
-            if (n == 0 || taken == n) eps = 0.0;
+            if (n_units == 0 || taken == n_units) eps = 0.0;
             else if (taken == 0) eps = edge[1];
             else eps = 0.5 * (edge[0] + edge[1]);
         }
@@ -237,15 +301,14 @@ __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int
 // members' weights, Eq. 12, which is what the slot's LSE yields directly).  COMPUTE iff measure > eps
 // (Eq. 13), or the units of largest measure taken in rank order while their member pairs fit into K - P.
 __global__ void __launch_bounds__(1024) plan_slots_kernel(PlanSlotsParams p) {
-    __shared__ double m_s[DT_MAX_P * DT_MAX_P];
-    __shared__ uint8_t size_s[DT_MAX_P * DT_MAX_P];
-    __shared__ uint8_t dist_s[DT_MAX_P * DT_MAX_P];
+    __shared__ double sum_s[DT_MAX_P * DT_MAX_P];
+    __shared__ RankScratch sc;
     __shared__ double edge[2];
+    __shared__ int n_units;
     const int P = p.P, S = p.S, total = P * S, g = p.group_size;
     const int e = threadIdx.x;
     const int i = e / S, s = e - i * S;
-    __shared__ double sum_s[DT_MAX_P * DT_MAX_P];
-    load_sums(p.sums_in, p.partials, P, S, p.BH, p.chunks, m_s, sum_s);   // m_s doubles as scratch here
+    load_sums(p.sums_in, p.partials, P, S, p.BH, p.chunks, reinterpret_cast<double *>(sc.k1), sum_s);   // sc.k1 is scratch here
     if (p.sums_out) {
         if (e < total) p.sums_out[e] = sum_s[e];
         return;
@@ -258,42 +321,21 @@ __global__ void __launch_bounds__(1024) plan_slots_kernel(PlanSlotsParams p) {
         size = (s == 0) ? 0 : (int)p.members[e];   // the local slot is no unit: always COMPUTE
         const int gi = i / g, k = s - 1;
         dist = k > gi ? k - gi : gi - k;
-        m_s[e] = m;
-        size_s[e] = (uint8_t)size;
-        dist_s[e] = (uint8_t)dist;
     }
     if (e < 2) edge[e] = 0.0;
     __syncthreads();
-    bool take = false;
-    int rank = -1;
-    const int budget = p.K - P;
-    if (e < total && size > 0) {
-        if (!p.mode_target) {
-            take = m > p.eps;
-        } else {
-            rank = 0;
-            int cum = size;
-            for (int o = 0; o < total; ++o) {
-                const int so = size_s[o];
-                if (o == e || so == 0) continue;
-                if (ranks_before(m_s[o], dist_s[o], o, m, dist, e)) { ++rank; cum += so; }
-            }
-            take = cum <= budget;
-        }
+    int taken = 0;
+    if (p.mode_target) {
+        taken = take_by_rank(sc, m, size, dist, total, p.K - P, edge, &n_units);
+    } else {
+        sc.dec[e] = (e < total && size > 0 && m > p.eps) ? 1 : 0;
+        __syncthreads();
     }
-    const int taken = __syncthreads_count(take);
-    if (p.mode_target && rank >= 0) {
-        if (rank == taken - 1) edge[0] = m;
-        if (rank == taken) edge[1] = m;
-    }
-    if (e < total) p.mask[e] = (s == 0 || take) ? 1 : 0;
-    __syncthreads();
+    if (e < total) p.mask[e] = (s == 0 || sc.dec[e]) ? 1 : 0;
     if (e == 0 && p.eps_out) {
         double eps = p.eps;
         if (p.mode_target) {
-            int n = 0;
-            for (int o = 0; o < total; ++o) n += size_s[o] > 0;
-            if (n == 0 || taken == n) eps = 0.0;
+            if (n_units == 0 || taken == n_units) eps = 0.0;
             else if (taken == 0) eps = edge[1];
             else eps = 0.5 * (edge[0] + edge[1]);
         }
