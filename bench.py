@@ -104,7 +104,8 @@ class ClockSampler:
 
 
 # DRAM traffic of attn_states_kernel per (head, COMPUTE pair) of the c3-shaped tiles, from the ncu capture
-# summarised in profiles/attn_states_kernel_c3_wan720p_h4.md: (276.4 MB read + 951.0 MB written) / (4 heads x 102 pairs).
+# summarised under profiles/ (kernel attn_states, workload c3_wan720p, 4 heads): (239.7 MB read + 941.4 MB written)
+# / (4 heads x 102 pairs).
 # Traffic grows in proportion to heads x pairs (the pair states written dominate it).
 NCU_ATTN_TRAFFIC_PER_HEAD_PAIR = {"c3_wan720p": (239.7e6 + 941.4e6) / (4 * 102)}
 

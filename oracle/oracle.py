@@ -227,7 +227,7 @@ class OracleSession:
 # --------------------------------------------------------------------------------------------------
 # Anchor-guided selection planning (Section 4; Algorithm 1), in plain numpy fp64.
 #
-# Readings where the paper is silent (also listed in the design doc):
+# Readings where the paper is silent:
 #   * ||AS||_2 (Eq. 9, Eq. 10) is the 2-norm of OUT and LSE stacked, taken over all rows and heads of the
 #     query partition;
 #   * delta(j, t, t_c) is evaluated against the last anchor for every state (Eq. 10 defines it only for
