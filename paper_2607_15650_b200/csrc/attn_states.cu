@@ -13,7 +13,8 @@
 //   warp 8           TMA producer: Q tiles once per work item, K and V tiles through a ring
 //   warp 9           MMA issuer: the whole warp runs the (warp-uniform) control flow and address arithmetic, one
 //                    lane issues tcgen05.mma / tcgen05.commit -- measured 4 % faster than a single-lane branch
-//   warp 10          K/V watcher: adds its arrival to p_full[0] once V_t and K_{t+1} have landed
+//   warp 10          K/V watcher: adds its arrival to p_full[0] once V_t and K_{t+1} have landed, and hands the
+//                    stages and the place of Q back to the producer once the MMAs that read them are done
 //   warp 11          idle (completes the producer warpgroup for the register hand-over)
 // TMEM (512 columns): S0 | S1 | O0 | O1.  S_t = Q K_t^T (fp32) lands in S; the softmax warpgroup
 // reads its row, writes P = exp2(s*scale*log2e - m) back over S as packed bf16 (fp16 for fp16 inputs),
@@ -345,8 +346,6 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             issue_qk(q, st);
                             if (leader) tc_commit(bars.s_full + 8 * q);
                         }
-                        if (leader) tc_commit(bars.kv_empty + 8 * st);
-                        if (it.tiles == 1) if (leader) tc_commit(bars.q_empty);
                     }
                     for (int k = 0; k <= it.tiles && ok; ++k) {
                         const uint32_t st_v = (abs0 + 2 * k - 1) % C::STAGES;   // V_{k-1} (k >= 1)
@@ -371,11 +370,6 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             }
                         }
                         if (!ok) break;
-                        if (has_pv) if (leader) tc_commit(bars.kv_empty + 8 * st_v);
-                        if (has_qk) {
-                            if (leader) tc_commit(bars.kv_empty + 8 * st_k);
-                            if (k + 2 == it.tiles) if (leader) tc_commit(bars.q_empty);
-                        }
                         go_phase ^= 1u;
                     }
                     of_phase ^= 1u;
@@ -446,8 +440,11 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             uint32_t p_phase = 0;
             bool ok = true;
             if constexpr (C::PREFETCH) {
-                // D = 64: one arrival on each go[q] per phase k, made once V_{k-1} and K_{k+1} are in shared memory
-                uint32_t abs0 = 0;
+                // D = 64: one arrival on each go[q] per phase k, made once V_{k-1} and K_{k+1} are in shared memory.
+                // As at D = 128 the watcher also hands the stages back: S_k of query tile 1 complete (committed last in
+                // phase k - 1, or in the item's prologue) tells that Q K_k^T and P_{k-2} V_{k-2} are done for both
+                // query tiles, o_full[1] that the last two P V are.
+                uint32_t abs0 = 0, s1_phase = 0, o1_phase = 0;
                 for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                     WorkItem it;
                     if (!decode_work<FUSED>(p, npairs, w, it)) continue;
@@ -463,6 +460,20 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         if (ok) {
 #pragma unroll
                             for (int q = 0; q < ATTN_NQ; ++q) mbar_arrive(bars.p_full + 8 * q);
+                            if (k < it.tiles) {
+                                ok = mbar_wait_bounded(bars.s_full + 8, s1_phase, abort_ptr, WAIT_LIMIT_NS);
+                                if (!ok) break;
+                                s1_phase ^= 1u;
+                                mbar_arrive(bars.kv_empty + 8 * ((abs0 + 2 * k) % C::STAGES));                        // K_k
+                                if (k >= 2) mbar_arrive(bars.kv_empty + 8 * ((abs0 + 2 * (k - 2) + 1) % C::STAGES));  // V_{k-2}
+                                if (k + 1 == it.tiles) mbar_arrive(bars.q_empty);   // that was the item's last Q K^T
+                            } else {
+                                ok = mbar_wait_bounded(bars.o_full + 8, o1_phase, abort_ptr, WAIT_LIMIT_NS);
+                                if (!ok) break;
+                                o1_phase ^= 1u;
+                                if (k >= 2) mbar_arrive(bars.kv_empty + 8 * ((abs0 + 2 * (k - 2) + 1) % C::STAGES));  // V_{tiles-2}
+                                mbar_arrive(bars.kv_empty + 8 * ((abs0 + 2 * (k - 1) + 1) % C::STAGES));              // V_{tiles-1}
+                            }
 #pragma unroll
                             for (int q = 0; q < ATTN_NQ; ++q)
                                 ok = ok && mbar_wait_bounded(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_NS);
