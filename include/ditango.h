@@ -60,7 +60,10 @@ typedef enum {
     DT_ERR_UNSUPPORTED = 2, /* D not in {64,128}, P > 32, unknown state dtype, device not sm_100 */
     DT_ERR_STATE = 3,       /* cache not bound or too small; REUSE of a pair never computed       */
     DT_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (text in dt_last_error)        */
-    DT_ERR_TIMEOUT = 5      /* a bounded device-side wait expired; the kernel returned normally   */
+    DT_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired; the kernel returned normally   */
+    DT_ERR_RANGE = 6        /* bf16 inputs: within one 128-key tile a logit (times log2 e) rose more than
+                               about 120 above everything the row had seen before (exp2 overflows fp32);
+                               the states of that launch are not valid.  fp16 inputs have no such limit. */
 } dt_status;
 
 enum { DT_STATE_FP32 = 0, DT_STATE_BF16 = 1 };
@@ -325,7 +328,7 @@ dt_status dt_launch_count(dt_ctx *ctx, uint64_t *count);
 dt_status dt_selftest_wait_timeout(dt_ctx *ctx, uint32_t limit_us, void *stream);
 
 /* Read (and clear) the device status word; synchronises the device.  Returns DT_OK,
- * DT_ERR_STATE or DT_ERR_TIMEOUT. */
+ * DT_ERR_STATE, DT_ERR_TIMEOUT or DT_ERR_RANGE. */
 dt_status dt_poll(dt_ctx *ctx);
 
 const char *dt_status_str(dt_status s);

@@ -14,7 +14,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libditango.so")
 
-DT_OK, DT_ERR_INVALID_ARG, DT_ERR_UNSUPPORTED, DT_ERR_STATE, DT_ERR_CUDA, DT_ERR_TIMEOUT = range(6)
+DT_OK, DT_ERR_INVALID_ARG, DT_ERR_UNSUPPORTED, DT_ERR_STATE, DT_ERR_CUDA, DT_ERR_TIMEOUT, DT_ERR_RANGE = range(7)
 DT_STATE_FP32, DT_STATE_BF16 = 0, 1
 DT_INPUT_BF16, DT_INPUT_FP16 = 0, 1
 DT_MAX_P = 32

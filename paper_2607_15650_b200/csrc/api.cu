@@ -134,6 +134,7 @@ const char *dt_status_str(dt_status s) {
         case DT_ERR_STATE: return "DT_ERR_STATE";
         case DT_ERR_CUDA: return "DT_ERR_CUDA";
         case DT_ERR_TIMEOUT: return "DT_ERR_TIMEOUT";
+        case DT_ERR_RANGE: return "DT_ERR_RANGE";
     }
     return "DT_ERR_UNKNOWN";
 }
@@ -895,6 +896,8 @@ dt_status dt_poll(dt_ctx *ctx) {
     if (e != cudaSuccess) return fail_cuda(ctx, e, "dt_poll");
     if (word & dt::STATUS_WAIT_TIMEOUT) return fail(ctx, DT_ERR_TIMEOUT, "a bounded device-side wait expired");
     if (word & dt::STATUS_REUSE_EMPTY) return fail(ctx, DT_ERR_STATE, "REUSE of a pair that was never computed");
+    if (word & dt::STATUS_LOGIT_RANGE)
+        return fail(ctx, DT_ERR_RANGE, "a logit rose more than 120 binades above the running reference within one K/V tile");
     return DT_OK;
 }
 

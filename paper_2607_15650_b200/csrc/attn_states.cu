@@ -54,7 +54,7 @@ constexpr int ATTN_THREADS = NUM_SOFTMAX_THREADS + 128;  // producer warpgroup: 
 constexpr int LAUNCH_REGS = 168, REGS_SOFTMAX = 208, REGS_PRODUCER = 88;
 static_assert((REGS_SOFTMAX - LAUNCH_REGS) * NUM_SOFTMAX_THREADS <= (LAUNCH_REGS - REGS_PRODUCER) * 128,
               "softmax warps would wait forever for registers nobody releases");
-constexpr long long WAIT_LIMIT_NS = 4000000000ll;   // SM clock cycles: about 2 s
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // SM clock cycles: about 2 s
 constexpr float ROWSUM_TRIGGER = 512.0f;   // a row sum of P at or above this sends the tile through the slow path
 constexpr float RESCALE_THRESHOLD = 1.0f;  // log2 units: in the slow path the reference moves if the maximum grew by more
 #ifndef DT_POLY_PER_8
@@ -72,7 +72,7 @@ struct Cfg {
     static constexpr int KV_BYTES = STAGES * TILE_BYTES;
     static constexpr int OUT_STAGE_BYTES = ATTN_TILE * 128;   // epilogue staging per query tile: 4 warps x [32 rows x 128 bytes]
     static constexpr int OUT_BYTES = ATTN_NQ * OUT_STAGE_BYTES;
-    static constexpr int NBARS = 2 + 2 * STAGES + 5 * ATTN_NQ;
+    static constexpr int NBARS = 2 + 2 * STAGES + 6 * ATTN_NQ;
     static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + Q_BYTES + KV_BYTES + OUT_BYTES + NBARS * 8 + 64;
     // TMEM columns.  D = 128 fills all 512 (S0 | S1 | O0 | O1) and P has to live over S.  D = 64 leaves 128 columns:
     // there P gets its own place (S0 | S1 | P0 | P1 | O0 | O1), so S may be overwritten as soon as the softmax has
@@ -87,8 +87,14 @@ struct Cfg {
 struct Bars {
     uint32_t q_full, q_empty;
     uint32_t kv_full, kv_empty;   // + 8*stage
-    uint32_t s_full, p_full, o_full, o_free, pv_done;  // + 8*q
+    uint32_t s_full, p_full, o_full, o_free, pv_done, s_free;  // + 8*q
 };
+
+// D = 64 (Cfg::PREFETCH): place of an item's K/V tiles in the order they are loaded and consumed --
+// K_0, K_1, V_0, K_2, V_1, ..., K_{n-1}, V_{n-2}, V_{n-1}: Q K_{t+1}^T is issued as soon as S_t has been read,
+// before P_t V_t.
+__device__ __forceinline__ uint32_t k_place(int t) { return t == 0 ? 0u : (uint32_t)(2 * t - 1); }
+__device__ __forceinline__ uint32_t v_place(int t, int tiles) { return t + 1 == tiles ? (uint32_t)(2 * tiles - 1) : (uint32_t)(2 * t + 2); }
 
 // Position in the K/V ring: stage index and the parity of its current use.
 template <int STAGES>
@@ -155,6 +161,12 @@ __device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, lon
 }
 
 // 32 consecutive elements of a cached state row as fp32
+__device__ __forceinline__ __nv_bfloat162 u32_as_bf162(uint32_t x) {
+    return *reinterpret_cast<const __nv_bfloat162 *>(&x);
+}
+__device__ __forceinline__ uint32_t bf162_as_u32(__nv_bfloat162 x) {
+    return *reinterpret_cast<const uint32_t *>(&x);
+}
 __device__ __forceinline__ void load_state_chunk(const float *src, float (&v)[32]) {
 #pragma unroll
     for (int c = 0; c < 32; c += 4) {
@@ -173,6 +185,27 @@ __device__ __forceinline__ void load_state_chunk(const __nv_bfloat16 *src, float
             v[c + 2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
         }
     }
+}
+
+// A row sum of P that reached ROWSUM_TRIGGER moves the row's reference up by e = floor(log2(row sum)) binades:
+// this thread's row of O (fp32, D columns) times 2^-e, in place; returns e (0 for a row below the trigger).
+// Out of line: it runs once in many tiles and would only lengthen the softmax loop.
+template <int D>
+__device__ __noinline__ int move_reference(uint32_t o_tmem, float row_sum) {
+    const bool need = !(row_sum < ROWSUM_TRIGGER);   // also true for inf / NaN
+    const int e = need ? min(((__float_as_int(row_sum) >> 23) & 0xFF) - 127, 126) : 0;
+    const float alpha = __int_as_float((127 - e) << 23);
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t o[32];
+        tmem_ld_x32(o_tmem + c0, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+        tmem_st_x32(o_tmem + c0, o);
+    }
+    tmem_wait_st();
+    return e;
 }
 
 template <int D, typename StateT, bool FUSED, bool FP16>
@@ -200,6 +233,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     bars.o_full = bars.p_full + 8 * ATTN_NQ;
     bars.o_free = bars.o_full + 8 * ATTN_NQ;
     bars.pv_done = bars.o_free + 8 * ATTN_NQ;   // D = 64 only: the PV MMAs that read P[q] have completed
+    bars.s_free = bars.pv_done + 8 * ATTN_NQ;   // D = 64 only: S[q] has been read (and the next K tile has landed)
 
     // warp index through a shuffle: the compiler then knows that it is the same in all lanes of a warp
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
@@ -208,16 +242,17 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp == TMA_WARP && lane == 0) {
         abort_flag = 0;
         mbar_init(bars.q_full, 1);
-        mbar_init(bars.q_empty, 1);
+        // D = 64: each of the two MMA warps hands Q's place and the K/V stages back with a commit of its own
+        mbar_init(bars.q_empty, C::PREFETCH ? 2 : 1);
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(bars.kv_full + 8 * s, 1);
-            mbar_init(bars.kv_empty + 8 * s, 1);
+            mbar_init(bars.kv_empty + 8 * s, C::PREFETCH ? 2 : 1);
         }
         for (int q = 0; q < ATTN_NQ; ++q) {
             mbar_init(bars.s_full + 8 * q, 1);
-            // D = 128: P ready (128 threads), tile 0: + the K/V watcher.  D = 64: "go" = S read + previous P stored
-            // (2 x 128) + the watcher, for both tiles
-            mbar_init(bars.p_full + 8 * q, C::PREFETCH ? 257 : 128 + (q == 0 ? 1 : 0));
+            // D = 128: P ready (128 threads), tile 0: + the K/V watcher.  D = 64: P stored (128 threads)
+            mbar_init(bars.p_full + 8 * q, C::PREFETCH ? 128 : 128 + (q == 0 ? 1 : 0));
+            mbar_init(bars.s_free + 8 * q, 128);   // D = 64: S read (128 threads)
             mbar_init(bars.o_full + 8 * q, 1);
             mbar_init(bars.o_free + 8 * q, 128);
             mbar_init(bars.pv_done + 8 * q, 1);
@@ -250,7 +285,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
                 if (!decode_work<FUSED>(p, npairs, w, it)) continue;
-                ok = mbar_wait_bounded(bars.q_empty, q_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                ok = mbar_wait_bounded(bars.q_empty, q_phase ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
                 if (!ok) break;
                 mbar_arrive_expect_tx(bars.q_full, C::Q_BYTES);
 #pragma unroll
@@ -260,12 +295,29 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         tma_load_4d(q_smem + q * C::TILE_BYTES + hf * C::HALF_BYTES, &tmap_q, bars.q_full, hf * 64, it.h,
                                     it.q_row0 + q * ATTN_TILE, it.b);
                 q_phase ^= 1u;
+                if constexpr (C::PREFETCH) {
+                    for (int n = 0; n < 2 * it.tiles && ok; ++n) {
+                        // place n of the item's load order: K_0 | K_{(n+1)/2} for odd n | V_{(n-2)/2} for even n | V_{tiles-1} last
+                        const bool is_k = (n == 0) || ((n & 1) && n + 1 < 2 * it.tiles);
+                        const int t = is_k ? (n + 1) / 2 : (n + 1 == 2 * it.tiles ? it.tiles - 1 : (n - 2) / 2);
+                        const int key0 = it.template tile<FUSED>(t).x;
+                        const uint32_t st = ring.st, ph = ring.ph;
+                        ok = mbar_wait_bounded(bars.kv_empty + 8 * st, ph ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(bars.kv_full + 8 * st, C::TILE_BYTES);
+#pragma unroll
+                        for (int hf = 0; hf < C::NHALF; ++hf)
+                            tma_load_4d(kv_smem + st * C::TILE_BYTES + hf * C::HALF_BYTES, is_k ? &tmap_k : &tmap_v,
+                                        bars.kv_full + 8 * st, hf * 64, it.h, key0, it.b);
+                        ring.advance();
+                    }
+                } else
                 for (int t = 0; t < it.tiles && ok; ++t) {
                     const int key0 = it.template tile<FUSED>(t).x;
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
                         const uint32_t st = ring.st, ph = ring.ph;
-                        ok = mbar_wait_bounded(bars.kv_empty + 8 * st, ph ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                        ok = mbar_wait_bounded(bars.kv_empty + 8 * st, ph ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
                         if (!ok) break;
                         mbar_arrive_expect_tx(bars.kv_full + 8 * st, C::TILE_BYTES);
 #pragma unroll
@@ -284,7 +336,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         }
-      } else if (warp == MMA_WARP) {
+      } else if (warp == MMA_WARP || (C::PREFETCH && warp == WATCH_WARP)) {
         // ------------------------------------------------------------ MMA issuer
         {
             const bool leader = (lane == 0);
@@ -325,52 +377,64 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             };
 
             if constexpr (C::PREFETCH) {
-                // D = 64.  Per item, "go" phases k = 0 .. tiles for each query tile: phase k is complete when the
-                // softmax has read S_k, stored P_{k-1}, and V_{k-1}, K_{k+1} have landed.  Then O += P_{k-1} V_{k-1}
-                // (commit pv_done: P's place is free again) and S_{k+1} = Q K_{k+1}^T (commit s_full) are issued.
-                // Stage of the n-th K/V tile of the run: (n mod STAGES).
-                uint32_t abs0 = 0, go_phase = 0;   // tiles loaded before this item (K_t = abs0 + 2t, V_t = abs0 + 2t + 1)
+                // D = 64: one MMA warp per query tile (this one: mq), so that the two tiles' chains of wait -> issue ->
+                // commit run side by side; the tensor pipe has room for both (an M = 128 MMA takes 64 cycles whatever
+                // its N, so a K/V tile costs 4 + 8 MMAs per query tile against 2048 cycles of exponentials per pair).
+                // Per K/V tile t: s_free[mq] -- the softmax has read S_t -- lets S_{t+1} = Q K_{t+1}^T overwrite S;
+                // p_full[mq] -- P_t is stored -- lets O += P_t V_t go (commit pv_done: P's place is free again, or o_full
+                // after the last tile).  This warp waits for the K/V tiles itself and hands them (and Q's place) back with
+                // a commit of its own: a stage is free when both warps' commits have arrived, so neither query tile can
+                // run ahead of the other by more than the ring holds.  Place n of the run of K/V tiles lives in ring
+                // stage (n mod STAGES).
+                const int mq = warp - MMA_WARP;
+                uint32_t abs0 = 0, t_phase = 0;   // tiles loaded before this item; parity of s_free / p_full (one phase per tile)
+                auto wait_kv = [&](uint32_t place, uint32_t &st) -> bool {
+                    const uint32_t a = abs0 + place;
+                    st = a % C::STAGES;
+                    return wait_all(bars.kv_full + 8 * st, (a / C::STAGES) & 1u, abort_ptr, WAIT_LIMIT_CYCLES);
+                };
                 for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                     WorkItem it;
                     if (!decode_work<FUSED>(p, npairs, w, it)) continue;
-                    ok = wait_all(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
+                    uint32_t st = 0;
+                    ok = wait_all(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_CYCLES) && wait_kv(0, st);
                     if (!ok) break;
                     q_phase ^= 1u;
-                    {
-                        const uint32_t st = abs0 % C::STAGES, ph = (abs0 / C::STAGES) & 1u;
-                        ok = wait_all(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
-                        if (!ok) break;
-                        tc_fence_after();
-#pragma unroll
-                        for (int q = 0; q < ATTN_NQ; ++q) {
-                            issue_qk(q, st);
-                            if (leader) tc_commit(bars.s_full + 8 * q);
-                        }
+                    tc_fence_after();
+                    issue_qk(mq, st);
+                    if (leader) {
+                        tc_commit(bars.s_full + 8 * mq);
+                        tc_commit(bars.kv_empty + 8 * st);            // K_0 is free once both query tiles' MMAs have read it
+                        if (it.tiles == 1) tc_commit(bars.q_empty);
                     }
-                    for (int k = 0; k <= it.tiles && ok; ++k) {
-                        const uint32_t st_v = (abs0 + 2 * k - 1) % C::STAGES;   // V_{k-1} (k >= 1)
-                        const uint32_t st_k = (abs0 + 2 * k + 2) % C::STAGES;   // K_{k+1}
-                        const bool has_pv = (k >= 1), has_qk = (k + 1 < it.tiles);
-#pragma unroll
-                        for (int q = 0; q < ATTN_NQ; ++q) {
-                            ok = wait_all(bars.p_full + 8 * q, go_phase, abort_ptr, WAIT_LIMIT_NS);
+                    for (int k = 0; k < it.tiles && ok; ++k) {
+                        const bool more = (k + 1 < it.tiles);
+                        ok = wait_all(bars.s_free + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES);
+                        if (!ok) break;
+                        if (more) {
+                            ok = wait_kv(k_place(k + 1), st);
                             if (!ok) break;
-                            if (k == 1) {  // first PV of the item: the previous item's epilogue must have drained O[q]
-                                ok = wait_all(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
-                                if (!ok) break;
-                            }
                             tc_fence_after();
-                            if (has_pv) {
-                                issue_pv(q, st_v, k > 1);
-                                if (leader) tc_commit(k < it.tiles ? bars.pv_done + 8 * q : bars.o_full + 8 * q);   // P's place is free
-                            }
-                            if (has_qk) {
-                                issue_qk(q, st_k);
-                                if (leader) tc_commit(bars.s_full + 8 * q);
+                            issue_qk(mq, st);
+                            if (leader) {
+                                tc_commit(bars.s_full + 8 * mq);
+                                tc_commit(bars.kv_empty + 8 * st);
+                                if (k + 2 == it.tiles) tc_commit(bars.q_empty);   // that was the item's last Q K^T
                             }
                         }
+                        ok = wait_all(bars.p_full + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES) && wait_kv(v_place(k, it.tiles), st);
                         if (!ok) break;
-                        go_phase ^= 1u;
+                        if (k == 0) {  // first PV of the item: the previous item's epilogue must have drained O[mq]
+                            ok = wait_all(bars.o_free + 8 * mq, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                        issue_pv(mq, st, k > 0);
+                        if (leader) {
+                            tc_commit(more ? bars.pv_done + 8 * mq : bars.o_full + 8 * mq);
+                            tc_commit(bars.kv_empty + 8 * st);
+                        }
+                        t_phase ^= 1u;
                     }
                     of_phase ^= 1u;
                     abs0 += 2u * (uint32_t)it.tiles;
@@ -379,13 +443,13 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                 WorkItem it;
                 if (!decode_work<FUSED>(p, npairs, w, it)) continue;
-                ok = wait_all(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_NS);
+                ok = wait_all(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_CYCLES);
                 if (!ok) break;
                 q_phase ^= 1u;
                 // first K tile
                 {
                     const uint32_t st = ring.st, ph = ring.ph;
-                    ok = wait_all(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_NS);
+                    ok = wait_all(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_CYCLES);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
@@ -405,10 +469,10 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     const bool more = (t + 1 < it.tiles);
 #pragma unroll
                     for (int q = 0; q < ATTN_NQ; ++q) {
-                        ok = wait_all(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_NS);
+                        ok = wait_all(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_CYCLES);
                         if (!ok) break;
                         if (t == 0) {  // the previous item's epilogue must have drained O[q]
-                            ok = wait_all(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_NS);
+                            ok = wait_all(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
                             if (!ok) break;
                         }
                         tc_fence_after();
@@ -440,48 +504,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             uint32_t p_phase = 0;
             bool ok = true;
             if constexpr (C::PREFETCH) {
-                // D = 64: one arrival on each go[q] per phase k, made once V_{k-1} and K_{k+1} are in shared memory.
-                // As at D = 128 the watcher also hands the stages back: S_k of query tile 1 complete (committed last in
-                // phase k - 1, or in the item's prologue) tells that Q K_k^T and P_{k-2} V_{k-2} are done for both
-                // query tiles, o_full[1] that the last two P V are.
-                uint32_t abs0 = 0, s1_phase = 0, o1_phase = 0;
-                for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
-                    WorkItem it;
-                    if (!decode_work<FUSED>(p, npairs, w, it)) continue;
-                    for (int k = 0; k <= it.tiles && ok; ++k) {
-                        if (k >= 1) {
-                            const uint32_t a = abs0 + 2 * k - 1;
-                            ok = mbar_wait_bounded(bars.kv_full + 8 * (a % C::STAGES), (a / C::STAGES) & 1u, abort_ptr, WAIT_LIMIT_NS);
-                        }
-                        if (ok && k + 1 < it.tiles) {
-                            const uint32_t a = abs0 + 2 * k + 2;
-                            ok = mbar_wait_bounded(bars.kv_full + 8 * (a % C::STAGES), (a / C::STAGES) & 1u, abort_ptr, WAIT_LIMIT_NS);
-                        }
-                        if (ok) {
-#pragma unroll
-                            for (int q = 0; q < ATTN_NQ; ++q) mbar_arrive(bars.p_full + 8 * q);
-                            if (k < it.tiles) {
-                                ok = mbar_wait_bounded(bars.s_full + 8, s1_phase, abort_ptr, WAIT_LIMIT_NS);
-                                if (!ok) break;
-                                s1_phase ^= 1u;
-                                mbar_arrive(bars.kv_empty + 8 * ((abs0 + 2 * k) % C::STAGES));                        // K_k
-                                if (k >= 2) mbar_arrive(bars.kv_empty + 8 * ((abs0 + 2 * (k - 2) + 1) % C::STAGES));  // V_{k-2}
-                                if (k + 1 == it.tiles) mbar_arrive(bars.q_empty);   // that was the item's last Q K^T
-                            } else {
-                                ok = mbar_wait_bounded(bars.o_full + 8, o1_phase, abort_ptr, WAIT_LIMIT_NS);
-                                if (!ok) break;
-                                o1_phase ^= 1u;
-                                if (k >= 2) mbar_arrive(bars.kv_empty + 8 * ((abs0 + 2 * (k - 2) + 1) % C::STAGES));  // V_{tiles-2}
-                                mbar_arrive(bars.kv_empty + 8 * ((abs0 + 2 * (k - 1) + 1) % C::STAGES));              // V_{tiles-1}
-                            }
-#pragma unroll
-                            for (int q = 0; q < ATTN_NQ; ++q)
-                                ok = ok && mbar_wait_bounded(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_NS);
-                            p_phase ^= 1u;
-                        }
-                    }
-                    abs0 += 2u * (uint32_t)it.tiles;
-                }
+                // (D = 64 has no watcher: this warp is the second MMA warp there)
             } else {
             // It also hands the ring stages (and Q's place) back to the producer, so that the MMA thread issues no
             // commit for that: the commit that closes the group of query tile 1 -- s_full[1], or o_full[1] after the
@@ -496,27 +519,27 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 if (!decode_work<FUSED>(p, npairs, w, it)) continue;
                 ring.advance();   // K_0 of the item: the MMA thread waits for that one itself
                 for (int t = 0; t < it.tiles && ok; ++t) {
-                    ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
+                    ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_CYCLES);
                     ring.advance();
                     if (ok && t + 1 < it.tiles) {
-                        ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_NS);
+                        ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_CYCLES);
                         ring.advance();
                     }
                     if (!ok) break;
                     mbar_arrive(bars.p_full);
                     // S_1 of tile t is complete: the first Q K^T (t = 0) or the groups of tile t - 1 are done
-                    ok = mbar_wait_bounded(bars.s_full + 8, s1_phase, abort_ptr, WAIT_LIMIT_NS);
+                    ok = mbar_wait_bounded(bars.s_full + 8, s1_phase, abort_ptr, WAIT_LIMIT_CYCLES);
                     if (!ok) break;
                     s1_phase ^= 1u;
                     if (t > 0) { mbar_arrive(bars.kv_empty + 8 * rel.st); rel.advance(); }   // V_{t-1}
                     mbar_arrive(bars.kv_empty + 8 * rel.st); rel.advance();                   // K_t
                     if (t + 1 == it.tiles) mbar_arrive(bars.q_empty);                         // that was the item's last Q K^T
                     // one arrival per phase: wait for the phase to close before the next one
-                    ok = mbar_wait_bounded(bars.p_full, p_phase, abort_ptr, WAIT_LIMIT_NS);
+                    ok = mbar_wait_bounded(bars.p_full, p_phase, abort_ptr, WAIT_LIMIT_CYCLES);
                     p_phase ^= 1u;
                 }
                 if (!ok) break;
-                ok = mbar_wait_bounded(bars.o_full + 8, o1_phase, abort_ptr, WAIT_LIMIT_NS);   // the last PVs are done
+                ok = mbar_wait_bounded(bars.o_full + 8, o1_phase, abort_ptr, WAIT_LIMIT_CYCLES);   // the last PVs are done
                 if (!ok) break;
                 o1_phase ^= 1u;
                 mbar_arrive(bars.kv_empty + 8 * rel.st); rel.advance();                       // V of the last tile
@@ -538,7 +561,6 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const uint32_t p_tmem = tmem_base + lane_addr + C::P_COL + q * C::P_STRIDE;   // D = 128: the same columns as S
         const uint32_t o_tmem = tmem_base + lane_addr + C::O_COL + q * D;
         uint32_t s_phase = 0, o_phase = 0, pv_phase = 0;
-        [[maybe_unused]] uint32_t go0_phase = 0;   // D = 64: parity of the current item's first phase of go[q]
         bool ok = true;
         StateT *o_state = static_cast<StateT *>(p.o_state);
 
@@ -546,23 +568,46 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             WorkItem it;
             if (!decode_work<FUSED>(p, npairs, w, it)) continue;
             float m_used = -INFINITY, l_sum = 0.f;
+            [[maybe_unused]] float rs_prev = 0.f;   // bf16 inputs: row sum of the previous tile's P
             for (int t = 0; t < it.tiles; ++t) {
                 const int valid = it.template tile<FUSED>(t).y;   // keys of this tile that count (issued before the wait)
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.s_full + 8 * q, s_phase, abort_ptr, WAIT_LIMIT_NS));
-                if (!ok) break;
+                // One vote tells that S_t has arrived for every lane and (bf16 inputs) that no row of the warp reached
+                // ROWSUM_TRIGGER with the previous tile's P.
+                const bool s_here = mbar_wait_bounded(bars.s_full + 8 * q, s_phase, abort_ptr, WAIT_LIMIT_CYCLES);
+                const bool fine = __all_sync(0xFFFFFFFFu, s_here && (FP16 || rs_prev < ROWSUM_TRIGGER));
                 s_phase ^= 1u;
                 tc_fence_after();
+                [[maybe_unused]] bool pv_waited = false;
+                if (!fine) {
+                    ok = __all_sync(0xFFFFFFFFu, s_here);
+                    if (!ok) break;
+                    if constexpr (!FP16) {
+                        // bf16 probabilities have fp32's exponent range, so a tile's P is exact whatever the reference, and
+                        // the reference can move after the fact: when the previous tile's row sum reached ROWSUM_TRIGGER, m
+                        // moves up by e = floor(log2(row sum)) binades and O and l are multiplied by 2^-e, which is exact.
+                        // Made here, a tile late, the move is off the S -> P chain and the logits of a tile never have to
+                        // be kept for a second pass.  (S_t complete tells that P_{t-1} V_{t-1} is -- D = 64: pv_done does.)
+                        if constexpr (C::PREFETCH) {
+                            ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_CYCLES));
+                            pv_phase ^= 1u;
+                            pv_waited = true;
+                            tc_fence_after();
+                        }
+                        const int e = move_reference<D>(o_tmem, rs_prev);
+                        m_used += (float)e;
+                        l_sum *= __int_as_float((127 - e) << 23);
+                    }
+                }
                 uint32_t s[4][32];   // this thread's row of S: 128 fp32 logits (before scaling)
                 tmem_ld_x32(s_tmem + 0, s[0]);
                 tmem_ld_x32(s_tmem + 32, s[1]);
                 tmem_ld_x32(s_tmem + 64, s[2]);
                 tmem_ld_x32(s_tmem + 96, s[3]);
                 tmem_wait_ld();
-                bool p_place_free = !C::PREFETCH || t == 0;   // D = 64: P's columns may still be read by the previous tile's PV
+                bool p_place_free = !C::PREFETCH || t == 0 || pv_waited;   // D = 64: P's columns may still be read by the previous tile's PV
                 if constexpr (C::PREFETCH) {
                     tc_fence_before();
-                    mbar_arrive(bars.p_full + 8 * q);               // S_t has been read: Q K_{t+1}^T may overwrite it
-                    if (t == 0) mbar_arrive(bars.p_full + 8 * q);   // stands in for "P_{-1} stored"
+                    mbar_arrive(bars.s_free + 8 * q);   // S_t has been read: Q K_{t+1}^T may overwrite it
                 }
                 if (valid < ATTN_TILE) {
 #pragma unroll
@@ -606,7 +651,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         }
                         if constexpr (C::PREFETCH) {
                             if (!p_place_free) {   // PV of tile t-1 is done with P's columns
-                                ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_NS));
+                                ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_CYCLES));
                                 pv_phase ^= 1u;
                                 p_place_free = true;
                                 tc_fence_after();
@@ -619,55 +664,51 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 };
                 if (t == 0) m_used = row_max() * p.scale_log2;   // first tile: no earlier maximum to lean on
                 float rs = exp_pass(m_used);
-                // (the negated comparison also catches inf / NaN after an overflow)
-                if (t > 0 && __any_sync(0xFFFFFFFFu, !(rs < ROWSUM_TRIGGER))) {
-                    const float m_tile = row_max() * p.scale_log2;
-                    const bool need = (m_tile - m_used > RESCALE_THRESHOLD);
-                    if (__any_sync(0xFFFFFFFFu, need)) {
-                        const float alpha = need ? ex2_approx(m_used - m_tile) : 1.0f;
-                        if (need) m_used = m_tile;
-                        l_sum *= alpha;
-                        tmem_wait_st();
+                if constexpr (FP16) {
+                    // (the negated comparison also catches inf / NaN after an overflow)
+                    if (t > 0 && __any_sync(0xFFFFFFFFu, !(rs < ROWSUM_TRIGGER))) {
+                        // fp16 probabilities overflow at 2^16: take the tile's own maximum and compute P again
+                        const float m_tile = row_max() * p.scale_log2;
+                        const bool need = (m_tile - m_used > RESCALE_THRESHOLD);
+                        if (__any_sync(0xFFFFFFFFu, need)) {
+                            const float alpha = need ? ex2_approx(m_used - m_tile) : 1.0f;
+                            if (need) m_used = m_tile;
+                            l_sum *= alpha;
+                            tmem_wait_st();
 #pragma unroll
-                        for (int c0 = 0; c0 < D; c0 += 32) {
-                            uint32_t o[32];
-                            tmem_ld_x32(o_tmem + c0, o);
-                            tmem_wait_ld();
+                            for (int c0 = 0; c0 < D; c0 += 32) {
+                                uint32_t o[32];
+                                tmem_ld_x32(o_tmem + c0, o);
+                                tmem_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                            tmem_st_x32(o_tmem + c0, o);
+                                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                                tmem_st_x32(o_tmem + c0, o);
+                            }
+                            rs = exp_pass(m_used);
                         }
-                        rs = exp_pass(m_used);
                     }
                 }
                 l_sum += rs;
+                if constexpr (!FP16) rs_prev = rs;
                 tmem_wait_st();
                 tc_fence_before();
-                if constexpr (C::PREFETCH) {
-                    // "P_0 stored" belongs to phase 1 of go[q].  From tile 1 on, the wait for pv_done keeps a thread from
-                    // getting here before phase t has closed; at tile 0 nothing does, and an arrival made while phase 0
-                    // is still open would be counted in place of a slower thread's "S_0 read" or of the watcher's.
-                    if (t == 0) {
-                        ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.p_full + 8 * q, go0_phase, abort_ptr, WAIT_LIMIT_NS));
-                        if (!ok) break;
-                    }
-                }
                 mbar_arrive(bars.p_full + 8 * q);
                 if (!ok) break;
             }
             if (!ok) break;
-            if constexpr (C::PREFETCH) {
-                mbar_arrive(bars.p_full + 8 * q);   // closes the last phase (no further S to read)
-                go0_phase ^= (uint32_t)(it.tiles + 1) & 1u;   // the item took tiles + 1 phases of go[q]
-            }
             // epilogue: OUT_ij = O / l, LSE_ij = ln2 * (m + log2 l); rows beyond the partition are dropped
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.o_full + 8 * q, o_phase, abort_ptr, WAIT_LIMIT_NS));
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.o_full + 8 * q, o_phase, abort_ptr, WAIT_LIMIT_CYCLES));
             if (!ok) break;
             o_phase ^= 1u;
             tc_fence_after();
             const int row_in_block = q * ATTN_TILE + row_in_tile;
             const bool row_valid = row_in_block < it.n_q;
             const float inv_l = 1.0f / l_sum;
+            if constexpr (!FP16) {
+                // a sum that is not finite: within one K/V tile a logit rose more than about 120 binades above the
+                // reference (exp2 overflowed); the launch's states are not valid (dt_poll: DT_ERR_RANGE)
+                if (row_valid && !(l_sum <= 3.0e38f)) atomicOr(p.status, STATUS_LOGIT_RANGE);
+            }
             const float lse_fresh = 0.69314718055994530942f * (m_used + log2f(l_sum));
             if constexpr (FUSED) {
                 // fresh state (+) composed reuse state (Eq. 2), straight to the attention output

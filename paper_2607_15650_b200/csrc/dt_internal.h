@@ -12,7 +12,7 @@
 namespace dt {
 
 // Device status word bits (read by dt_poll).
-enum : int { STATUS_REUSE_EMPTY = 1, STATUS_WAIT_TIMEOUT = 2 };
+enum : int { STATUS_REUSE_EMPTY = 1, STATUS_WAIT_TIMEOUT = 2, STATUS_LOGIT_RANGE = 4 };
 
 constexpr int PLAN_CHUNK_ROWS = 1024;  // rows of one (b, h, partition) handled by one dt_plan block
 constexpr int ATTN_TILE = 128;         // query rows per TMEM accumulator / keys per KV tile

@@ -565,3 +565,43 @@ def test_growing_logits_move_the_reference_maximum(D, fp16):
             check_o(ctx.o_state[j, 0, h].float().cpu().numpy(), so, f"growing logits state {j}")
             check_lse(ctx.lse_state[j, 0, h].cpu().numpy(), sl, f"growing logits state {j}")
     assert lse_max > 150.0      # the case really is extreme
+
+
+def test_logit_jump_beyond_fp32_range_is_reported():
+    """bf16 inputs: the reference of a row moves after the fact by whole binades, which is exact as long as exp2 of a
+    logit taken against the previous tiles' reference stays inside fp32.  A logit that rises by more than that within
+    one K/V tile (here about 430 binades) cannot be represented: the launch reports DT_ERR_RANGE through dt_poll instead
+    of returning a wrong state, and the context stays usable.  fp16 inputs take the tile's own maximum first and have
+    no such limit."""
+    B, H, D, L, P = 1, 1, 64, 512, 1
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(3)
+    u = np.zeros(D, np.float32); u[:4] = 0.5
+    q = 0.1 * rng.standard_normal((B, L, H, D)).astype(np.float32) + 10.0 * u
+    k = 0.1 * rng.standard_normal((B, L, H, D)).astype(np.float32)
+    k[0, 128:, 0, :] += 30.0 * u          # keys of the second tile onwards: logits about 300 (natural units) higher
+    v = rng.standard_normal((B, L, H, D)).astype(np.float32)
+    off = np.array([0, L], dtype=np.int32)
+    mask = torch.ones(P * P, dtype=torch.uint8, device=dev)
+    for fp16 in (False, True):
+        dt = torch.float16 if fp16 else torch.bfloat16
+        qt, kt, vt = (torch.from_numpy(x).to(dt).to(dev) for x in (q, k, v))
+        ctx = binding.Context(B, H, D, L, off, 1.0, input_dtype=binding.DT_INPUT_FP16 if fp16 else binding.DT_INPUT_BF16)
+        out = torch.empty((B, L, H, D), dtype=dt, device=dev)
+        lse = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+        ctx.dt_attn_states(qt, kt, vt, mask, 0)
+        ctx.dt_state_merge(out, lse)
+        if not fp16:
+            with pytest.raises(binding.DitangoError) as ei:
+                ctx.dt_poll()
+            assert ei.value.status == binding.DT_ERR_RANGE
+            ctx.dt_poll()                       # the word was cleared: the context is usable again
+            kt = torch.from_numpy(k * 0.1).to(dt).to(dev)   # the same shape of inputs with a jump of 43 binades
+            ctx.dt_attn_states(qt, kt, vt, mask, 1)
+            ctx.dt_state_merge(out, lse)
+        ctx.dt_poll()
+        qb, kb, vb = (inputs.bf16_bits(x) for x in (qt, kt, vt))
+        rows = np.arange(L, dtype=np.int32)
+        ro, rl = orc.full_attention(qb, kb, vb, 1.0, 0, 0, rows, fp16=fp16)
+        check_o(out[0, :, 0].float().cpu().numpy(), ro, "logit jump")
+        check_lse(lse[0, 0].cpu().numpy(), rl, "logit jump")
