@@ -36,6 +36,9 @@ sys.path.insert(0, ROOT)
 
 from paper_2607_15650_b200 import inputs  # noqa: E402
 
+# --policy alg1: (eps_local, cache ratio R) per workload, chosen so that the online policy computes about the share of
+# pairs the fixed-fraction plans of the workload compute
+ALG1_DEFAULTS = {"c3_wan720p": (0.0075, 0.85)}
 METRIC = "effective_attn_tflops"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "c3_wan720p"
@@ -103,11 +106,19 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# DRAM traffic of attn_states_kernel per (head, COMPUTE pair) of the c3-shaped tiles, from the ncu capture
-# summarised under profiles/ (kernel attn_states, workload c3_wan720p, 4 heads): (239.7 MB read + 941.4 MB written)
-# / (4 heads x 102 pairs).
-# Traffic grows in proportion to heads x pairs (the pair states written dominate it).
-NCU_ATTN_TRAFFIC_PER_HEAD_PAIR = {"c3_wan720p": (239.7e6 + 941.4e6) / (4 * 102)}
+def ncu_attn_traffic(workload: str):
+    """DRAM bytes (read + written) of one attn_states_kernel launch per (head, COMPUTE pair), from the ncu capture
+    that profiles/attn_states_traffic.json names (a capture on a few heads of the workload; the traffic grows in
+    proportion to heads x pairs because the pair states written dominate it).  None if there is no capture."""
+    path = os.path.join(ROOT, "profiles", "attn_states_traffic.json")
+    if not os.path.exists(path):
+        return None, None
+    with open(path) as fh:
+        rec = json.load(fh).get(workload)
+    if not rec:
+        return None, None
+    per = (rec["dram_bytes_read"] + rec["dram_bytes_written"]) / (rec["heads"] * rec["computed_pairs"])
+    return per, rec["capture"]
 
 
 def full_flops(wl) -> float:
@@ -155,6 +166,38 @@ def dist_info():
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     return world, rank, local
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_ranks(n: int, argv, script=None) -> int:
+    """`--gpus N` without a launcher around it: start N ranks of this script (one per GPU) under torch's launcher on
+    127.0.0.1 and return its exit code.  With WORLD_SIZE already in the environment the caller is a rank and runs
+    the bench itself instead."""
+    script = script or os.path.abspath(__file__)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port()), script] + list(argv)
+    return subprocess.run(cmd).returncode
+
+
+def probe_world(args):
+    """What a rank of `--gpus N --probe-world` does: join a gloo group on the CPU and let rank 0 print the world size
+    (the launch path of the multi-GPU bench without a GPU)."""
+    import torch.distributed as dist
+    world, rank, local = dist_info()
+    dist.init_process_group("gloo")
+    t = torch.ones(1, dtype=torch.float64)
+    dist.all_reduce(t)
+    if rank == 0:
+        print(json.dumps({"probe": "world", "world_size": dist.get_world_size(), "ranks_counted": int(t.item()),
+                          "n_gpus": args.gpus}))
+    dist.barrier()
+    dist.destroy_process_group()
 
 
 def max_over_ranks(value: float, world: int, device=None) -> float:
@@ -281,6 +324,31 @@ def run_cuda(args, wl):
     sums = torch.empty(PP, dtype=torch.float64, device=dev)
     frac = args.fraction if args.fraction is not None else wl.fractions[-1]
     stream = torch.cuda.current_stream()
+
+    if args.policy == "alg1":
+        if world > 1 or args.group_size != 1:
+            raise SystemExit("--policy alg1 is measured on one GPU with the pair cache")
+        dflt = ALG1_DEFAULTS.get(wl.name, (0.01, 0.8))
+        eps_local = args.eps_local if args.eps_local is not None else dflt[0]
+        ratio = args.cache_ratio if args.cache_ratio is not None else dflt[1]
+        n = max(args.steps, 2)
+        measure_alg1(binding, dev, wl, ctx, steps_in, max(args.warmup, n // 2), eps_local, ratio, host_replay=False)
+        rec = measure_alg1(binding, dev, wl, ctx, steps_in, n, eps_local, ratio, host_replay=not args.no_e2e)
+        line = {"metric": METRIC, "value": rec["effective_tflops"], "unit": UNIT, "n_gpus": 1, "steps": n,
+                "warmup": max(args.warmup, n // 2), "ms_per_step": rec["step_ms_mean"], "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
+                "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "D": wl.D, "L": wl.L, "P": wl.P,
+                           "policy": "alg1", "state_dtype": args.state_dtype,
+                           "step": "dt_attn_local + dt_planner_step + dt_attn_states + dt_state_merge + dt_planner_commit",
+                           "l2": "inputs and state cache larger than L2; no flush"},
+                "clocks": rec["clocks"],
+                "e2e": ({"value": full_flops(wl) / 1e12 / (rec["e2e_step_ms_mean"] / 1e3), "unit": UNIT,
+                         "ms_per_step": rec["e2e_step_ms_mean"], "h2d_bytes_per_step": 3 * wl.B * wl.L * wl.H * wl.D * 2 + wl.P * wl.P,
+                         "d2h_bytes_per_step": wl.B * wl.L * wl.H * (wl.D * 2 + 4), "includes": rec["e2e_includes"]}
+                        if "e2e_step_ms_mean" in rec else None),
+                "gpu_launches": None, "alg1": rec}
+        print(json.dumps(line))
+        return
 
     def plan(mask_buf):
         if args.shard_heads:   # local sums -> all-reduce of P*S doubles -> the same plan on every rank
@@ -445,6 +513,7 @@ def run_cuda(args, wl):
         cpu = {"value": eff, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds": secs}
 
     attn_avg_ms = float(np.mean(attn_ms))
+    traffic_per, traffic_src = ncu_attn_traffic(args.workload)
     achieved = comp_fl / 1e12 / (attn_avg_ms / 1e3)
     peak = peaks["bf16_tflops_sustained"]
     line = {
@@ -467,10 +536,10 @@ def run_cuda(args, wl):
         "gpu_launches": launches,
         "roofline": {"kernel": "attn_states_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
                      "unit": "TFLOP/s", "frac": achieved / peak,
-                     "traffic": (NCU_ATTN_TRAFFIC_PER_HEAD_PAIR[args.workload] * wl.H * n_comp
-                                 if args.workload in NCU_ATTN_TRAFFIC_PER_HEAD_PAIR and args.state_dtype == "fp32" and g == 1
+                     "traffic": (traffic_per * wl.H * n_comp
+                                 if traffic_per is not None and args.state_dtype == "fp32" and g == 1 and args.dtype == "bf16"
                                  else None),
-                     "traffic_note": "bytes per launch, ncu dram read+write of a 4-head capture scaled by heads x pairs",
+                     "traffic_note": f"bytes per launch: ncu dram read + write of {traffic_src}, scaled by heads x pairs",
                      "peak_source": f"{peaks['source']} bf16 sustained", "frac_of_burst": achieved / peaks["bf16_tflops"],
                      "frac_of_nominal_2250": achieved / 2250.0, "launch_ms": attn_avg_ms,
                      "algorithmic_flops_per_launch": comp_fl},
@@ -479,6 +548,8 @@ def run_cuda(args, wl):
             "attn_ms": attn_avg_ms, "merge_ms": float(np.mean(merge_ms)), "plan_ms": float(np.mean(plan_ms)),
             "merge_gbs": merge_bytes(wl, sbytes, S) / 1e9 / (float(np.mean(merge_ms)) / 1e3),
             "merge_frac_of_hbm": merge_bytes(wl, sbytes, S) / 1e9 / (float(np.mean(merge_ms)) / 1e3) / peaks["hbm_gbs"],
+            "merge_frac_of_nominal_8000": merge_bytes(wl, sbytes, S) / 1e9 / (float(np.mean(merge_ms)) / 1e3) / 8000.0,
+            "merge_note": "the measured peak is a plain copy (half reads, half writes); a kernel that mostly reads can exceed it",
             "plan_gbs": plan_bytes(wl, S) / 1e9 / (float(np.mean(plan_ms)) / 1e3),
             "hbm_peak_gbs": peaks["hbm_gbs"], "compose_once_ms": compose_ms,
         },
@@ -489,7 +560,183 @@ def run_cuda(args, wl):
                            "full_attention_one_pass_ms": dense_ms,
                            "full_attention_one_pass_tflops": full_flops(wl) / 1e12 / (dense_ms / 1e3)},
     }
+    # ---- further records of the default line, measured after the headline loop (not part of `value`)
+    default_shape = (not (args.fused or args.composed or args.shard_heads) and args.group_size == 1 and args.heads is None
+                     and args.state_dtype == "fp32" and args.dtype == "bf16" and args.workload == DEFAULT_WORKLOAD
+                     and args.fraction is None)
+    if default_shape and not args.no_extra and world == 1:
+        extras = []
+        extras.append(measure_config(binding, dev, wl, frac, fused=True, peaks=peaks, ctx=ctx, steps_in=steps_in))
+        eps_local, ratio = ALG1_DEFAULTS[wl.name]
+        extras.append(measure_alg1(binding, dev, wl, ctx, steps_in, wl.steps, eps_local, ratio))
+        ctx.close()
+        del steps_in, out, lse
+        torch.cuda.empty_cache()
+        for name, f in (("c1_cogvideox", 0.5), ("c4_hunyuan720p", 0.125)):
+            extras.append(measure_config(binding, dev, inputs.WORKLOADS[name], f, peaks=peaks))
+            torch.cuda.empty_cache()
+        line["extra_configs"] = extras
     print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------ further records
+def _ev():
+    return torch.cuda.Event(enable_timing=True)
+
+
+def measure_config(binding, dev, wl, fraction, steps=5, warmup=3, fused=False, state_dtype="fp32", peaks=None, ctx=None,
+                   steps_in=None):
+    """One more configuration, outside the timed headline loop: anchor step + plan at `fraction`, then `steps` timed
+    selective steps through dt_attn_states + dt_state_merge + dt_plan, or (fused) through dt_compose_reuse once and
+    dt_attn_fused per step.  Returns a record with the kernels' times, TFLOP/s on the computed blocks, the merge's GB/s
+    and the clocks sampled meanwhile."""
+    sbytes = 2 if state_dtype == "bf16" else 4
+    own = ctx is None
+    if own:
+        ctx = binding.Context(wl.B, wl.H, wl.D, wl.L, wl.offsets(), wl.scale,
+                              binding.DT_STATE_BF16 if state_dtype == "bf16" else binding.DT_STATE_FP32, dev.index or 0)
+        gen = inputs.StepInputs(wl, seed=0, device=dev)
+        steps_in = [gen.next() for _ in range(wl.steps)]
+        del gen
+    stream = torch.cuda.current_stream()
+    PP = wl.P * wl.P
+    out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    ones = torch.ones(PP, dtype=torch.uint8, device=dev)
+    masks = [torch.ones(PP, dtype=torch.uint8, device=dev), torch.ones(PP, dtype=torch.uint8, device=dev)]
+    q, k, v = steps_in[0]
+    ctx.dt_attn_states(q, k, v, ones, 0)
+    ctx.dt_state_merge(out, lse)
+    ctx.dt_plan(masks[0], target_fraction=fraction)
+    comp_o = comp_l = None
+    if fused:
+        comp_o = torch.empty((wl.B, wl.H, wl.L, wl.D), dtype=ctx.o_state.dtype, device=dev)
+        comp_l = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+        ctx.dt_compose_reuse(masks[0], comp_o, comp_l)
+    torch.cuda.synchronize()
+    ctx.dt_poll()
+    cur, t, timers = 0, 1, []
+    sampler = ClockSampler(dev.index or 0)
+    for it in range(warmup + steps):
+        if it == warmup:
+            torch.cuda.synchronize()
+            sampler.start()
+        q, k, v = steps_in[1 + (t % (wl.steps - 1))] if wl.steps > 1 else steps_in[0]
+        e = [_ev() for _ in range(4)]
+        e[0].record(stream)
+        if fused:
+            ctx.dt_attn_fused(q, k, v, masks[cur], comp_o, comp_l, out, lse)
+            for i in (1, 2, 3):
+                e[i].record(stream)
+        else:
+            ctx.dt_attn_states(q, k, v, masks[cur], t)
+            e[1].record(stream)
+            ctx.dt_state_merge(out, lse)
+            e[2].record(stream)
+            ctx.dt_plan(masks[cur ^ 1], target_fraction=fraction)
+            e[3].record(stream)
+            cur ^= 1
+        t += 1
+        if it >= warmup:
+            timers.append(e)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ctx.dt_poll()
+    mask_np = masks[cur].cpu().numpy()
+    n_comp = int((mask_np != 0).sum())
+    comp_fl = computed_flops(wl, mask_np)
+    attn = float(np.mean([e[0].elapsed_time(e[1]) for e in timers]))
+    merge = float(np.mean([e[1].elapsed_time(e[2]) for e in timers]))
+    plan = float(np.mean([e[2].elapsed_time(e[3]) for e in timers]))
+    step = float(np.mean([e[0].elapsed_time(e[3]) for e in timers]))
+    rec = {"workload": wl.name, "computed_pairs": n_comp, "computed_pair_fraction": n_comp / PP, "state_dtype": state_dtype,
+           "step": "dt_compose_reuse once + dt_attn_fused per step" if fused else "dt_attn_states + dt_state_merge + dt_plan",
+           "steps": steps, "warmup": warmup, "step_ms": step, "attn_ms": attn,
+           "tflops_on_computed": comp_fl / 1e12 / (attn / 1e3),
+           "effective_tflops": full_flops(wl) / 1e12 / (step / 1e3), "clocks": clocks,
+           "cache_gb": wl.P * wl.B * wl.H * wl.L * (wl.D * sbytes + 4) / 1e9}
+    if peaks is not None:
+        rec["frac_of_sustained_peak"] = rec["tflops_on_computed"] / peaks["bf16_tflops_sustained"]
+    if not fused:
+        rec.update({"merge_ms": merge, "plan_ms": plan, "merge_gbs": merge_bytes(wl, sbytes) / 1e9 / (merge / 1e3)})
+    if own:
+        ctx.close()
+    return rec
+
+
+def measure_alg1(binding, dev, wl, ctx, steps_in, n_steps, eps_local, cache_ratio, host_replay=True):
+    """The step loop of Algorithm 1 with the anchors decided on the device: per step dt_attn_local -> dt_planner_step ->
+    dt_attn_states on the remaining COMPUTE pairs -> dt_state_merge -> dt_planner_commit (which refreshes w, alpha and
+    the snapshot on anchors only).  The host reads the anchor flag and the mask after the timed region only."""
+    stream = torch.cuda.current_stream()
+    P = wl.P
+    PP = P * P
+    out = torch.empty((wl.B, wl.L, wl.H, wl.D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    snap_o = torch.zeros((wl.B, wl.H, wl.L, wl.D), dtype=ctx.o_state.dtype, device=dev)
+    snap_l = torch.zeros((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
+    ctx.dt_planner_init(snap_o, snap_l, group_size=1, eps_initial=0.0, eps_local=eps_local, cache_ratio=cache_ratio)
+    not_eye = (1 - torch.eye(P, dtype=torch.uint8, device=dev)).reshape(-1)
+    masks = [torch.zeros(PP, dtype=torch.uint8, device=dev) for _ in range(n_steps)]
+    rests = [torch.zeros(PP, dtype=torch.uint8, device=dev) for _ in range(n_steps)]
+    flags = torch.zeros(n_steps, dtype=torch.int32, device=dev)
+    drel = torch.zeros(n_steps, dtype=torch.float64, device=dev)
+    evs = []
+    sampler = ClockSampler(dev.index or 0)
+    torch.cuda.synchronize()
+    sampler.start()
+    for t in range(n_steps):
+        q, k, v = steps_in[t % len(steps_in)]
+        e = [_ev() for _ in range(6)]
+        e[0].record(stream)
+        ctx.dt_attn_local(q, k, v, t)
+        e[1].record(stream)
+        ctx.dt_planner_step(masks[t], flags[t:t + 1], None, drel[t:t + 1])
+        e[2].record(stream)
+        torch.mul(masks[t], not_eye, out=rests[t])          # the local pairs are done already
+        ctx.dt_attn_states(q, k, v, rests[t], t)
+        e[3].record(stream)
+        ctx.dt_state_merge(out, lse)
+        e[4].record(stream)
+        ctx.dt_planner_commit()
+        e[5].record(stream)
+        evs.append(e)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ctx.dt_poll()
+    fl = flags.cpu().numpy().astype(bool)
+    ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(5)] for e in evs])      # local, plan, rest, merge, commit
+    step_ms = ms.sum(axis=1)
+    frac = np.array([float(m.sum().item()) / PP for m in masks])
+    planner_ms = ms[:, 1] + ms[:, 4]
+    rec = {"workload": wl.name, "policy": "Algorithm 1 on the device", "eps_local": eps_local, "cache_ratio": cache_ratio,
+           "steps": n_steps, "anchors": int(fl.sum()), "anchor_steps": [int(i) for i in np.nonzero(fl)[0]],
+           "computed_pair_fraction_per_step": [round(float(x), 4) for x in frac],
+           "mean_computed_pair_fraction": float(frac.mean()),
+           "step_ms_mean": float(step_ms.mean()),
+           "step_ms_anchor": float(step_ms[fl].mean()) if fl.any() else None,
+           "step_ms_selective": float(step_ms[~fl].mean()) if (~fl).any() else None,
+           "planner_ms_anchor": float(planner_ms[fl].mean()) if fl.any() else None,
+           "planner_ms_selective": float(planner_ms[~fl].mean()) if (~fl).any() else None,
+           "planner_share_of_all_compute_pass": (float(planner_ms[fl].mean() / step_ms[fl].mean()) if fl.any() else None),
+           "local_drift_rel_per_step": [round(float(x), 5) for x in drel.cpu().numpy()],
+           "effective_tflops": full_flops(wl) / 1e12 / (float(step_ms.mean()) / 1e3), "clocks": clocks}
+    if host_replay:
+        # the same sequence of plans end to end from host buffers (dt_step_host; the planner's kernels are not part of it)
+        ws = torch.empty(binding.dt_step_host_workspace_bytes(ctx.cfg), dtype=torch.uint8, device=dev)
+        oh = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+        lh = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+        host_in = [tuple(x.cpu().pin_memory() for x in steps_in[i]) for i in range(min(2, len(steps_in)))]
+        times = []
+        for t in range(n_steps):
+            qh, kh, vh = host_in[t % len(host_in)]
+            mh = masks[t].cpu()
+            t0 = time.perf_counter()
+            ctx.dt_step_host(qh, kh, vh, mh, n_steps + t, oh, lh, ws)
+            times.append(time.perf_counter() - t0)
+        rec["e2e_step_ms_mean"] = 1e3 * float(np.mean(times[1:]))
+        rec["e2e_includes"] = "dt_step_host with the recorded plan of every step: H2D q,k,v,mask + attention + merge + D2H out,lse"
+    return rec
 
 
 def main():
@@ -517,7 +764,17 @@ def main():
                          "instead of running N independent replicas")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="leave out the extra_configs records of the default line")
+    ap.add_argument("--policy", default="fraction", choices=["fraction", "alg1"],
+                    help="alg1: the step loop of Algorithm 1 (anchors decided online) instead of a fixed target fraction")
+    ap.add_argument("--eps-local", type=float, default=None, help="--policy alg1: anchor threshold on the local drift")
+    ap.add_argument("--cache-ratio", type=float, default=None, help="--policy alg1: R, the share of units kept in the cache")
+    ap.add_argument("--probe-world", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
+    if args.probe_world:
+        return probe_world(args)
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     wl = inputs.WORKLOADS[args.workload]
     if args.heads is not None:

@@ -231,6 +231,7 @@ dt_status dt_destroy(dt_ctx *ctx) {
     cudaFree(ctx->planner_state_dev);
     cudaFree(ctx->planner_local_partials_dev);
     cudaFree(ctx->planner_norm_partials_dev);
+    cudaFree(ctx->attn_norm_partials_dev);
     for (cudaEvent_t ev : ctx->events) cudaEventDestroy(ev);
     if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
     if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
@@ -280,6 +281,7 @@ dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const v
     p.status = ctx->status_dev;
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;
+    p.norm_partials = ctx->attn_norm_partials_dev;
     p.B = c.B; p.H = c.H; p.L = c.L; p.P = c.P; p.S = ctx->S;
     p.h0 = h0; p.H_launch = hc < 0 ? c.H : hc;
     p.in_fp16 = c.input_dtype == DT_INPUT_FP16;
@@ -670,6 +672,8 @@ dt::PlannerParams planner_params(dt_ctx *ctx) {
     p.nonempty = ctx->nonempty_dev;
     p.local_partials = ctx->planner_local_partials_dev;
     p.norm_partials = ctx->planner_norm_partials_dev;
+    p.attn_norm_partials = ctx->attn_norm_partials_dev;
+    p.qblocks = ctx->qblocks_max;
     p.w_partials = ctx->plan_partials_dev;
     p.P = c.P; p.S = ctx->S; p.BH = c.B * c.H; p.L = c.L; p.D = c.D; p.chunks = ctx->plan_chunks;
     p.group_size = ctx->planner_group_size;
@@ -701,6 +705,9 @@ dt_status dt_planner_init(dt_ctx *ctx, const dt_planner_config *pc, void *snap_o
         bool ok = cudaMalloc(&ctx->planner_state_dev, sizeof(dt::PlannerState)) == cudaSuccess;
         ok = ok && cudaMalloc(&ctx->planner_local_partials_dev, BH * c.P * ctx->plan_chunks * 2 * sizeof(float)) == cudaSuccess;
         ok = ok && cudaMalloc(&ctx->planner_norm_partials_dev, BH * c.P * ctx->plan_chunks * ctx->S0 * sizeof(float)) == cudaSuccess;
+        const size_t attn_norm_bytes = BH * c.P * ctx->S0 * ctx->qblocks_max * (dt::ATTN_NQ * 4) * sizeof(float);
+        ok = ok && cudaMalloc(&ctx->attn_norm_partials_dev, attn_norm_bytes) == cudaSuccess;
+        ok = ok && cudaMemsetAsync(ctx->attn_norm_partials_dev, 0, attn_norm_bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess;
         if (!ok) return fail(ctx, DT_ERR_CUDA, "planner scratch allocation failed");
     }
     ctx->snap_o = snap_o_dev;

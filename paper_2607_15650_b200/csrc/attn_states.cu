@@ -57,10 +57,16 @@ static_assert((REGS_SOFTMAX - LAUNCH_REGS) * NUM_SOFTMAX_THREADS <= (LAUNCH_REGS
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // SM clock cycles: about 2 s
 constexpr float ROWSUM_TRIGGER = 512.0f;   // a row sum of P at or above this sends the tile through the slow path
 constexpr float RESCALE_THRESHOLD = 1.0f;  // log2 units: in the slow path the reference moves if the maximum grew by more
-#ifndef DT_POLY_PER_8
-#define DT_POLY_PER_8 0
+// Key pairs (of every 8) whose exp2 runs as a cubic on the FMA pipe instead of the MUFU.  D = 64 is bound by the
+// exponentials (2048 MUFU cycles per 256 x 128 tile pair against 1536 of MMA issue), and one pair in eight measured
+// +2 % there (two in eight: no further gain); at D = 128 the softmax is a link of the S -> P -> S chain and the extra
+// dependent instructions cost what the MUFU time saves.
+#ifndef DT_POLY_PER_8_D64
+#define DT_POLY_PER_8_D64 1
 #endif
-constexpr int POLY_PER_8 = DT_POLY_PER_8;           // key pairs (of every 8) whose exp2 runs on the FMA pipe
+#ifndef DT_POLY_PER_8_D128
+#define DT_POLY_PER_8_D128 0
+#endif
 
 template <int D>
 struct Cfg {
@@ -78,6 +84,7 @@ struct Cfg {
     // there P gets its own place (S0 | S1 | P0 | P1 | O0 | O1), so S may be overwritten as soon as the softmax has
     // read it and the next tile's Q K^T runs while this tile's exponentials are being taken.
     static constexpr bool PREFETCH = (D == 64);
+    static constexpr int POLY_PER_8 = (D == 64) ? DT_POLY_PER_8_D64 : DT_POLY_PER_8_D128;
     static constexpr int S_COL = 0;                                              // S tile q: S_COL + q*128
     static constexpr int P_COL = PREFETCH ? ATTN_NQ * 128 : 0;                   // P tile q: P_COL + q*(PREFETCH ? 64 : 128)
     static constexpr int P_STRIDE = PREFETCH ? 64 : 128;
@@ -644,7 +651,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         for (int c = half * 64; c < half * 64 + 64; c += 2) {
                             const float s0 = __uint_as_float(s[c >> 5][c & 31]), s1 = __uint_as_float(s[(c + 1) >> 5][(c + 1) & 31]);
                             const float2 x = __ffma2_rn(make_float2(s0, s1), sc2, nm2);
-                            const float2 pp = (((c >> 1) & 7) < POLY_PER_8) ? exp2_poly2(x)
+                            const float2 pp = (((c >> 1) & 7) < C::POLY_PER_8) ? exp2_poly2(x)
                                                                             : make_float2(ex2_approx(x.x), ex2_approx(x.y));
                             rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
                             pk[(c >> 1) & 31] = pack_half2<FP16>(pp.x, pp.y);
@@ -767,6 +774,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 const uint32_t my_row = stage + lane * 128;
                 const int rows_left = it.n_q - (row_in_block - lane);   // valid rows of this warp's 32
                 uint8_t *gbase = reinterpret_cast<uint8_t *>(o_state + (srow - lane) * D);   // row 0 of this warp
+                float row_sq = lse_fresh * lse_fresh;   // ||AS||^2 of this row: OUT and LSE stacked (Eq. 9)
 #pragma unroll
                 for (int c0 = 0; c0 < D; c0 += CH) {
                     uint32_t o[CH / 32][32];
@@ -781,17 +789,23 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     for (int c = 0; c < 8; ++c) {   // 16-byte piece c of this row's 128 bytes
                         uint4 v;
                         if constexpr (sizeof(StateT) == 4) {
-                            v.x = __float_as_uint(__uint_as_float(o[0][4 * c]) * inv_l);
-                            v.y = __float_as_uint(__uint_as_float(o[0][4 * c + 1]) * inv_l);
-                            v.z = __float_as_uint(__uint_as_float(o[0][4 * c + 2]) * inv_l);
-                            v.w = __float_as_uint(__uint_as_float(o[0][4 * c + 3]) * inv_l);
+                            const float f0 = __uint_as_float(o[0][4 * c]) * inv_l, f1 = __uint_as_float(o[0][4 * c + 1]) * inv_l;
+                            const float f2 = __uint_as_float(o[0][4 * c + 2]) * inv_l, f3 = __uint_as_float(o[0][4 * c + 3]) * inv_l;
+                            row_sq = fmaf(f0, f0, fmaf(f1, f1, fmaf(f2, f2, fmaf(f3, f3, row_sq))));
+                            v.x = __float_as_uint(f0); v.y = __float_as_uint(f1); v.z = __float_as_uint(f2); v.w = __float_as_uint(f3);
                         } else {
                             const uint32_t(&oo)[32] = o[(8 * c) / 32];
                             const int b0 = (8 * c) % 32;
-                            v.x = pack_bf16x2(__uint_as_float(oo[b0]) * inv_l, __uint_as_float(oo[b0 + 1]) * inv_l);
-                            v.y = pack_bf16x2(__uint_as_float(oo[b0 + 2]) * inv_l, __uint_as_float(oo[b0 + 3]) * inv_l);
-                            v.z = pack_bf16x2(__uint_as_float(oo[b0 + 4]) * inv_l, __uint_as_float(oo[b0 + 5]) * inv_l);
-                            v.w = pack_bf16x2(__uint_as_float(oo[b0 + 6]) * inv_l, __uint_as_float(oo[b0 + 7]) * inv_l);
+                            float f[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                f[u] = __uint_as_float(oo[b0 + u]) * inv_l;
+                                row_sq = fmaf(f[u], f[u], row_sq);
+                            }
+                            v.x = pack_bf16x2(f[0], f[1]);
+                            v.y = pack_bf16x2(f[2], f[3]);
+                            v.z = pack_bf16x2(f[4], f[5]);
+                            v.w = pack_bf16x2(f[6], f[7]);
                         }
                         const uint32_t dst = my_row + (uint32_t)((c ^ (lane & 7)) << 4);
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -810,6 +824,17 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     __syncwarp();
                 }
                 if (row_valid) p.lse_state[srow] = lse_fresh;
+                if (p.norm_partials != nullptr) {
+                    // the state norms Algorithm 1 wants at an anchor come out of this epilogue instead of a pass over the
+                    // cache: one partial per warp, summed by an xor butterfly (a fixed order: same bits every run)
+                    if (!row_valid) row_sq = 0.f;
+#pragma unroll
+                    for (int sft = 16; sft > 0; sft >>= 1) row_sq += __shfl_xor_sync(0xFFFFFFFFu, row_sq, sft);
+                    if (lane == 0) {
+                        const int qb = (it.q_row0 - p.off[it.i]) / (ATTN_NQ * ATTN_TILE);
+                        p.norm_partials[((((long long)it.bh * p.P + it.i) * p.S + it.slot) * p.qblocks_max + qb) * (ATTN_NQ * 4) + warp] = row_sq;
+                    }
+                }
             }
         }
         if (!ok && lane == 0) {

@@ -33,6 +33,9 @@ struct AttnParams {
     int32_t *status;          // device status word
     void *o_state;            // [S][B][H][L][D]
     float *lse_state;         // [S][B][H][L]
+    // Squared 2-norms of the states this launch writes (OUT and LSE stacked, Eq. 9), one partial sum per softmax
+    // warp: [B*H][P][S][qblocks_max][ATTN_NQ * 4], or null when no planner is attached.
+    float *norm_partials;
     int B, H, L, P, S;
     int in_fp16;              // q, k, v (and the fused output) are fp16 instead of bf16
     int h0, H_launch;         // heads [h0, h0 + H_launch) are processed by this launch (the whole range: 0, H)
@@ -119,6 +122,7 @@ struct PlanFinalParams {
 struct PlannerState {
     double w[DT_MAX_P * DT_MAX_P];       // partition importance weights of the last anchor (Eq. 8)
     double alpha[DT_MAX_P * DT_MAX_P];   // scale ratios of the last anchor (Eq. 9)
+    double nsq[DT_MAX_P * DT_MAX_P];     // scratch: squared state norms of the anchor being committed
     double eps;                          // current threshold (Eq. 13)
     int have_anchor;                     // an anchor has been committed
     int is_anchor;                       // the step being planned is an anchor
@@ -135,7 +139,9 @@ struct PlannerParams {
     const int32_t *off;           // device, P+1
     const uint32_t *nonempty;     // device, P words: slots that exist for the query partition
     float *local_partials;        // [BH][P][chunks][2]
-    float *norm_partials;         // [BH][P][chunks][S]
+    float *norm_partials;         // [BH][P][chunks][S]: norms taken by a pass over the cache (after a group compose)
+    const float *attn_norm_partials;   // [BH][P][S][qblocks][ATTN_NQ * 4]: norms emitted by the attention epilogue
+    int qblocks;
     const float *w_partials;      // [BH][P][chunks][S] from plan_partial_kernel
     uint8_t *mask;                // out, P*S
     int32_t *is_anchor_out;       // out, may be null
@@ -199,6 +205,7 @@ struct dt_ctx {
     dt::PlannerState *planner_state_dev = nullptr;
     float *planner_local_partials_dev = nullptr;
     float *planner_norm_partials_dev = nullptr;
+    float *attn_norm_partials_dev = nullptr;
     void *snap_o = nullptr;
     float *snap_lse = nullptr;
     int planner_group_size = 1;

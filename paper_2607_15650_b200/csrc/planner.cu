@@ -23,12 +23,30 @@ namespace {
 
 constexpr int PL_THREADS = 256;
 
+// 16 bytes of state elements as fp32 values: 4 (fp32 cache) or 8 (bf16 cache)
 template <typename T>
-__device__ __forceinline__ float to_f32(T x);
+struct Vec16;
 template <>
-__device__ __forceinline__ float to_f32<float>(float x) { return x; }
+struct Vec16<float> {
+    static constexpr int N = 4;
+    __device__ static __forceinline__ void load(const float *p, float (&v)[4]) {
+        const float4 x = __ldcs(reinterpret_cast<const float4 *>(p));
+        v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+    }
+};
 template <>
-__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+struct Vec16<__nv_bfloat16> {
+    static constexpr int N = 8;
+    __device__ static __forceinline__ void load(const __nv_bfloat16 *p, float (&v)[8]) {
+        const uint4 x = __ldcs(reinterpret_cast<const uint4 *>(p));
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            v[2 * e] = __uint_as_float(w[e] << 16);
+            v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+        }
+    }
+};
 
 // fixed-order block sum of two values per thread; result valid in thread 0
 __device__ __forceinline__ void block_sum2(float &a, float &b) {
@@ -59,10 +77,16 @@ __global__ void __launch_bounds__(PL_THREADS) planner_local_kernel(PlannerParams
     float diff = 0.f, base = 0.f;
     const long long n = (long long)max(row1 - row0, 0) * p.D;      // the rows are contiguous in both buffers
     const StateT *cur = o + (slot + row0) * p.D, *old = so + (snap + row0) * p.D;
-    for (long long e = threadIdx.x; e < n; e += PL_THREADS) {
-        const float a = to_f32(cur[e]), b = to_f32(old[e]);
-        diff += (a - b) * (a - b);
-        base += b * b;
+    constexpr int V = Vec16<StateT>::N;        // rows are multiples of 16 bytes and start on such a boundary
+    for (long long e = (long long)threadIdx.x * V; e < n; e += (long long)PL_THREADS * V) {
+        float a[V], b[V];
+        Vec16<StateT>::load(cur + e, a);
+        Vec16<StateT>::load(old + e, b);
+#pragma unroll
+        for (int u = 0; u < V; ++u) {
+            diff = fmaf(a[u] - b[u], a[u] - b[u], diff);
+            base = fmaf(b[u], b[u], base);
+        }
     }
     for (int r = row0 + (int)threadIdx.x; r < row1; r += PL_THREADS) {
         const float a = p.lse_state[slot + r], b = p.snap_lse[snap + r];
@@ -169,11 +193,10 @@ __global__ void __launch_bounds__(1024) planner_decide_kernel(PlannerParams p) {
     }
 }
 
-// grid (chunks, P (query partition i), BH * S (slot j)): sum of squares of the state rows; anchor steps only
+// grid (chunks, P * S (query partition i, slot j), BH): sum of squares of the state rows of a composed cache
 template <typename StateT>
 __global__ void __launch_bounds__(PL_THREADS) planner_norm_kernel(PlannerParams p) {
-    if (!p.force && !p.state->is_anchor) return;
-    const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z / p.S, j = blockIdx.z - bh * p.S;
+    const int c = blockIdx.x, i = blockIdx.y / p.S, j = blockIdx.y - i * p.S, bh = blockIdx.z;
     if (!(p.nonempty[i] >> j & 1u)) {   // no such slot for this query partition
         if (threadIdx.x == 0) p.norm_partials[(((long long)bh * p.P + i) * p.chunks + c) * p.S + j] = 0.f;
         return;
@@ -184,9 +207,12 @@ __global__ void __launch_bounds__(PL_THREADS) planner_norm_kernel(PlannerParams 
     float sq = 0.f, unused = 0.f;
     const long long n = (long long)max(row1 - row0, 0) * p.D;
     const StateT *src = o + (slot + row0) * p.D;
-    for (long long e = threadIdx.x; e < n; e += PL_THREADS) {
-        const float a = to_f32(src[e]);
-        sq += a * a;
+    constexpr int V = Vec16<StateT>::N;
+    for (long long e = (long long)threadIdx.x * V; e < n; e += (long long)PL_THREADS * V) {
+        float a[V];
+        Vec16<StateT>::load(src + e, a);
+#pragma unroll
+        for (int u = 0; u < V; ++u) sq = fmaf(a[u], a[u], sq);
     }
     for (int r = row0 + (int)threadIdx.x; r < row1; r += PL_THREADS) {
         const float a = p.lse_state[slot + r];
@@ -194,6 +220,31 @@ __global__ void __launch_bounds__(PL_THREADS) planner_norm_kernel(PlannerParams 
     }
     block_sum2(sq, unused);
     if (threadIdx.x == 0) p.norm_partials[(((long long)bh * p.P + i) * p.chunks + c) * p.S + j] = sq;
+}
+
+// grid P * S, one block per (query partition i, slot j): ||AS(i, j)||^2 of an anchor, which has computed every state,
+// as the sum of the attention epilogue's partials in a fixed order (thread-strided sums, then a fixed tree)
+__global__ void __launch_bounds__(PL_THREADS) planner_attn_norm_kernel(PlannerParams p) {
+    PlannerState *st = p.state;
+    if (!st->is_anchor) return;
+    __shared__ double red[PL_THREADS];
+    const int e = blockIdx.x, i = e / p.S, j = e - i * p.S;
+    const int per_item = p.qblocks * (ATTN_NQ * 4);
+    double acc = 0.0;
+    if (p.nonempty[i] >> j & 1u) {
+        const long long total = (long long)p.BH * per_item;
+        for (long long k = threadIdx.x; k < total; k += PL_THREADS) {
+            const long long bh = k / per_item, r = k - bh * per_item;
+            acc += (double)p.attn_norm_partials[((bh * p.P + i) * p.S + j) * per_item + r];
+        }
+    }
+    red[threadIdx.x] = acc;
+    __syncthreads();
+    for (int s = PL_THREADS / 2; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) st->nsq[e] = red[0];
 }
 
 // one block: w (Eq. 8, mean over rows and heads) and alpha (Eq. 9) from the partial sums; anchor steps only
@@ -209,8 +260,9 @@ __global__ void __launch_bounds__(1024) planner_commit_kernel(PlannerParams p) {
             for (int c = 0; c < p.chunks; ++c) {
                 const long long idx = (((long long)bh * P + i) * p.chunks + c) * S + j;
                 w += (double)p.w_partials[idx];
-                n += (double)p.norm_partials[idx];
+                if (p.force) n += (double)p.norm_partials[idx];
             }
+        if (!p.force) n = st->nsq[e];   // from planner_attn_norm_kernel
         st->w[e] = w / ((double)p.BH * (double)(p.off[i + 1] - p.off[i]));
         nsq[e] = n;
     }
@@ -264,12 +316,16 @@ cudaError_t launch_planner_step(const PlannerParams &p, int state_dtype, cudaStr
 }
 
 cudaError_t launch_planner_commit(const PlannerParams &p, int state_dtype, cudaStream_t stream) {
-    dim3 grid_n((unsigned)p.chunks, (unsigned)p.P, (unsigned)(p.BH * p.S));
+    dim3 grid_n((unsigned)p.chunks, (unsigned)(p.P * p.S), (unsigned)p.BH);
     dim3 grid_s((unsigned)p.chunks, (unsigned)p.P, (unsigned)p.BH);
-    if (state_dtype == DT_STATE_FP32) planner_norm_kernel<float><<<grid_n, PL_THREADS, 0, stream>>>(p);
-    else planner_norm_kernel<__nv_bfloat16><<<grid_n, PL_THREADS, 0, stream>>>(p);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (p.force) {   // after a group compose the states were not written by the attention kernel: take the norms from the cache
+        if (state_dtype == DT_STATE_FP32) planner_norm_kernel<float><<<grid_n, PL_THREADS, 0, stream>>>(p);
+        else planner_norm_kernel<__nv_bfloat16><<<grid_n, PL_THREADS, 0, stream>>>(p);
+    } else {
+        planner_attn_norm_kernel<<<p.P * p.S, PL_THREADS, 0, stream>>>(p);
+    }
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     planner_commit_kernel<<<1, 1024, 0, stream>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (p.force) return cudaSuccess;   // a refresh after a group compose keeps the anchor's snapshot

@@ -458,11 +458,26 @@ def test_algorithm1_planner_over_denoising_steps():
     part = np.searchsorted(off, np.arange(wl.L), side="right") - 1
     eps, have_anchor = 0.0, False
     anchors, selective = 0, 0
+    anchor_local = None          # the oracle's local states of the last anchor: {(b, h, i): (OUT, LSE)}
     for t in range(wl.steps):
         q, k, v = run.gen.next()
         ctx.dt_attn_local(q, k, v, t)                              # local states of the step
         ctx.dt_planner_step(mask, flag, ase, drel)
         torch.cuda.synchronize()
+        # --- the device's drift (Eq. 10's norm, Eq. 14's relative drift) against the oracle's own states: the local
+        # states of this step by Eq. 1 from the same inputs, the anchor's kept from the step that was one
+        qb_, kb_, vb_ = (inputs.bf16_bits(x) for x in (q, k, v))
+        local_now = {}
+        for b_ in range(wl.B):
+            for h_ in range(wl.H):
+                for i in range(P):
+                    rows_i = np.arange(off[i], off[i + 1], dtype=np.int32)
+                    local_now[(b_, h_, i)] = orc.pair_state(qb_, kb_, vb_, wl.scale, b_, h_, rows_i, int(off[i]), int(off[i + 1]))
+        if anchor_local is not None:
+            d_or = sum(orc.state_norm_sq(local_now[key][0] - anchor_local[key][0], local_now[key][1] - anchor_local[key][1])
+                       for key in local_now)
+            b_or = sum(orc.state_norm_sq(*anchor_local[key]) for key in local_now)
+            assert drel.item() == pytest.approx(np.sqrt(d_or / b_or), rel=3e-2), t
         # --- the oracle rule on the GPU's own quantities
         w_g, alpha_g, eps_before, have_g = ctx.dt_planner_get()
         assert have_g == have_anchor
@@ -503,6 +518,7 @@ def test_algorithm1_planner_over_denoising_steps():
         if ref["is_anchor"]:
             anchors += 1
             have_anchor = True
+            anchor_local = local_now
             # w (Eq. 8) and alpha (Eq. 9) against the oracle's states of this anchor
             w_g, alpha_g, _, _ = ctx.dt_planner_get()
             lse_ref = np.empty((P, wl.B, wl.H, wl.L)); nsq = np.zeros((P, P))

@@ -132,3 +132,14 @@ def test_head_range_covers_every_head_once():
     assert sharding.all_reduce_sums(t) is t and float(t.sum()) == 4.0     # no process group: one shard
     with pytest.raises(TypeError):
         sharding.all_reduce_sums(torch.ones(4))
+
+
+def test_gpus_flag_starts_its_own_ranks():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks itself (the same code path the GPU bench
+    takes; here the ranks only join a gloo group and count themselves)."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--probe-world"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(x) for x in r.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1 and lines[0]["world_size"] == 2 and lines[0]["ranks_counted"] == 2 and lines[0]["n_gpus"] == 2
