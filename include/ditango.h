@@ -170,7 +170,7 @@ dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32
 /* Head-sharded planning.  The (batch, head) slices of a layer are independent in dt_attn_states and
  * dt_state_merge, so the heads of one layer may be spread over several contexts (one per GPU) with no
  * exchange there.  Only the plan needs one: W of Eq. 8 is a mean over all heads, and every shard must
- * arrive at the same mask (Section 4.3: the compute / reuse strategy is the same on all devices).  The
+ * arrive at the same mask (Section 5.1.1: the compute / reuse strategy is the same on all devices).  The
  * two halves of dt_plan, with the exchange left to the caller:
  *   dt_plan_sums       sums_dev (device, double [P*S], written) = sum over this context's batch, heads and
  *                      the rows of partition i of the per-row weights w (Eq. 8), not yet divided by a count
@@ -264,7 +264,7 @@ dt_status dt_attn_fused(dt_ctx *ctx, const void *q_dev, const void *k_dev, const
  *                    was never computed).  The memory behind the first S slots of the bound buffers is no
  *                    longer used.  If the planner is initialised, its w and alpha are taken again from the
  *                    composed cache (the anchor's snapshot of the local states stays).  DT_ERR_STATE if only one group is left.  Synchronises the stream.
- * dt_group_fit       the memory-driven trigger of Section 4.2: while the slots in use (S * B*H*L * (D*sizeof(state) + 4)
+ * dt_group_fit       the memory-driven trigger of Section 5.1.3: while the slots in use (S * B*H*L * (D*sizeof(state) + 4)
  *                    bytes) exceed max_bytes and more than one group is left, dt_group_compose; *composed (may be
  *                    NULL) = how many times.  DT_ERR_STATE if one group is left and the budget is still exceeded.
  * dt_group_reset     back to the creation-time g (an anchor step recomputes every state): all t_c = -1, the
@@ -288,9 +288,12 @@ dt_status dt_group_reset(dt_ctx *ctx, void *stream);
  *     the process exits).  Problems that need more than 262144 partial sums, i.e.
  *     B*H*P*P*ceil(max_i n_i / 1024) > 262144, are refused with DT_ERR_UNSUPPORTED and nothing runs.
  *   - Calls nothing that allocates or frees: no cudaMalloc / cudaFree, no allocating library routine.
- *     The offsets are copied into the array's header with one cudaMemcpyAsync on `stream`.
+ *     The offsets travel to the device as a kernel argument (a small kernel writes them into the
+ *     array's header), so `part_offsets_host` is read before the call returns and never afterwards.
  *   - The first call on each device looks up the array's device address (the current device must
  *     be the one that owns `stream` and the buffers); make that first call outside any stream capture.
+ *     The address is remembered per device for the life of the process: after a cudaDeviceReset the
+ *     library has to be loaded again before this entry point is used on that device.
  *   - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing
  *     in it has to start at zero (stage 1 overwrites every slot stage 2 reads), but two calls whose
  *     kernels can overlap on the GPU (different streams, no ordering between them) race on it:

@@ -534,6 +534,7 @@ static dt_status plan_impl(dt_ctx *ctx, double eps, double target_fraction, int3
 
 dt_status dt_plan_grouped(dt_ctx *ctx, double eps, double target_fraction, int32_t group_size, uint8_t *mask_dev,
                           double *w_dev, double *eps_out_dev, void *stream) {
+    if (!ctx) return DT_ERR_INVALID_ARG;
     return plan_impl(ctx, eps, target_fraction, group_size, mask_dev, w_dev, eps_out_dev, stream, nullptr, nullptr, 0);
 }
 

@@ -168,12 +168,6 @@ __device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, lon
 }
 
 // 32 consecutive elements of a cached state row as fp32
-__device__ __forceinline__ __nv_bfloat162 u32_as_bf162(uint32_t x) {
-    return *reinterpret_cast<const __nv_bfloat162 *>(&x);
-}
-__device__ __forceinline__ uint32_t bf162_as_u32(__nv_bfloat162 x) {
-    return *reinterpret_cast<const uint32_t *>(&x);
-}
 __device__ __forceinline__ void load_state_chunk(const float *src, float (&v)[32]) {
 #pragma unroll
     for (int c = 0; c < 32; c += 4) {

@@ -437,6 +437,15 @@ static __device__ __align__(256) float g_plan_static_scratch[STATIC_PLAN_OFFSET_
 // In host code the array's name is only a handle: the device address is looked up once per device.
 float *g_plan_static_ptr[STATIC_PLAN_MAX_DEVICES] = {nullptr};
 
+// The partition offsets reach the device as a kernel argument: they are copied when the launch is
+// made, so nothing refers to the caller's host array after dt_plan_static has returned.
+struct StaticOffsets {
+    int32_t v[DT_MAX_P + 1];
+};
+__global__ void static_offsets_kernel(StaticOffsets o, int n, int32_t *dst) {
+    if ((int)threadIdx.x < n) dst[threadIdx.x] = o.v[threadIdx.x];
+}
+
 }  // namespace
 
 extern "C" dt_status dt_plan_static(const float *lse_state_dev, const int32_t *part_offsets_host, int32_t B, int32_t H,
@@ -470,8 +479,10 @@ extern "C" dt_status dt_plan_static(const float *lse_state_dev, const int32_t *p
     int32_t *off_dev = reinterpret_cast<int32_t *>(scratch);
     float *partials = scratch + STATIC_PLAN_OFFSET_SLOTS;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(off_dev, part_offsets_host, (P + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return DT_ERR_CUDA;
+    StaticOffsets ov;
+    for (int i = 0; i <= P; ++i) ov.v[i] = part_offsets_host[i];
+    static_offsets_kernel<<<1, 64, 0, st>>>(ov, P + 1, off_dev);
+    if (cudaGetLastError() != cudaSuccess) return DT_ERR_CUDA;
 
     dt::PlanParams pp;
     pp.lse_state = lse_state_dev;

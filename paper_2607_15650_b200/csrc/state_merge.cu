@@ -205,6 +205,10 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
         if (!mbar_wait_bounded(bar, (uint32_t)phase, abort_flag, MERGE_WAIT_LIMIT)) {
             if (p.status) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
             *abort_flag = 1;
+            // copies may still be in flight towards this block's shared memory: stay resident until they have had
+            // time to land (every thread waits on the same barrier, so all of them take this way out)
+            const uint64_t t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
             return;
         }
         if (active && !empty) {

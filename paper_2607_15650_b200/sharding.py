@@ -3,7 +3,7 @@
 The (batch, head) slices of a layer are independent in dt_attn_states and dt_state_merge, so a rank that holds
 H_local of the H heads runs both on its slice with no exchange.  The plan is the one step that needs one: the
 partition importance W (Eq. 8) is a mean over all heads, and every rank must take the same COMPUTE / REUSE mask
-(Section 4.3: the strategy is the same on all devices).  Each rank therefore sums its own per-row weights
+(Section 5.1.1: the strategy is the same on all devices).  Each rank therefore sums its own per-row weights
 (dt_plan_sums), the P x S sums are added over the ranks by one all-reduce of doubles, and each rank finishes the
 plan from the same totals (dt_plan_from_sums).  This module holds that plumbing only; every step of the
 arithmetic runs in the library's kernels.

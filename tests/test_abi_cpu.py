@@ -74,3 +74,25 @@ def test_status_strings(lib):
     assert binding.status_str(99) == "DT_ERR_UNKNOWN"
     assert lib.dt_destroy(None) == binding.DT_OK
     assert lib.dt_poll(None) == binding.DT_ERR_INVALID_ARG
+
+
+def test_null_context_is_an_argument_error_on_every_entry_point(lib):
+    """Every call that takes a context returns DT_ERR_INVALID_ARG for a null one (dt_destroy accepts it, like free);
+    nothing is dereferenced and no CUDA call is made."""
+    text = open(os.path.join(ROOT, "include", "ditango.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    with_ctx = sorted(set(re.findall(r"\bdt_status\s+(dt_[a-z_0-9]+)\s*\(\s*dt_ctx\s*\*\s*ctx\b", text)))
+    assert len(with_ctx) >= 25 and "dt_plan" in with_ctx and "dt_plan_grouped" in with_ctx
+    for name in with_ctx:
+        fn = getattr(lib, name)
+        args = []
+        for t in fn.argtypes[1:]:
+            if t in (C.c_double, C.c_float):
+                args.append(0.0)
+            elif t in (C.c_int32, C.c_int64, C.c_uint32, C.c_size_t, C.c_int):
+                args.append(0)
+            else:
+                args.append(None)
+        got = fn(None, *args)
+        assert got == (binding.DT_OK if name == "dt_destroy" else binding.DT_ERR_INVALID_ARG), name
+    assert lib.dt_last_error(None) in (b"", None) or isinstance(lib.dt_last_error(None), bytes)

@@ -21,7 +21,7 @@ pytestmark = pytest.mark.gpu
 O_MAX, O_MEAN, LSE_ABS = 2e-2, 2e-3, 5e-3
 
 
-def _run_full_size(name, fraction, n_samples, n_selective, state_dtype=binding.DT_STATE_FP32):
+def _run_full_size(name, fraction, n_samples, n_selective, state_dtype=binding.DT_STATE_FP32, record=None):
     build.build()
     wl = inputs.WORKLOADS[name]
     dev = torch.device("cuda", 0)
@@ -38,6 +38,7 @@ def _run_full_size(name, fraction, n_samples, n_selective, state_dtype=binding.D
     eps = torch.empty(1, dtype=torch.float64, device=dev)
     errs = []
     for t in range(1 + n_selective):
+        step_means = []
         q, k, v = gen.next()
         mask_h = mask.cpu().numpy().reshape(P, P).copy()
         ctx.dt_attn_states(q, k, v, mask, t)
@@ -53,13 +54,15 @@ def _run_full_size(name, fraction, n_samples, n_selective, state_dtype=binding.D
             eo = np.abs(got_o - ref_o[(b, h)])
             el = np.abs(got_l - ref_l[(b, h)])
             errs.append((eo.max(), eo.mean(), el.max()))
+            step_means.append((eo.mean(), eo.size))
             assert eo.max() <= O_MAX and el.max() <= LSE_ABS, (name, t, b, h, eo.max(), el.max())
             # the cached pair states of those rows, fresh or reused
             st_o = ctx.o_state[:, b, h][:, ridx].float().cpu().numpy()          # [P, n, D]
             st_l = ctx.lse_state[:, b, h][:, ridx].cpu().numpy()                # [P, n]
             assert np.abs(st_o.transpose(1, 0, 2) - ses.o[(b, h)]).max() <= O_MAX
             assert np.abs(st_l.T - ses.lse[(b, h)]).max() <= LSE_ABS
-        assert np.mean([e[1] for e in errs]) <= O_MEAN
+        # mean absolute error of this step's sampled outputs (every step on its own, not a running mean)
+        assert sum(m * n for m, n in step_means) / sum(n for _, n in step_means) <= O_MEAN, (name, t)
         assert (ctx.dt_get_tc() == ses.tc).all()
         if t == 0:
             # plan from the anchor step's LSE cache; the oracle gets the very same fp32 values
@@ -74,31 +77,49 @@ def _run_full_size(name, fraction, n_samples, n_selective, state_dtype=binding.D
             assert (got_mask == own_mask).all() and eps.item() == own_eps and got_mask.sum() == K
             ref_mask, ref_eps, _ = orc.target_fraction(W_ref, fraction)
             offd = ~np.eye(P, dtype=bool)
-            margin = np.abs(W_ref[offd] - ref_eps).min() / ref_eps
-            if margin > 1e-4:           # otherwise the oracle's own plan is not resolvable in fp32
-                assert (got_mask == ref_mask).all()
+            # The GPU's W carries fp32 rounding (2e-5 relative above): a pair whose oracle measure lies closer than 1e-4
+            # (relative) to the oracle's threshold cannot be decided from it.  Such pairs are left out of the comparison
+            # and the plan is reported as ill-conditioned by name; every other pair must agree.
+            rel = np.abs(W_ref - ref_eps) / ref_eps
+            decidable = (rel > 1e-4) | ~offd
+            margin = rel[offd].min()
+            verdict = "well-conditioned" if margin > 1e-4 else f"ILL-CONDITIONED ({int((~decidable).sum())} pairs undecidable)"
+            print(f"[plan margin] {name} f={fraction}: min |W - eps| / eps = {margin:.3e} -> {verdict}; "
+                  f"GPU mask == oracle mask on all decidable pairs: {bool((got_mask == ref_mask)[decidable].all())}")
+            if record is not None:
+                record("plan_margin", float(margin))
+                record("plan_conditioning", verdict)
+            assert (got_mask == ref_mask)[decidable].all()
+            assert decidable.sum() >= P * P - 2, "more than two undecidable pairs: the workload's plan is degenerate"
             # locality of the synthetic workload: contribution falls with partition distance
             d = np.abs(np.subtract.outer(np.arange(P), np.arange(P)))
             assert W_ref[d == 0].mean() > W_ref[d == 1].mean() > W_ref[d >= 3].mean()
     return errs
 
 
-def test_full_size_c3_wan720p_headline():
+def test_full_size_c3_wan720p_headline(record_property):
     """The configuration bench.py times: 75 600 tokens, 40 heads, D 128, P 16, f = 0.40."""
-    _run_full_size("c3_wan720p", 0.40, n_samples=2048, n_selective=2)
+    _run_full_size("c3_wan720p", 0.40, n_samples=2048, n_selective=2, record=record_property)
 
 
-def test_full_size_c1_cogvideox_d64_with_text_tokens():
-    _run_full_size("c1_cogvideox", 0.5, n_samples=2048, n_selective=2)
+def test_full_size_c1_cogvideox_d64_with_text_tokens(record_property):
+    _run_full_size("c1_cogvideox", 0.5, n_samples=2048, n_selective=2, record=record_property)
 
 
-def test_full_size_c2_wan480p_uneven_partitions():
-    _run_full_size("c2_wan480p", 0.25, n_samples=2048, n_selective=1)
+def test_full_size_c2_wan480p_uneven_partitions(record_property):
+    _run_full_size("c2_wan480p", 0.25, n_samples=2048, n_selective=1, record=record_property)
 
 
-def test_full_size_c4_hunyuan_p32_bf16_state_cache():
+def test_full_size_c4_hunyuan_p32_bf16_state_cache(record_property):
     """Largest footprint: 118 800 tokens, P = 32 (3712/3713-row partitions), states cached in bf16."""
-    _run_full_size("c4_hunyuan720p", 0.125, n_samples=2048, n_selective=1, state_dtype=binding.DT_STATE_BF16)
+    _run_full_size("c4_hunyuan720p", 0.125, n_samples=2048, n_selective=1, state_dtype=binding.DT_STATE_BF16,
+                   record=record_property)
+
+
+def test_full_size_c4_hunyuan_p32_fp32_pair_cache(record_property):
+    """The footprint stress case as the workload names it: all 1024 pair states cached in fp32 (47 GB resident), the
+    anchor step at f = 1.0 and one selective step at f = 0.125."""
+    _run_full_size("c4_hunyuan720p", 0.125, n_samples=1536, n_selective=1, record=record_property)
 
 
 def test_full_size_c4_hunyuan_grouped_cache_and_dynamic_compose():

@@ -263,9 +263,13 @@ def _plan_case(wl, lse_host, off, fractions, eps_list):
         assert got.sum() == K
         # and it equals the oracle's plan whenever the oracle's own margin is resolvable in fp32
         offd = ~np.eye(P, dtype=bool)
-        gap = np.abs(W_ref[offd] - ref_eps).min() / max(ref_eps, 1e-300)
+        rel = np.abs(W_ref - ref_eps) / max(ref_eps, 1e-300)
+        decidable = (rel > 1e-4) | ~offd            # pairs the fp32 measure can decide; the rest are reported by name
+        gap = rel[offd].min()
+        print(f"[plan margin] {wl.name} f={f}: min |W - eps| / eps = {gap:.3e} -> "
+              + ("well-conditioned" if gap > 1e-4 else f"ILL-CONDITIONED ({int((~decidable).sum())} pairs undecidable)"))
+        assert (got == ref_mask)[decidable].all()
         if gap > 1e-4:
-            assert (got == ref_mask).all()
             assert eps_out.item() == pytest.approx(ref_eps, rel=1e-4)
     for eps in eps_list:
         ctx.dt_plan(mask, eps=eps, w_dev=W, eps_out_dev=eps_out)

@@ -388,6 +388,32 @@ def test_target_fraction_banded_measure_gives_banded_mask_and_tie_rule():
     assert mask1.sum() == P + 1 and mask1[0, 1] == 1
 
 
+def test_target_fraction_ties_go_to_the_nearer_partition_and_eps_is_the_midpoint():
+    """Hand-checked: a measure with only two values, so that the rank order is decided by the tie rule alone --
+    equal W: the pair with the smaller |i - j| first, then the smaller i*P + j -- and the reported threshold is the
+    midpoint between the last selected and the first unselected value."""
+    P = 4
+    W = np.full((P, P), 0.1)
+    W[0, 3] = W[3, 0] = 0.3                       # the two far corners carry the large value
+    # K = 4 + 2: the two corners (largest W) and nothing else; eps midway between 0.3 and 0.1
+    mask, eps, K = orc.target_fraction(W, 6 / 16)
+    want = np.eye(P, dtype=np.uint8); want[0, 3] = want[3, 0] = 1
+    assert K == 6 and (mask == want).all() and eps == 0.5 * (0.3 + 0.1)
+    # K = 4 + 2 + 3: among the ten tied pairs the distance-1 ones come first, in index order: (0,1), (1,0), (1,2)
+    mask, eps, K = orc.target_fraction(W, 9 / 16)
+    want[0, 1] = want[1, 0] = want[1, 2] = 1
+    assert K == 9 and (mask == want).all() and eps == 0.1        # the cut runs through a tie: eps is the tied value
+    # K = 4 + 2 + 6 + 1: all six distance-1 pairs, then the first distance-2 pair (0,2); (2,0) and the rest stay REUSE
+    mask, eps, K = orc.target_fraction(W, 13 / 16)
+    d = np.abs(np.subtract.outer(np.arange(P), np.arange(P)))
+    want = ((d <= 1) | (d == 3)).astype(np.uint8); want[0, 2] = 1
+    assert K == 13 and (mask == want).all()
+    # a tie across distances with the larger value on the far pair: value wins over distance
+    W2 = np.full((P, P), 0.2); W2[0, 2] = 0.25
+    mask, eps, K = orc.target_fraction(W2, 5 / 16)
+    assert K == 5 and mask[0, 2] == 1 and mask.sum() == 5 and eps == 0.5 * (0.25 + 0.2)
+
+
 def test_group_plan_with_group_size_one_is_the_ungrouped_rule():
     """g = 1: every unit is a single off-diagonal pair, so the grouped rule must reproduce Eq. 13 and
     the target-fraction selection exactly."""
