@@ -194,6 +194,8 @@ dt_status dt_create(dt_ctx **ctx_out, const dt_config *cfg) {
     ok = ok && cudaMalloc(&ctx->nonempty_dev, P * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->tc_dev, P * S * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->worklist_dev, (1 + P * S) * sizeof(int32_t)) == cudaSuccess;
+    if (ctx->group_size0 <= 1)   // pair mode: at most ceil(P * tiles / 2) items per KV partition
+        ok = ok && cudaMalloc(&ctx->tile_pairs_dev, (1 + (size_t)P * (((size_t)P * ctx->qblocks_max * dt::ATTN_NQ + 1) / 2)) * sizeof(int4)) == cudaSuccess;
     ctx->max_tiles = cfg->L / dt::ATTN_TILE + 2 * DT_MAX_P + 4;   // one pass over all keys + one ragged tile per run
     ok = ok && cudaMalloc(&ctx->tile_tab_dev, (size_t)P * ctx->max_tiles * sizeof(int2)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->tile_cnt_dev, P * sizeof(int32_t)) == cudaSuccess;
@@ -223,6 +225,7 @@ dt_status dt_destroy(dt_ctx *ctx) {
     cudaFree(ctx->nonempty_dev);
     cudaFree(ctx->tc_dev);
     cudaFree(ctx->worklist_dev);
+    cudaFree(ctx->tile_pairs_dev);
     cudaFree(ctx->tile_tab_dev);
     cudaFree(ctx->tile_cnt_dev);
     cudaFree(ctx->status_dev);
@@ -272,12 +275,13 @@ dt_status attn_launch(dt_ctx *ctx, const void *q_dev, const void *k_dev, const v
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dt_config &c = ctx->cfg;
     cudaError_t e = dt::launch_worklist(mask_dev, ctx->tc_dev, ctx->worklist_dev, ctx->status_dev, ctx->slot_tab_dev, c.P,
-                                        ctx->S, ctx->group_size0 > 1 ? 1 : 0, step, st);
+                                        ctx->S, ctx->group_size0 > 1 ? 1 : 0, step, ctx->off_dev, ctx->tile_pairs_dev, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "work-list launch");
     dt::AttnParams p = {};
     p.off = ctx->off_dev;
     p.slot_tab = ctx->slot_tab_dev;
     p.worklist = ctx->worklist_dev;
+    p.tile_pairs = ctx->tile_pairs_dev;
     p.status = ctx->status_dev;
     p.o_state = ctx->o_state;
     p.lse_state = ctx->lse_state;

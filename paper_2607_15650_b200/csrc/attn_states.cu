@@ -5,8 +5,10 @@
 // (query partition, slot) whose keys are the slot's one or two key ranges: the group's state, the
 // composition (Eq. 2) of its members' states, comes out of one pass over their keys.
 //
-// One persistent CTA per SM walks the work list (b*h slowest, then COMPUTE pair, then query
-// block), so CTAs running at the same time share one head's K/V partition through L2.
+// One persistent CTA per SM walks the work list (b*h slowest, then KV partition, then the query tiles of every query
+// partition that computes it, two per item), so CTAs running at the same time share one head's K/V partition through L2.
+// The two 128-row query tiles of an item need not be neighbours: a partition with an odd number of tiles leaves one over,
+// which is paired with the first tile of the next query partition that attends to the same KV partition.
 //
 // Per CTA (12 warps; the producer warpgroup gives registers to the softmax warpgroups):
 //   warps 0-3 / 4-7  softmax warpgroups for query tile 0 / 1 (128 rows each, one row per thread)
@@ -119,8 +121,10 @@ struct RingPos {
 
 struct WorkItem {
     int bh, b, h, i, slot;
-    int q_row0;     // first query row of the block (global token index)
-    int n_q;        // valid query rows in the block (<= NQ*128)
+    // The two query tiles of the item: first row (global token index), valid rows (0: the tile is absent), query
+    // partition and tile index within it.  In pair mode the two tiles may come from different query partitions (they
+    // share the K/V stream of slot j); otherwise they are the two halves of one 256-row block of partition i.
+    int qrow[ATTN_NQ], qn[ATTN_NQ], qi[ATTN_NQ], qt[ATTN_NQ];
     int r1, n1;     // first key range of the slot
     int r2, n2;     // second key range (n2 == 0: none)
     int tiles1;     // ceil(n1 / 128)
@@ -135,36 +139,65 @@ struct WorkItem {
     }
 };
 
-// Work index -> item.  Returns false when the block lies beyond the end of partition i (or has no keys).
-// npairs = work items per (b, h) and query block: COMPUTE states of the work list, or P in fused mode.
+// Work index -> item.  Returns false when the item has no query rows (or no keys).
+// per_bh = work items per (b, h): tile pairs of the pair-mode list, COMPUTE states x query blocks with a grouped cache,
+// or P x query blocks in fused mode.
 template <bool FUSED>
-__device__ __forceinline__ bool decode_work(const AttnParams &p, int npairs, long long w, WorkItem &it) {
-    const long long per_bh = (long long)npairs * p.qblocks_max;
+__device__ __forceinline__ long long work_per_bh(const AttnParams &p) {
+    if constexpr (FUSED) return (long long)p.P * p.qblocks_max;
+    if (p.tile_pairs != nullptr) return p.tile_pairs[0].x;
+    return (long long)p.worklist[0] * p.qblocks_max;
+}
+
+template <bool FUSED>
+__device__ __forceinline__ bool decode_work(const AttnParams &p, long long per_bh, long long w, WorkItem &it) {
     const int bh_launch = (int)(w / per_bh);          // index among the (b, h) of this launch
     const int rem = (int)(w - (long long)bh_launch * per_bh);
-    const int pair = rem / p.qblocks_max;
-    const int qb = rem - pair * p.qblocks_max;
-    const int code = FUSED ? pair : p.worklist[1 + pair];
-    it.i = code & 0xFF;
-    it.slot = code >> 8;
     it.b = bh_launch / p.H_launch;
     it.h = p.h0 + bh_launch - it.b * p.H_launch;
     it.bh = it.b * p.H + it.h;
-    const int qs = p.off[it.i], qe = p.off[it.i + 1];
-    it.q_row0 = qs + qb * (ATTN_NQ * ATTN_TILE);
-    it.n_q = min(qe - it.q_row0, ATTN_NQ * ATTN_TILE);
+    if (!FUSED && p.tile_pairs != nullptr) {
+        // pair mode: (i_a | j << 8, tile_a, i_b or -1, tile_b) -- two 128-row query tiles that attend to KV partition j
+        const int4 e = __ldg(p.tile_pairs + 1 + rem);
+        it.i = e.x & 0xFF;
+        it.slot = e.x >> 8;
+        const int ia[ATTN_NQ] = {it.i, e.z}, ta[ATTN_NQ] = {e.y, e.w};
+#pragma unroll
+        for (int q = 0; q < ATTN_NQ; ++q) {
+            const bool have = ia[q] >= 0;
+            const int iq = have ? ia[q] : it.i;
+            it.qi[q] = iq;
+            it.qt[q] = ta[q];
+            it.qrow[q] = p.off[iq] + (have ? ta[q] : e.y) * ATTN_TILE;
+            it.qn[q] = have ? min(p.off[iq + 1] - it.qrow[q], ATTN_TILE) : 0;
+        }
+    } else {
+        const int pair = rem / p.qblocks_max;
+        const int qb = rem - pair * p.qblocks_max;
+        const int code = FUSED ? pair : p.worklist[1 + pair];
+        it.i = code & 0xFF;
+        it.slot = code >> 8;
+        const int qs = p.off[it.i], qe = p.off[it.i + 1];
+#pragma unroll
+        for (int q = 0; q < ATTN_NQ; ++q) {
+            it.qi[q] = it.i;
+            it.qt[q] = qb * ATTN_NQ + q;
+            it.qrow[q] = qs + it.qt[q] * ATTN_TILE;
+            it.qn[q] = max(min(qe - it.qrow[q], ATTN_TILE), 0);
+        }
+    }
     if constexpr (FUSED) {
         it.tab = p.tile_tab + (long long)it.i * p.max_tiles;
         it.tiles = p.tile_cnt[it.i];
         it.r1 = it.n1 = it.r2 = it.n2 = it.tiles1 = 0;
-        return it.n_q > 0 && it.tiles > 0;
+        return it.qn[0] > 0 && it.tiles > 0;
     }
     it.tab = nullptr;
     const int4 rg = *reinterpret_cast<const int4 *>(p.slot_tab + it.i * p.S + it.slot);
     it.r1 = rg.x; it.n1 = rg.y; it.r2 = rg.z; it.n2 = rg.w;
     it.tiles1 = (it.n1 + ATTN_TILE - 1) / ATTN_TILE;
     it.tiles = it.tiles1 + (it.n2 + ATTN_TILE - 1) / ATTN_TILE;
-    return it.n_q > 0;
+    return it.qn[0] > 0;
 }
 
 // 32 consecutive elements of a cached state row as fp32
@@ -269,8 +302,8 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    const int npairs = FUSED ? p.P : p.worklist[0];
-    const long long total_work = (long long)npairs * p.qblocks_max * p.B * p.H_launch;
+    const long long npairs = work_per_bh<FUSED>(p);   // work items per (b, h)
+    const long long total_work = npairs * p.B * p.H_launch;
 
     if (warp >= TMA_WARP) {
       reg_dealloc<REGS_PRODUCER>();
@@ -294,7 +327,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 #pragma unroll
                     for (int hf = 0; hf < C::NHALF; ++hf)
                         tma_load_4d(q_smem + q * C::TILE_BYTES + hf * C::HALF_BYTES, &tmap_q, bars.q_full, hf * 64, it.h,
-                                    it.q_row0 + q * ATTN_TILE, it.b);
+                                    it.qrow[q], it.b);
                 q_phase ^= 1u;
                 if constexpr (C::PREFETCH) {
                     for (int n = 0; n < 2 * it.tiles && ok; ++n) {
@@ -702,8 +735,11 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             if (!ok) break;
             o_phase ^= 1u;
             tc_fence_after();
-            const int row_in_block = q * ATTN_TILE + row_in_tile;
-            const bool row_valid = row_in_block < it.n_q;
+            // this warpgroup's query tile (selected, not indexed: the arrays stay in registers)
+            const int my_qn = q ? it.qn[1] : it.qn[0], my_qrow = q ? it.qrow[1] : it.qrow[0];
+            const int my_qi = q ? it.qi[1] : it.qi[0], my_qt = q ? it.qt[1] : it.qt[0];
+            const bool row_valid = row_in_tile < my_qn;
+            const int q_row = my_qrow + row_in_tile;   // this thread's query row (global token index)
             const float inv_l = 1.0f / l_sum;
             if constexpr (!FP16) {
                 // a sum that is not finite: within one K/V tile a logit rose more than about 120 binades above the
@@ -713,7 +749,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             const float lse_fresh = 0.69314718055994530942f * (m_used + log2f(l_sum));
             if constexpr (FUSED) {
                 // fresh state (+) composed reuse state (Eq. 2), straight to the attention output
-                const long long crow = (long long)it.bh * p.L + it.q_row0 + row_in_block;
+                const long long crow = (long long)it.bh * p.L + q_row;
                 float w_f = inv_l, w_c = 0.f, lse_row = lse_fresh;
                 if (p.comp_o != nullptr && row_valid) {
                     const float lc = __ldcs(p.comp_lse + crow);
@@ -724,7 +760,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     w_c = ec / z;
                     lse_row = M + __logf(z);
                 }
-                __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) + it.b * p.sb + (long long)(it.q_row0 + row_in_block) * p.sl +
+                __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) + it.b * p.sb + (long long)q_row * p.sl +
                                      it.h * p.sh;
                 const StateT *csrc = static_cast<const StateT *>(p.comp_o) + crow * D;
 #pragma unroll
@@ -757,7 +793,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 }
                 if (row_valid && p.lse_out != nullptr) p.lse_out[crow] = lse_row;
             } else {
-                const long long srow = ((long long)it.slot * p.B * p.H + it.bh) * p.L + it.q_row0 + row_in_block;
+                const long long srow = ((long long)it.slot * p.B * p.H + it.bh) * p.L + q_row;
                 // Rows leave through shared memory, warp by warp: each thread writes 128 bytes of its row (swizzled,
                 // so the 32 lanes hit different banks), then the warp reads the 4 KB back so that 8 lanes hold the
                 // 128 contiguous bytes of one row and stores them -- whole lines to the cache instead of 16 bytes per
@@ -766,7 +802,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 constexpr int CH = 128 / (int)sizeof(StateT);          // state elements per 128-byte chunk
                 const uint32_t stage = out_smem + warp * 4096;          // [32 rows][128 bytes]
                 const uint32_t my_row = stage + lane * 128;
-                const int rows_left = it.n_q - (row_in_block - lane);   // valid rows of this warp's 32
+                const int rows_left = my_qn - (row_in_tile - lane);   // valid rows of this warp's 32
                 uint8_t *gbase = reinterpret_cast<uint8_t *>(o_state + (srow - lane) * D);   // row 0 of this warp
                 float row_sq = lse_fresh * lse_fresh;   // ||AS||^2 of this row: OUT and LSE stacked (Eq. 9)
 #pragma unroll
@@ -825,8 +861,8 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 #pragma unroll
                     for (int sft = 16; sft > 0; sft >>= 1) row_sq += __shfl_xor_sync(0xFFFFFFFFu, row_sq, sft);
                     if (lane == 0) {
-                        const int qb = (it.q_row0 - p.off[it.i]) / (ATTN_NQ * ATTN_TILE);
-                        p.norm_partials[((((long long)it.bh * p.P + it.i) * p.S + it.slot) * p.qblocks_max + qb) * (ATTN_NQ * 4) + warp] = row_sq;
+                        p.norm_partials[((((long long)it.bh * p.P + my_qi) * p.S + it.slot) * (p.qblocks_max * ATTN_NQ) + my_qt) * 4 +
+                                        (warp & 3)] = row_sq;
                     }
                 }
             }

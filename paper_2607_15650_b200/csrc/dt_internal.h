@@ -30,6 +30,9 @@ struct AttnParams {
     const int32_t *off;       // device, P+1
     const SlotRange *slot_tab; // device, [P][S]
     const int32_t *worklist;  // device: [0] = number of COMPUTE states, then i | (slot << 8) per state
+    // pair mode: [0].x = number of work items per (b, h), then per item (i_a | j << 8, tile_a, i_b or -1, tile_b): two
+    // 128-row query tiles (partition, tile index) that attend to KV partition j.  null: items are 256-row query blocks
+    const int4 *tile_pairs;
     int32_t *status;          // device status word
     void *o_state;            // [S][B][H][L][D]
     float *lse_state;         // [S][B][H][L]
@@ -158,7 +161,7 @@ cudaError_t launch_planner_step(const PlannerParams &p, int state_dtype, cudaStr
 cudaError_t launch_planner_commit(const PlannerParams &p, int state_dtype, cudaStream_t stream);
 
 cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, const SlotRange *slot_tab,
-                            int P, int S, int group_mode, int step, cudaStream_t stream);
+                            int P, int S, int group_mode, int step, const int32_t *off, int4 *tile_pairs, cudaStream_t stream);
 cudaError_t launch_attn_states(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                                const AttnParams &p, int D, int state_dtype, int num_ctas, cudaStream_t stream);
 cudaError_t launch_attn_fused(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
@@ -196,6 +199,7 @@ struct dt_ctx {
     int32_t *off_dev = nullptr;
     int32_t *tc_dev = nullptr;
     int32_t *worklist_dev = nullptr;
+    int4 *tile_pairs_dev = nullptr;   // pair mode: work items of the attention kernel
     int2 *tile_tab_dev = nullptr;     // fused mode: [P][max_tiles]
     int32_t *tile_cnt_dev = nullptr;  // [P]
     int max_tiles = 0;

@@ -264,12 +264,14 @@ __global__ void __launch_bounds__(1024) plan_final_kernel(PlanFinalParams p) {
     }
 }
 
+__device__ void build_tile_pairs(bool is_compute, const int32_t *off, int P, int4 *out);
+
 // mask -> compact list of COMPUTE states (ordered by i*S+slot), t_c update, REUSE-of-empty detection.
 // mask == nullptr: the local states only, and no REUSE-of-empty check (the other states of the step are
 // decided later).  Slots that do not exist for a query partition are never listed and never flagged.
 __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int32_t *tc, int32_t *worklist,
                                                         int32_t *status, const SlotRange *slot_tab, int P, int S,
-                                                        int group_mode, int step) {
+                                                        int group_mode, int step, const int32_t *off, int4 *tile_pairs) {
     __shared__ int warp_cnt[32];
     const int total = P * S, e = threadIdx.x;
     bool f = false;
@@ -294,6 +296,56 @@ __global__ void __launch_bounds__(1024) worklist_kernel(const uint8_t *mask, int
     }
     if (f) worklist[1 + pos] = (e / S) | ((e % S) << 8);
     if (e == 0) worklist[0] = cnt;
+    if (tile_pairs != nullptr) build_tile_pairs(f, off, P, tile_pairs);   // pair mode (S == P): the attention kernel's items
+}
+
+// Pair mode: the work items of the attention kernel.  For every KV partition j the 128-row query tiles of all query
+// partitions i with (i, j) COMPUTE, in the order of i, taken two at a time: a partition with an odd number of tiles
+// shares its last item with the first tile of the next one (both attend to the same keys), so no item runs half
+// empty except the last of a KV partition.  Items are listed by j, so neighbours in the list share K/V.
+// (called by all 1024 threads of worklist_kernel; is_compute = this thread's pair (i, j) = (e / P, e % P) is COMPUTE)
+__device__ void build_tile_pairs(bool is_compute, const int32_t *off, int P, int4 *out) {
+    __shared__ uint8_t flag[DT_MAX_P * DT_MAX_P];
+    __shared__ int items_of[DT_MAX_P], base_of[DT_MAX_P + 1];
+    const int e = threadIdx.x;
+    if (e < P * P) flag[e] = is_compute ? 1 : 0;
+    __syncthreads();
+    if (e < P) {   // thread j: tiles of column j
+        int tiles = 0;
+        for (int i = 0; i < P; ++i)
+            if (flag[i * P + e]) tiles += (off[i + 1] - off[i] + ATTN_TILE - 1) / ATTN_TILE;
+        items_of[e] = (tiles + 1) / 2;
+    }
+    __syncthreads();
+    if (e == 0) {
+        int acc = 0;
+        for (int j = 0; j < P; ++j) { base_of[j] = acc; acc += items_of[j]; }
+        base_of[P] = acc;
+        out[0] = make_int4(acc, 0, 0, 0);
+    }
+    __syncthreads();
+    // one warp per KV partition j: lane l writes the items l, l + 32, ... of the column
+    const int j = e >> 5, lane = e & 31;
+    if (j < P) {
+        for (int it = lane; it < items_of[j]; it += 32) {
+            int4 rec = make_int4(0, 0, -1, 0);
+            int seen = 0;             // tiles of the column before partition i
+            for (int i = 0; i < P; ++i) {
+                if (!flag[i * P + j]) continue;
+                const int t_i = (off[i + 1] - off[i] + ATTN_TILE - 1) / ATTN_TILE;
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int g = 2 * it + q - seen;      // index of the item's q-th tile within partition i
+                    if (g >= 0 && g < t_i) {
+                        if (q == 0) { rec.x = i | (j << 8); rec.y = g; }
+                        else { rec.z = i; rec.w = g; }
+                    }
+                }
+                seen += t_i;
+            }
+            out[1 + base_of[j] + it] = rec;
+        }
+    }
 }
 
 // Decisions for a grouped cache (Section 4.2.1 - 4.2.3): W[i][s] from the partial sums; every non-local slot
@@ -403,8 +455,8 @@ cudaError_t launch_plan_final(const PlanFinalParams &p, cudaStream_t stream) {
 }
 
 cudaError_t launch_worklist(const uint8_t *mask, int32_t *tc, int32_t *worklist, int32_t *status, const SlotRange *slot_tab,
-                            int P, int S, int group_mode, int step, cudaStream_t stream) {
-    worklist_kernel<<<1, 1024, 0, stream>>>(mask, tc, worklist, status, slot_tab, P, S, group_mode, step);
+                            int P, int S, int group_mode, int step, const int32_t *off, int4 *tile_pairs, cudaStream_t stream) {
+    worklist_kernel<<<1, 1024, 0, stream>>>(mask, tc, worklist, status, slot_tab, P, S, group_mode, step, off, tile_pairs);
     return cudaGetLastError();
 }
 
