@@ -597,6 +597,15 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         uint32_t s_phase = 0, o_phase = 0, pv_phase = 0;
         bool ok = true;
         StateT *o_state = static_cast<StateT *>(p.o_state);
+        if constexpr (C::PREFETCH) {
+            // D = 64: the two warpgroups share the MUFU and are otherwise independent (an MMA warp each).  Started
+            // half a tile apart, one takes its exponentials while the other waits for S, stores P or runs its epilogue
+            // (measured +1 %); nothing brings them back into step.
+            if (q == 1) {
+                const long long t0 = clock64();
+                while (clock64() - t0 < 1200) {}
+            }
+        }
 
         for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
             WorkItem it;
