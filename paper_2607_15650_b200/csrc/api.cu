@@ -487,6 +487,7 @@ static dt_status plan_impl(dt_ctx *ctx, double eps, double target_fraction, int3
     pp.off = ctx->off_dev;
     pp.partials = ctx->plan_partials_dev;
     pp.nonempty = ctx->group_size0 > 1 ? ctx->nonempty_dev : nullptr;
+    pp.only_if = nullptr;
     pp.P = c.P; pp.S = ctx->S; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
     pp.R = (long long)c.B * c.H * c.L;
     cudaError_t e = cudaSuccess;
@@ -753,8 +754,10 @@ dt_status dt_planner_commit(dt_ctx *ctx, void *stream) {
     pp.off = ctx->off_dev;
     pp.partials = ctx->plan_partials_dev;
     pp.nonempty = ctx->group_size0 > 1 ? ctx->nonempty_dev : nullptr;
+    pp.only_if = nullptr;
     pp.P = c.P; pp.S = ctx->S; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
     pp.R = (long long)c.B * c.H * c.L;
+    pp.only_if = &ctx->planner_state_dev->is_anchor;   // Eq. 8's weights are refreshed at anchors only
     cudaError_t e = dt::launch_plan_partial(pp, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "plan launch");
     dt::PlannerParams p = planner_params(ctx);
@@ -844,6 +847,7 @@ dt_status dt_group_compose(dt_ctx *ctx, void *stream) {
         pp.off = ctx->off_dev;
         pp.partials = ctx->plan_partials_dev;
         pp.nonempty = ctx->nonempty_dev;
+        pp.only_if = nullptr;
         pp.P = c.P; pp.S = ctx->S; pp.BH = c.B * c.H; pp.L = c.L; pp.chunks = ctx->plan_chunks;
         pp.R = (long long)R;
         e = dt::launch_plan_partial(pp, st);

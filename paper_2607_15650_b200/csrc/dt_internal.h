@@ -83,6 +83,7 @@ struct PlanParams {
     const float *lse_state;  // [S][R]
     const int32_t *off;      // device, P+1
     const uint32_t *nonempty; // device, P words: slots that exist for the query partition (null = all)
+    const int *only_if;      // device flag, or null: the kernel returns at once while it is 0 (planner: not an anchor)
     float *partials;         // [BH][P][chunks][S]
     int P, S, BH, L, chunks;
     long long R;

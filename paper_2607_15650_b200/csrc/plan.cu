@@ -30,6 +30,7 @@ constexpr int PLAN_THREADS = 256;
 
 template <int PMAX>
 __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS(PMAX)) plan_partial_kernel(PlanParams p) {
+    if (p.only_if != nullptr && *p.only_if == 0) return;
     const int c = blockIdx.x, i = blockIdx.y, bh = blockIdx.z;
     const int P = p.S;   // columns: cache slots (pair mode: one per KV partition)
     const uint32_t have = p.nonempty ? p.nonempty[i] : 0xFFFFFFFFu;   // slots that exist for this query partition
@@ -541,6 +542,7 @@ extern "C" dt_status dt_plan_static(const float *lse_state_dev, const int32_t *p
     pp.off = off_dev;
     pp.partials = partials;
     pp.nonempty = nullptr;
+    pp.only_if = nullptr;
     pp.P = P; pp.S = P; pp.BH = B * H; pp.L = L; pp.chunks = chunks;
     pp.R = (long long)B * H * L;
     if (dt::launch_plan_partial(pp, st) != cudaSuccess) return DT_ERR_CUDA;
