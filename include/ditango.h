@@ -62,7 +62,7 @@ typedef enum {
     DT_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (text in dt_last_error)        */
     DT_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired; the kernel returned normally   */
     DT_ERR_RANGE = 6        /* bf16 inputs: within one 128-key tile a logit (times log2 e) rose more than
-                               about 120 above everything the row had seen before (exp2 overflows fp32);
+                               about 100 above everything the row had seen before (exp2 overflows fp32);
                                the states of that launch are not valid.  fp16 inputs have no such limit. */
 } dt_status;
 

@@ -913,7 +913,7 @@ dt_status dt_poll(dt_ctx *ctx) {
     if (word & dt::STATUS_WAIT_TIMEOUT) return fail(ctx, DT_ERR_TIMEOUT, "a bounded device-side wait expired");
     if (word & dt::STATUS_REUSE_EMPTY) return fail(ctx, DT_ERR_STATE, "REUSE of a pair that was never computed");
     if (word & dt::STATUS_LOGIT_RANGE)
-        return fail(ctx, DT_ERR_RANGE, "a logit rose more than 120 binades above the running reference within one K/V tile");
+        return fail(ctx, DT_ERR_RANGE, "a logit rose more than 100 binades above the running reference within one K/V tile");
     return DT_OK;
 }
 

@@ -24,10 +24,11 @@
 // accumulating in O.  While one query tile is in softmax the tensor core works on the other
 // (ping-pong).  With D = 64 there is room for S0 | S1 | P0 | P1 | O0 | O1: P has columns of its own and
 // the next tile's Q K^T is issued as soon as the softmax has read S (see Cfg::PREFETCH).
-// P is computed against the reference maximum of the earlier tiles; only when a row sum of P reaches
-// ROWSUM_TRIGGER is the tile's own maximum taken and, if it lies more than 2^RESCALE_THRESHOLD above the
-// reference, the reference moved and O, l rescaled: stale references cancel exactly in OUT = O / l and
-// LSE = m + log l.
+// P is computed against the reference maximum m of the earlier tiles, never against the tile's own: stale
+// references cancel exactly in OUT = O / l and LSE = m + log l.  bf16 inputs: when a row's running sum l reaches
+// LSUM_TRIGGER, m moves up by floor(log2 l) binades and O, l are scaled by that power of two (exact).  fp16
+// inputs (P overflows at 2^16): when a tile's row sum reaches ROWSUM_TRIGGER the tile's own maximum is taken and,
+// if it lies more than 2^RESCALE_THRESHOLD above the reference, the reference moved and P computed again.
 // Epilogue: the rows leave through warp-private shared-memory tiles so that the cache is written in whole
 // 128-byte lines; the fused mode (dt_attn_fused) composes the fresh state with the composed reuse state in
 // registers and stores the attention output itself.
@@ -57,7 +58,8 @@ constexpr int LAUNCH_REGS = 168, REGS_SOFTMAX = 208, REGS_PRODUCER = 88;
 static_assert((REGS_SOFTMAX - LAUNCH_REGS) * NUM_SOFTMAX_THREADS <= (LAUNCH_REGS - REGS_PRODUCER) * 128,
               "softmax warps would wait forever for registers nobody releases");
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // SM clock cycles: about 2 s
-constexpr float ROWSUM_TRIGGER = 512.0f;   // a row sum of P at or above this sends the tile through the slow path
+constexpr float ROWSUM_TRIGGER = 512.0f;   // fp16 inputs: a row sum of P at or above this sends the tile through the slow path
+constexpr float LSUM_TRIGGER = 16777216.0f;   // bf16 inputs: a running sum l at or above 2^24 moves the row's reference
 constexpr float RESCALE_THRESHOLD = 1.0f;  // log2 units: in the slow path the reference moves if the maximum grew by more
 // Key pairs (of every 8) whose exp2 runs as a cubic on the FMA pipe instead of the MUFU.  D = 64 is bound by the
 // exponentials (2048 MUFU cycles per 256 x 128 tile pair against 1536 of MMA issue), and one pair in eight measured
@@ -221,12 +223,12 @@ __device__ __forceinline__ void load_state_chunk(const __nv_bfloat16 *src, float
     }
 }
 
-// A row sum of P that reached ROWSUM_TRIGGER moves the row's reference up by e = floor(log2(row sum)) binades:
+// A running sum l that reached LSUM_TRIGGER moves the row's reference up by e = floor(log2(l)) binades:
 // this thread's row of O (fp32, D columns) times 2^-e, in place; returns e (0 for a row below the trigger).
 // Out of line: it runs once in many tiles and would only lengthen the softmax loop.
 template <int D>
 __device__ __noinline__ int move_reference(uint32_t o_tmem, float row_sum) {
-    const bool need = !(row_sum < ROWSUM_TRIGGER);   // also true for inf / NaN
+    const bool need = !(row_sum < LSUM_TRIGGER);   // also true for inf / NaN
     const int e = need ? min(((__float_as_int(row_sum) >> 23) & 0xFF) - 127, 126) : 0;
     const float alpha = __int_as_float((127 - e) << 23);
 #pragma unroll 1
@@ -611,13 +613,12 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             WorkItem it;
             if (!decode_work<FUSED>(p, npairs, w, it)) continue;
             float m_used = -INFINITY, l_sum = 0.f;
-            [[maybe_unused]] float rs_prev = 0.f;   // bf16 inputs: row sum of the previous tile's P
             for (int t = 0; t < it.tiles; ++t) {
                 const int valid = it.template tile<FUSED>(t).y;   // keys of this tile that count (issued before the wait)
-                // One vote tells that S_t has arrived for every lane and (bf16 inputs) that no row of the warp reached
-                // ROWSUM_TRIGGER with the previous tile's P.
+                // One vote tells that S_t has arrived for every lane and (bf16 inputs) that no row's running sum l has reached
+                // LSUM_TRIGGER.
                 const bool s_here = mbar_wait_bounded(bars.s_full + 8 * q, s_phase, abort_ptr, WAIT_LIMIT_CYCLES);
-                const bool fine = __all_sync(0xFFFFFFFFu, s_here && (FP16 || rs_prev < ROWSUM_TRIGGER));
+                const bool fine = __all_sync(0xFFFFFFFFu, s_here && (FP16 || l_sum < LSUM_TRIGGER));
                 s_phase ^= 1u;
                 tc_fence_after();
                 [[maybe_unused]] bool pv_waited = false;
@@ -626,17 +627,18 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     if (!ok) break;
                     if constexpr (!FP16) {
                         // bf16 probabilities have fp32's exponent range, so a tile's P is exact whatever the reference, and
-                        // the reference can move after the fact: when the previous tile's row sum reached ROWSUM_TRIGGER, m
-                        // moves up by e = floor(log2(row sum)) binades and O and l are multiplied by 2^-e, which is exact.
-                        // Made here, a tile late, the move is off the S -> P chain and the logits of a tile never have to
-                        // be kept for a second pass.  (S_t complete tells that P_{t-1} V_{t-1} is -- D = 64: pv_done does.)
+                        // the reference can move after the fact: when the running sum l of a row has reached LSUM_TRIGGER, m
+                        // moves up by e = floor(log2(l)) binades and O and l are multiplied by 2^-e, which is exact.  The test
+                        // costs one compare on a value that is live anyway; made here, at the top of the next tile, the move
+                        // is off the S -> P chain and the logits of a tile never have to be kept for a second pass.
+                        // (S_t complete tells that P_{t-1} V_{t-1} is -- D = 64: pv_done does.)
                         if constexpr (C::PREFETCH) {
                             ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_CYCLES));
                             pv_phase ^= 1u;
                             pv_waited = true;
                             tc_fence_after();
                         }
-                        const int e = move_reference<D>(o_tmem, rs_prev);
+                        const int e = move_reference<D>(o_tmem, l_sum);
                         m_used += (float)e;
                         l_sum *= __int_as_float((127 - e) << 23);
                     }
@@ -657,13 +659,12 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     for (int c = 0; c < 128; ++c)
                         if (c >= valid) s[c >> 5][c & 31] = 0xFF800000u;  // -inf
                 }
-                // P = exp2(s * scale_log2 - m_used) with the reference maximum of the earlier tiles.  While
-                // the row sum of P stays below ROWSUM_TRIGGER no element can have exceeded it, so the tile's
-                // own maximum is not needed.  Only when a sum reaches it (rare after the first tiles) is the
-                // maximum taken and, if it lies more than 2^RESCALE_THRESHOLD above the reference, the
-                // reference moved, O and l rescaled and P computed again; afterwards every P <= 2 and the
-                // row sum is at most 256, so the slow path does not fire again until the maximum grows.
-                // The result does not depend on the reference: it cancels in OUT = O / l and LSE = m + log l.
+                // P = exp2(s * scale_log2 - m_used) with the reference maximum of the earlier tiles; the result does not
+                // depend on the reference: it cancels in OUT = O / l and LSE = m + log l.  fp16 inputs: while the row
+                // sum of P stays below ROWSUM_TRIGGER no element can have exceeded it, so the tile's own maximum is not
+                // needed; only when a sum reaches it (rare after the first tiles) is the maximum taken and, if it lies
+                // more than 2^RESCALE_THRESHOLD above the reference, the reference moved, O and l rescaled and P
+                // computed again.  bf16 inputs: see the top of the tile.
                 const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
                 auto row_max = [&]() -> float {   // raw maximum of the row: four chains of three-input max
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -732,7 +733,6 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     }
                 }
                 l_sum += rs;
-                if constexpr (!FP16) rs_prev = rs;
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bars.p_full + 8 * q);
@@ -751,7 +751,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             const int q_row = my_qrow + row_in_tile;   // this thread's query row (global token index)
             const float inv_l = 1.0f / l_sum;
             if constexpr (!FP16) {
-                // a sum that is not finite: within one K/V tile a logit rose more than about 120 binades above the
+                // a sum that is not finite: within one K/V tile a logit rose more than about 100 binades above the
                 // reference (exp2 overflowed); the launch's states are not valid (dt_poll: DT_ERR_RANGE)
                 if (row_valid && !(l_sum <= 3.0e38f)) atomicOr(p.status, STATUS_LOGIT_RANGE);
             }
