@@ -464,7 +464,10 @@ def run_cuda(args, wl):
                 import torch.distributed as dist
                 dist.barrier()           # every replica runs its end-to-end step at the same time
             t0 = time.perf_counter()
-            ctx.dt_step_host(qh, kh, vh, mh, t, oh, lh, ws)
+            ctx.dt_step_host(qh, kh, vh, mh, t, oh, lh, ws)     # returns when out and lse are in host memory
+            if not args.shard_heads:
+                ctx.dt_plan(masks[cur ^ 1], target_fraction=frac, w_dev=W)   # the next step's plan, as in the timed loop
+                torch.cuda.synchronize()
             times.append(time.perf_counter() - t0)
             t += 1
         e2e_s = max_over_ranks(float(np.mean(times[1:])), world, dev)
@@ -472,7 +475,7 @@ def run_cuda(args, wl):
         d2h = oh.numel() * 2 + lh.numel() * 4
         e2e = {"value": job_throughput(e2e_s), "unit": UNIT, "ms_per_step": 1e3 * e2e_s,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "includes": "dt_step_host: H2D q,k,v,mask + dt_attn_states + dt_state_merge + D2H out,lse"}
+               "includes": "dt_step_host: H2D q,k,v,mask + dt_attn_states + dt_state_merge + D2H out,lse; then dt_plan"}
         del ws
 
     if rank != 0:
