@@ -83,12 +83,12 @@ def _run_full_size(name, fraction, n_samples, n_selective, state_dtype=binding.D
             rel = np.abs(W_ref - ref_eps) / ref_eps
             decidable = (rel > 1e-4) | ~offd
             margin = rel[offd].min()
-            verdict = "well-conditioned" if margin > 1e-4 else f"ILL-CONDITIONED ({int((~decidable).sum())} pairs undecidable)"
-            print(f"[plan margin] {name} f={fraction}: min |W - eps| / eps = {margin:.3e} -> {verdict}; "
+            conditioning = "well-conditioned" if margin > 1e-4 else f"ILL-CONDITIONED ({int((~decidable).sum())} pairs undecidable)"
+            print(f"[plan margin] {name} f={fraction}: min |W - eps| / eps = {margin:.3e} -> {conditioning}; "
                   f"GPU mask == oracle mask on all decidable pairs: {bool((got_mask == ref_mask)[decidable].all())}")
             if record is not None:
                 record("plan_margin", float(margin))
-                record("plan_conditioning", verdict)
+                record("plan_conditioning", conditioning)
             assert (got_mask == ref_mask)[decidable].all()
             assert decidable.sum() >= P * P - 2, "more than two undecidable pairs: the workload's plan is degenerate"
             # locality of the synthetic workload: contribution falls with partition distance
