@@ -22,8 +22,10 @@
  * first-order error propagation identity (Eq. 4) by finite differences,
  * row sums of w, closed-form softmax for synthetic LSE, equality case of
  * the threshold.  The target-fraction rule (orc_target_fraction) follows a
- * reading of the paper's "eps as a percentile matching a target ratio" and is
- * pinned only by its invariants (count, diagonal, monotonicity).
+ * reading of the paper's "eps as a percentile matching a target ratio"; what
+ * it computes is pinned by its invariants (count, diagonal, monotonicity) and
+ * by a hand-checked two-valued measure that fixes the tie order and the
+ * midpoint threshold.
  */
 #include <math.h>
 #include <stdint.h>

@@ -1,4 +1,4 @@
-// dt_attn_states: Eq. 1 for every COMPUTE pair -- flash attention of one query block of
+// dt_attn_states: Eq. 1 for every COMPUTE pair -- flash attention of the query tiles of
 // partition i against the keys of partition j only, emitting the partition-normalised output
 // OUT_ij and LSE_ij straight into the state cache.  REUSE pairs never appear in the work list,
 // so they cost no instruction and no byte.  With a grouped cache (Section 4.2.1) a work item is a
@@ -15,8 +15,10 @@
 //   warp 8           TMA producer: Q tiles once per work item, K and V tiles through a ring
 //   warp 9           MMA issuer: the whole warp runs the (warp-uniform) control flow and address arithmetic, one
 //                    lane issues tcgen05.mma / tcgen05.commit -- measured 4 % faster than a single-lane branch
-//   warp 10          K/V watcher: adds its arrival to p_full[0] once V_t and K_{t+1} have landed, and hands the
-//                    stages and the place of Q back to the producer once the MMAs that read them are done
+//   warp 10          D = 128: K/V watcher -- adds its arrival to p_full[0] once V_t and K_{t+1} have landed, and hands
+//                    the stages and the place of Q back to the producer once the MMAs that read them are done.
+//                    D = 64: the second MMA warp (one per query tile; each waits for its K/V tiles itself and hands
+//                    them back with commits of its own)
 //   warp 11          idle (completes the producer warpgroup for the register hand-over)
 // TMEM (512 columns): S0 | S1 | O0 | O1.  S_t = Q K_t^T (fp32) lands in S; the softmax warpgroup
 // reads its row, writes P = exp2(s*scale*log2e - m) back over S as packed bf16 (fp16 for fp16 inputs),
