@@ -105,6 +105,21 @@ def test_ragged_partitions_and_tails(D, grid, n_text, offsets):
     run.step(np.eye(P, dtype=np.uint8), check_states=True)
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_query_tiles_pair_across_partitions(D):
+    """The attention kernel's work items are pairs of 128-row query tiles that attend to the same KV partition, taken
+    from all query partitions that compute it: partitions of 3, 1, 5 and 2 tiles (the last ones ragged) make items whose
+    two tiles belong to different query partitions, under masks that leave columns with one, several or all of them.
+    Every pair state and the merged output, element by element."""
+    offsets = [0, 300, 420, 1000, 1190]                  # 300, 120, 580, 190 rows: 3, 1, 5, 2 tiles
+    wl = inputs.Workload("tilepairs", 1, 2, D, (2, 17, 35), 0, 4, 3, 0.05)
+    assert wl.L == offsets[-1]
+    run = Run(wl, offsets=offsets, seed=8)
+    run.step(np.ones((4, 4), np.uint8), check_states=True)
+    run.step(np.array([[1, 0, 1, 0], [1, 1, 0, 0], [0, 1, 1, 1], [1, 0, 0, 1]], np.uint8), check_states=True)
+    run.step(np.eye(4, dtype=np.uint8), check_states=True)
+
+
 def test_batch_two_and_bf16_state_cache():
     wl = inputs.Workload("b2", 2, 2, 128, (2, 10, 13), 0, 2, 2, 0.05)
     run = Run(wl, state_dtype=binding.DT_STATE_BF16, seed=2)
