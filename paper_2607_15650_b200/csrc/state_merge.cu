@@ -85,7 +85,7 @@ struct MergeCfg {
     }
     static int staged(int mode, int P) { return chunked(mode, P) ? MERGE_CHUNK : P; }
     static size_t smem_bytes(int mode, int P) {
-        return (size_t)staged(mode, P) * rows(mode, P) * ROW_BYTES + (size_t)rows(mode, P) * (DT_MAX_P + 1) * sizeof(float) + 40 + 64;
+        return (size_t)staged(mode, P) * rows(mode, P) * ROW_BYTES + (size_t)rows(mode, P) * (DT_MAX_P + 1 + 2) * sizeof(float) + 64 + 64;
     }
 };
 
@@ -118,23 +118,49 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
     int *abort_flag = reinterpret_cast<int *>(bar_ptr + 1);
     int *nsrc_s = abort_flag + 1;
     uint8_t *src_s = reinterpret_cast<uint8_t *>(abort_flag + 2);                             // [NS] source ids in staging order
+    float *rowz_s = reinterpret_cast<float *>(src_s + ((NS + 3) & ~3));                       // [ROWS] sum of a row's weights
+    float *rowm_s = rowz_s + ROWS;                                                            // [ROWS] a row's largest log-sum-exp
     const uint32_t bar = smem_u32(bar_ptr);
 
     const long long row0 = p.row_begin + (long long)blockIdx.x * ROWS;
     const int valid = (int)min((long long)ROWS, p.row_begin + p.row_count - row0);   // rows of this block that exist
     const uint32_t bytes = (uint32_t)valid * Cf::ROW_BYTES;
 
-    // query partition of a cache row (token index l = row mod L); the offsets travel as kernel
-    // parameters, so this needs no memory access
-    auto partition_of = [&](long long row) -> int {
-        const int l = (int)(row % p.L);
-        int i = 0;
+    // Token index of a cache row (row mod L) and its query partition.  The offsets travel as kernel parameters, so
+    // this needs no memory access; it is instruction count that matters here (the subset modes were issue-bound on
+    // a 64-bit modulo and a linear search per looked-up row): 32-bit arithmetic whenever the row count allows it, a
+    // binary search once per thread, and from there a step or two along the offsets for the block's other rows.
+    const bool rows32 = (p.R < (1ll << 31));
+    auto mod_L = [&](long long row) -> int {
+        return rows32 ? (int)((uint32_t)row % (uint32_t)p.L) : (int)(row % p.L);
+    };
+    auto partition_of_l = [&](int l) -> int {
+        int lo = 0, hi = p.P;
+#pragma unroll 1
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (p.off_val[mid] <= l) lo = mid; else hi = mid;
+        }
+        return lo;
+    };
+    // (only the threads that look rows up: thread 0 for the block's source list, and those that fetch log-sum-exps)
+    const bool need_parts = ((MODE != MERGE_ALL) || (p.sel_bits != nullptr)) &&
+                            (threadIdx.x == 0 || (int)threadIdx.x < valid * nslots);
+    const int l_first = need_parts ? mod_L(row0) : 0;                 // token index of the block's first row
+    const int i_first = need_parts ? partition_of_l(l_first) : 0;     // and its query partition
+    // query partition of the block's r-th row
+    auto partition_of_row = [&](int r) -> int {
+        int l = l_first + r, i = i_first;
+        if (l >= p.L) {               // the block runs into the next (b, h): start over from partition 0
+            l %= p.L;
+            i = 0;
+        }
 #pragma unroll 1
         while (i + 1 < p.P && p.off_val[i + 1] <= l) ++i;
         return i;
     };
     // per query partition, bit j set = slot j takes part (prepared on the device from the mask)
-    auto sel_of = [&](long long row) -> uint32_t { return __ldg(p.sel_bits + partition_of(row)); };
+    auto sel_of = [&](int r) -> uint32_t { return __ldg(p.sel_bits + partition_of_row(r)); };
     const uint32_t all_bits = (P == 32) ? 0xFFFFFFFFu : ((1u << P) - 1u);
     // copies for the sources [first, first + count) of the staging order into tile slots 0..count-1
     auto stage = [&](int first, int count) {
@@ -156,9 +182,9 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
             // sources any row of the block needs; its rows are consecutive, so only the partitions of its
             // two ends and those between them matter
             uint32_t need = 0;
-            const int i0 = partition_of(row0), i1 = partition_of(row0 + valid - 1);
+            const int i0 = i_first, i1 = partition_of_row(valid - 1);
             if (valid >= p.L) { for (int i = 0; i < p.P; ++i) need |= __ldg(p.sel_bits + i); }   // a block longer than the sequence
-            else if (i0 <= i1 && (row0 % p.L) + valid <= p.L) { for (int i = i0; i <= i1; ++i) need |= __ldg(p.sel_bits + i); }
+            else if (i0 <= i1 && l_first + valid <= p.L) { for (int i = i0; i <= i1; ++i) need |= __ldg(p.sel_bits + i); }
             else { for (int i = 0; i < p.P; ++i) if (i >= i0 || i <= i1) need |= __ldg(p.sel_bits + i); }   // wraps into the next (b, h)
             nsrc = 0;
             for (int j = 0; j < P; ++j) if (need >> j & 1u) src_s[nsrc++] = (uint8_t)j;
@@ -173,7 +199,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
         const int r = e / nslots, j = e - r * nslots;
         float x = -INFINITY;
         if (j < P) {
-            const uint32_t sel = (MODE == MERGE_ALL && p.sel_bits == nullptr) ? all_bits : sel_of(row0 + r);
+            const uint32_t sel = (MODE == MERGE_ALL && p.sel_bits == nullptr) ? all_bits : sel_of(r);
             if (sel >> j & 1u) x = __ldg(p.lse_state + (long long)j * p.R + row0 + r);
         } else {
             x = __ldg(p.comp_lse + row0 + r);
@@ -182,19 +208,41 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
     }
     __syncthreads();   // also publishes the mbarrier initialisation and the staging order
 
+    // The weights exp(LSE_j - M) of a row are the same for every thread that works on it: eight lanes per row form them
+    // once -- only the block's sources can carry mass, every other entry of the row is -inf -- and leave them in place
+    // of the log-sum-exps, with the row's maximum M and the sum Z beside them.  (Every thread of the row used to repeat
+    // this; the subset modes were bound by instruction issue, not by memory.)
+    const int nsrc = *nsrc_s;
+    {
+        const int wr = threadIdx.x >> 3, wl = threadIdx.x & 7;
+        if (wr < ROWS) {            // ROWS * 8 <= 256 threads, whole warps
+            float *row_lse = lse_s + wr * NS;
+            float m = -INFINITY;
+            for (int k = wl; k < nsrc; k += 8) m = fmaxf(m, row_lse[(MODE == MERGE_ALL) ? k : (int)src_s[k]]);
+#pragma unroll
+            for (int sft = 1; sft < 8; sft <<= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, sft));
+            float z = 0.f;
+            for (int k = wl; k < nsrc; k += 8) {
+                const int src = (MODE == MERGE_ALL) ? k : (int)src_s[k];
+                const float w = (m == -INFINITY) ? 0.f : __expf(row_lse[src] - m);
+                row_lse[src] = w;
+                z += w;
+            }
+#pragma unroll
+            for (int sft = 1; sft < 8; sft <<= 1) z += __shfl_xor_sync(0xFFFFFFFFu, z, sft);
+            if (wl == 0) { rowz_s[wr] = z; rowm_s[wr] = m; }
+        }
+    }
+    __syncthreads();
     const int r = threadIdx.x / TPR, lane = threadIdx.x % TPR;
     const bool active = r < valid;
-    const float *my_lse = lse_s + (active ? r : 0) * NS;
-    float M = -INFINITY, Z = 0.f;
-    for (int j = 0; j < nslots; ++j) M = fmaxf(M, my_lse[j]);
+    const float *my_w = lse_s + (active ? r : 0) * NS;
+    const float Z = rowz_s[active ? r : 0], M = rowm_s[active ? r : 0];
     const bool empty = (M == -INFINITY);   // no source has any mass: output 0, LSE = -inf
-    if (!empty)
-        for (int j = 0; j < nslots; ++j) Z += __expf(my_lse[j] - M);
 
     float acc[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
-    const int nsrc = *nsrc_s;
     const StateT *mine = tile + (size_t)(active ? r : 0) * D + lane * VEC;
     for (int first = 0, phase = 0; first < nsrc; first += staged, phase ^= 1) {
         const int count = min(nsrc - first, staged);
@@ -215,7 +263,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
 #pragma unroll 4
             for (int k = 0; k < count; ++k) {
                 const int src = (MODE == MERGE_ALL) ? first + k : (int)src_s[first + k];
-                const float wt = __expf(my_lse[src] - M);
+                const float wt = my_w[src];
                 if (wt != 0.f) {   // rows of another partition may not use this source at all
                     float v[VEC];
                     StateVec<StateT>::load(mine + (size_t)k * ROWS * D, v);
@@ -237,7 +285,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) state_merge_kernel(const __grid
         if (lane == 0) p.comp_lse_out[row] = lse_row;
         return;
     }
-    const long long bh = row / p.L;
+    const long long bh = rows32 ? (long long)((uint32_t)row / (uint32_t)p.L) : row / p.L;
     const int l = (int)(row - bh * p.L);
     const int b = (int)(bh / p.H), h = (int)(bh - (long long)b * p.H);
     __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(p.out) + b * p.sb + l * p.sl + h * p.sh + lane * VEC;
@@ -253,7 +301,7 @@ cudaError_t launch_mode(const MergeParams &p, cudaStream_t stream) {
     const long long blocks = (p.row_count + rows - 1) / rows;
     if (blocks <= 0 || blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(state_merge_kernel<StateT, D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         MERGE_STAGE_BYTES + MERGE_THREADS * (DT_MAX_P + 1) * (int)sizeof(float) + 128);
+                                         MERGE_STAGE_BYTES + MERGE_THREADS * (DT_MAX_P + 1 + 2) * (int)sizeof(float) + 256);
     if (e != cudaSuccess) return e;
     state_merge_kernel<StateT, D, MODE><<<(unsigned)blocks, MERGE_THREADS, smem, stream>>>(p, rows, Cf::staged(MODE, p.S));
     return cudaGetLastError();
