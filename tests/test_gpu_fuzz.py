@@ -41,7 +41,11 @@ def _random_case(seed):
     return rng, D, B, H, P, grid, n_text, offsets, g, state_dtype, fp16
 
 
-@pytest.mark.parametrize("seed", range(int(os.environ.get("DT_FUZZ_CASES", "24"))))
+# DT_FUZZ_CASES / DT_FUZZ_FIRST: how many seeds and the first one (a longer soak takes a later range)
+_FIRST = int(os.environ.get("DT_FUZZ_FIRST", "0"))
+
+
+@pytest.mark.parametrize("seed", range(_FIRST, _FIRST + int(os.environ.get("DT_FUZZ_CASES", "24"))))
 def test_random_configuration(seed):
     rng, D, B, H, P, grid, n_text, offsets, g, state_dtype, fp16 = _random_case(seed)
     wl = inputs.Workload(f"fuzz{seed}", B, H, D, grid, n_text, P, 3, 0.05)
