@@ -71,7 +71,15 @@ constexpr float RESCALE_THRESHOLD = 1.0f;  // log2 units: in the slow path the r
 #define DT_POLY_PER_8_D64 1
 #endif
 #ifndef DT_POLY_PER_8_D128
-#define DT_POLY_PER_8_D128 0
+#define DT_POLY_PER_8_D128 1
+#endif
+#ifndef DT_D128_SHARED_S
+#define DT_D128_SHARED_S 1
+#endif
+// Shared place for S: after how many of a tile's four 32-key pieces the softmax asks for the next tile's S (0: only
+// when P is stored).
+#ifndef DT_S_REQ_PIECE
+#define DT_S_REQ_PIECE 2
 #endif
 
 template <int D>
@@ -84,23 +92,32 @@ struct Cfg {
     static constexpr int KV_BYTES = STAGES * TILE_BYTES;
     static constexpr int OUT_STAGE_BYTES = ATTN_TILE * 128;   // epilogue staging per query tile: 4 warps x [32 rows x 128 bytes]
     static constexpr int OUT_BYTES = ATTN_NQ * OUT_STAGE_BYTES;
-    static constexpr int NBARS = 2 + 2 * STAGES + 6 * ATTN_NQ;
+    static constexpr int NBARS = 2 + 2 * STAGES + 7 * ATTN_NQ;
     static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + Q_BYTES + KV_BYTES + OUT_BYTES + NBARS * 8 + 64;
     // TMEM columns.  D = 128 fills all 512 (S0 | S1 | O0 | O1) and P has to live over S.  D = 64 leaves 128 columns:
     // there P gets its own place (S0 | S1 | P0 | P1 | O0 | O1), so S may be overwritten as soon as the softmax has
     // read it and the next tile's Q K^T runs while this tile's exponentials are being taken.
-    static constexpr bool PREFETCH = (D == 64);
+    // D = 128 with DT_D128_SHARED_S: S | P0 | P1 | O0 | O1 -- the two query tiles share ONE place for S.  A softmax
+    // thread takes its whole row of S into registers as soon as it arrives, so the place is free again a few dozen
+    // cycles after every Q K^T, and giving the second tile's 128 columns to P0 | P1 takes P_t V_t out of the way of
+    // Q K_{t+1}^T: the S -> P -> S chain of a query tile loses P V's 512 cycles.
+    static constexpr bool SHARED_S = (D == 128) && (DT_D128_SHARED_S != 0);
+    static constexpr bool PREFETCH = (D == 64) || SHARED_S;   // P has columns of its own; one MMA warp per query tile
+    static constexpr int S_REQ = SHARED_S ? DT_S_REQ_PIECE : 0;
     static constexpr int POLY_PER_8 = (D == 64) ? DT_POLY_PER_8_D64 : DT_POLY_PER_8_D128;
-    static constexpr int S_COL = 0;                                              // S tile q: S_COL + q*128
-    static constexpr int P_COL = PREFETCH ? ATTN_NQ * 128 : 0;                   // P tile q: P_COL + q*(PREFETCH ? 64 : 128)
+    static constexpr int S_COL = 0;                                              // S tile q: S_COL + q*S_STRIDE
+    static constexpr int S_STRIDE = SHARED_S ? 0 : 128;
+    static constexpr int S_TILES = SHARED_S ? 1 : ATTN_NQ;
+    static constexpr int P_COL = PREFETCH ? S_TILES * 128 : 0;                   // P tile q: P_COL + q*P_STRIDE
     static constexpr int P_STRIDE = PREFETCH ? 64 : 128;
-    static constexpr int O_COL = PREFETCH ? ATTN_NQ * 128 + ATTN_NQ * 64 : ATTN_NQ * 128;   // O tile q: O_COL + q*D
+    static constexpr int O_COL = PREFETCH ? S_TILES * 128 + ATTN_NQ * 64 : ATTN_NQ * 128;   // O tile q: O_COL + q*D
+    static_assert(O_COL + ATTN_NQ * D <= 512, "beyond the tensor memory of an SM");
 };
 
 struct Bars {
     uint32_t q_full, q_empty;
     uint32_t kv_full, kv_empty;   // + 8*stage
-    uint32_t s_full, p_full, o_full, o_free, pv_done, s_free;  // + 8*q
+    uint32_t s_full, p_full, o_full, o_free, pv_done, s_free, s_req;  // + 8*q
 };
 
 // D = 64 (Cfg::PREFETCH): place of an item's K/V tiles in the order they are loaded and consumed --
@@ -271,7 +288,8 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     bars.o_full = bars.p_full + 8 * ATTN_NQ;
     bars.o_free = bars.o_full + 8 * ATTN_NQ;
     bars.pv_done = bars.o_free + 8 * ATTN_NQ;   // D = 64 only: the PV MMAs that read P[q] have completed
-    bars.s_free = bars.pv_done + 8 * ATTN_NQ;   // D = 64 only: S[q] has been read (and the next K tile has landed)
+    bars.s_free = bars.pv_done + 8 * ATTN_NQ;   // S[q] has been read (and the next K tile has landed)
+    bars.s_req = bars.s_free + 8 * ATTN_NQ;     // shared place for S: query tile q's softmax will be ready for its next S shortly
 
     // warp index through a shuffle: the compiler then knows that it is the same in all lanes of a warp
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
@@ -294,6 +312,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             mbar_init(bars.o_full + 8 * q, 1);
             mbar_init(bars.o_free + 8 * q, 128);
             mbar_init(bars.pv_done + 8 * q, 1);
+            mbar_init(bars.s_req + 8 * q, 128);
         }
         fence_mbar_init();
     }
@@ -398,7 +417,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             auto issue_qk = [&](int q, uint32_t st) {
                 const uint64_t a0 = qdesc0 + (uint64_t)((q * C::TILE_BYTES) >> 4);
                 const uint64_t b0 = kdesc0 + (uint64_t)((st * C::TILE_BYTES) >> 4);
-                const uint32_t d = tmem_base + C::S_COL + q * 128;
+                const uint32_t d = tmem_base + C::S_COL + q * C::S_STRIDE;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t koff = ((kk / 4) * C::HALF_BYTES + (kk % 4) * 32) >> 4;
@@ -431,6 +450,11 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     st = a % C::STAGES;
                     return wait_all(bars.kv_full + 8 * st, (a / C::STAGES) & 1u, abort_ptr, WAIT_LIMIT_CYCLES);
                 };
+                // One place for S (D = 128): its uses alternate strictly -- tile 0, tile 1, tile 0, ... -- because every
+                // Q K^T waits until the softmax has read the S before it, and a phase of the one s_free barrier is one
+                // such read.  Tile 0's warp therefore always waits for an odd phase and tile 1's for an even one (for the
+                // very first use that is the phase before the first, which counts as complete).
+                [[maybe_unused]] const uint32_t s_turn = mq ? 0u : 1u;
                 for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                     WorkItem it;
                     if (!decode_work<FUSED>(p, npairs, w, it)) continue;
@@ -438,6 +462,10 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     ok = wait_all(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_CYCLES) && wait_kv(0, st);
                     if (!ok) break;
                     q_phase ^= 1u;
+                    if constexpr (C::SHARED_S) {
+                        ok = wait_all(bars.s_free, s_turn, abort_ptr, WAIT_LIMIT_CYCLES);
+                        if (!ok) break;
+                    }
                     tc_fence_after();
                     issue_qk(mq, st);
                     if (leader) {
@@ -447,21 +475,46 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     }
                     for (int k = 0; k < it.tiles && ok; ++k) {
                         const bool more = (k + 1 < it.tiles);
-                        ok = wait_all(bars.s_free + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES);
-                        if (!ok) break;
-                        if (more) {
-                            ok = wait_kv(k_place(k + 1), st);
+                        if constexpr (C::SHARED_S) {
+                            // Q K_{k+1}^T first -- the softmax waits for it, and asks for it a little before it has
+                            // stored P_k, so that S_{k+1} lands about when it is ready to read it -- then P_k V_k, which
+                            // nothing waits for until the next P is to be stored
+                            ok = wait_all((C::S_REQ ? bars.s_req : bars.p_full) + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES);
                             if (!ok) break;
-                            tc_fence_after();
-                            issue_qk(mq, st);
-                            if (leader) {
-                                tc_commit(bars.s_full + 8 * mq);
-                                tc_commit(bars.kv_empty + 8 * st);
-                                if (k + 2 == it.tiles) tc_commit(bars.q_empty);   // that was the item's last Q K^T
+                            if (more) {
+                                ok = wait_kv(k_place(k + 1), st) && wait_all(bars.s_free, s_turn, abort_ptr, WAIT_LIMIT_CYCLES);
+                                if (!ok) break;
+                                tc_fence_after();
+                                issue_qk(mq, st);
+                                if (leader) {
+                                    tc_commit(bars.s_full + 8 * mq);
+                                    tc_commit(bars.kv_empty + 8 * st);
+                                    if (k + 2 == it.tiles) tc_commit(bars.q_empty);   // that was the item's last Q K^T
+                                }
                             }
+                            if constexpr (C::S_REQ) {
+                                ok = wait_all(bars.p_full + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES);   // P_k is stored
+                                if (!ok) break;
+                            }
+                            ok = wait_kv(v_place(k, it.tiles), st);
+                            if (!ok) break;
+                        } else {
+                            ok = wait_all(bars.s_free + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES);
+                            if (!ok) break;
+                            if (more) {
+                                ok = wait_kv(k_place(k + 1), st);
+                                if (!ok) break;
+                                tc_fence_after();
+                                issue_qk(mq, st);
+                                if (leader) {
+                                    tc_commit(bars.s_full + 8 * mq);
+                                    tc_commit(bars.kv_empty + 8 * st);
+                                    if (k + 2 == it.tiles) tc_commit(bars.q_empty);   // that was the item's last Q K^T
+                                }
+                            }
+                            ok = wait_all(bars.p_full + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES) && wait_kv(v_place(k, it.tiles), st);
+                            if (!ok) break;
                         }
-                        ok = wait_all(bars.p_full + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES) && wait_kv(v_place(k, it.tiles), st);
-                        if (!ok) break;
                         if (k == 0) {  // first PV of the item: the previous item's epilogue must have drained O[mq]
                             ok = wait_all(bars.o_free + 8 * mq, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
                             if (!ok) break;
@@ -595,7 +648,8 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const int q = warp / 4;                       // query tile handled by this warpgroup
         const int row_in_tile = (warp % 4) * 32 + lane;
         const uint32_t lane_addr = ((uint32_t)((warp % 4) * 32)) << 16;
-        const uint32_t s_tmem = tmem_base + lane_addr + C::S_COL + q * 128;
+        const uint32_t s_tmem = tmem_base + lane_addr + C::S_COL + q * C::S_STRIDE;
+        const uint32_t s_free_bar = bars.s_free + (C::SHARED_S ? 0 : 8 * q);   // one place for S: one barrier
         const uint32_t p_tmem = tmem_base + lane_addr + C::P_COL + q * C::P_STRIDE;   // D = 128: the same columns as S
         const uint32_t o_tmem = tmem_base + lane_addr + C::O_COL + q * D;
         uint32_t s_phase = 0, o_phase = 0, pv_phase = 0;
@@ -651,10 +705,11 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 tmem_ld_x32(s_tmem + 64, s[2]);
                 tmem_ld_x32(s_tmem + 96, s[3]);
                 tmem_wait_ld();
+                [[maybe_unused]] bool s_asked = false;   // (one request per tile, also when P is computed twice)
                 bool p_place_free = !C::PREFETCH || t == 0 || pv_waited;   // D = 64: P's columns may still be read by the previous tile's PV
                 if constexpr (C::PREFETCH) {
                     tc_fence_before();
-                    mbar_arrive(bars.s_free + 8 * q);   // S_t has been read: Q K_{t+1}^T may overwrite it
+                    mbar_arrive(s_free_bar);   // S_t has been read: the next Q K^T may overwrite it
                 }
                 if (valid < ATTN_TILE) {
 #pragma unroll
@@ -694,6 +749,12 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                                                                             : make_float2(ex2_approx(x.x), ex2_approx(x.y));
                             rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
                             pk[(c >> 1) & 31] = pack_half2<FP16>(pp.x, pp.y);
+                            if constexpr (C::S_REQ > 0) {
+                                if (c + 2 == C::S_REQ * 32 && !s_asked) {   // this many keys are done: ask for the next tile's S
+                                    mbar_arrive(bars.s_req + 8 * q);
+                                    s_asked = true;
+                                }
+                            }
                         }
                         if constexpr (C::PREFETCH) {
                             if (!p_place_free) {   // PV of tile t-1 is done with P's columns
