@@ -738,9 +738,15 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 auto exp_pass = [&](float m_ref) -> float {
                     const float2 nm2 = make_float2(-m_ref, -m_ref);
                     float2 rs4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                    // 64 keys as packed 16-bit pairs in the inputs' type (even key in the low half), twice.  With P's own
+                    // columns the store has to wait until P_{t-1} V_{t-1} has read them: at D = 64 the first half goes out
+                    // as soon as it is complete (by then the wait is over); with the shared place for S (D = 128), where
+                    // P V is issued behind the next Q K^T, both halves go out after the last exponential.
+                    constexpr bool LATE_STORE = C::SHARED_S;
+                    uint32_t pk2[2][32];
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
-                        uint32_t pk[32];  // 64 keys as packed 16-bit pairs in the inputs' type (even key in the low half)
+                        uint32_t (&pk)[32] = pk2[half];
 #pragma unroll
                         for (int c = half * 64; c < half * 64 + 64; c += 2) {
                             const float s0 = __uint_as_float(s[c >> 5][c & 31]), s1 = __uint_as_float(s[(c + 1) >> 5][(c + 1) & 31]);
@@ -756,6 +762,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                                 }
                             }
                         }
+                        if (LATE_STORE && half == 0) continue;
                         if constexpr (C::PREFETCH) {
                             if (!p_place_free) {   // PV of tile t-1 is done with P's columns
                                 ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_CYCLES));
@@ -764,6 +771,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                                 tc_fence_after();
                             }
                         }
+                        if (LATE_STORE) tmem_st_x32(p_tmem, pk2[0]);
                         tmem_st_x32(p_tmem + 32 * half, pk);
                     }
                     const float2 r = __fadd2_rn(__fadd2_rn(rs4[0], rs4[1]), __fadd2_rn(rs4[2], rs4[3]));
