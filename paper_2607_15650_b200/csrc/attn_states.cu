@@ -12,20 +12,21 @@
 //
 // Per CTA (12 warps; the producer warpgroup gives registers to the softmax warpgroups):
 //   warps 0-3 / 4-7  softmax warpgroups for query tile 0 / 1 (128 rows each, one row per thread)
-//   warp 8           TMA producer: Q tiles once per work item, K and V tiles through a ring
-//   warp 9           MMA issuer: the whole warp runs the (warp-uniform) control flow and address arithmetic, one
-//                    lane issues tcgen05.mma / tcgen05.commit -- measured 4 % faster than a single-lane branch
-//   warp 10          D = 128: K/V watcher -- adds its arrival to p_full[0] once V_t and K_{t+1} have landed, and hands
-//                    the stages and the place of Q back to the producer once the MMAs that read them are done.
-//                    D = 64: the second MMA warp (one per query tile; each waits for its K/V tiles itself and hands
-//                    them back with commits of its own)
+//   warp 8           TMA producer: Q tiles once per work item, K and V tiles through a ring, in the order the MMAs
+//                    consume them (K_0, K_1, V_0, K_2, V_1, ...)
+//   warps 9, 10      MMA issuers of query tile 0 / 1: the whole warp runs the (warp-uniform) control flow and address
+//                    arithmetic, one lane issues tcgen05.mma / tcgen05.commit.  Each waits for its own barriers and
+//                    for the K/V tiles itself, and hands the stages (and Q's place) back with commits of its own
 //   warp 11          idle (completes the producer warpgroup for the register hand-over)
-// TMEM (512 columns): S0 | S1 | O0 | O1.  S_t = Q K_t^T (fp32) lands in S; the softmax warpgroup
-// reads its row, writes P = exp2(s*scale*log2e - m) back over S as packed bf16 (fp16 for fp16 inputs),
-// and the PV MMA takes P from TMEM as its A operand and V from shared memory (MN-major) as B,
-// accumulating in O.  While one query tile is in softmax the tensor core works on the other
-// (ping-pong).  With D = 64 there is room for S0 | S1 | P0 | P1 | O0 | O1: P has columns of its own and
-// the next tile's Q K^T is issued as soon as the softmax has read S (see Cfg::PREFETCH).
+// TMEM (512 columns).  S_t = Q K_t^T (fp32) lands in S; the softmax thread reads its row, writes P =
+// exp2(s*scale*log2e - m) as packed bf16 (fp16 for fp16 inputs) into P's own columns, and the PV MMA takes P from
+// TMEM as its A operand and V from shared memory (MN-major) as B, accumulating in O.  P_t V_t therefore never
+// stands between a softmax and its next S:
+//   D = 64   S0 | S1 | P0 | P1 | O0 | O1.  Q K_{t+1}^T is issued as soon as the softmax has read S_t.
+//   D = 128  S | P0 | P1 | O0 | O1: the columns leave room for ONE place for S, which the two query tiles use in
+//            turn.  A softmax thread takes its whole row into registers at once, so the place is busy only from a
+//            Q K^T to the read that follows it; a softmax asks for its next S half-way through a tile (s_req), and the
+//            MMA warp issues Q K_{t+1}^T ahead of P_t V_t.
 // P is computed against the reference maximum m of the earlier tiles, never against the tile's own: stale
 // references cancel exactly in OUT = O / l and LSE = m + log l.  bf16 inputs: when a row's running sum l reaches
 // LSUM_TRIGGER, m moves up by floor(log2 l) binades and O, l are scaled by that power of two (exact).  fp16
@@ -48,7 +49,7 @@ namespace {
 constexpr int NUM_SOFTMAX_THREADS = ATTN_NQ * 128;
 constexpr int TMA_WARP = NUM_SOFTMAX_THREADS / 32;
 constexpr int MMA_WARP = TMA_WARP + 1;
-constexpr int WATCH_WARP = TMA_WARP + 2;   // vouches for K/V arrival on behalf of the MMA thread
+constexpr int MMA_WARP_1 = TMA_WARP + 2;   // the MMA issuer of query tile 1 (MMA_WARP: query tile 0)
 constexpr int ATTN_THREADS = NUM_SOFTMAX_THREADS + 128;  // producer warpgroup: TMA, MMA and two idle warps
 // Per-thread register budgets after the role split.  setmaxnreg.inc can only take registers that a
 // setmaxnreg.dec of the same CTA has released (registers the launch left unallocated do not count);
@@ -71,10 +72,7 @@ constexpr float RESCALE_THRESHOLD = 1.0f;  // log2 units: in the slow path the r
 #define DT_POLY_PER_8_D64 1
 #endif
 #ifndef DT_POLY_PER_8_D128
-#define DT_POLY_PER_8_D128 1
-#endif
-#ifndef DT_D128_SHARED_S
-#define DT_D128_SHARED_S 1
+#define DT_POLY_PER_8_D128 0
 #endif
 // Shared place for S: after how many of a tile's four 32-key pieces the softmax asks for the next tile's S (0: only
 // when P is stored).
@@ -94,23 +92,21 @@ struct Cfg {
     static constexpr int OUT_BYTES = ATTN_NQ * OUT_STAGE_BYTES;
     static constexpr int NBARS = 2 + 2 * STAGES + 7 * ATTN_NQ;
     static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + Q_BYTES + KV_BYTES + OUT_BYTES + NBARS * 8 + 64;
-    // TMEM columns.  D = 128 fills all 512 (S0 | S1 | O0 | O1) and P has to live over S.  D = 64 leaves 128 columns:
-    // there P gets its own place (S0 | S1 | P0 | P1 | O0 | O1), so S may be overwritten as soon as the softmax has
-    // read it and the next tile's Q K^T runs while this tile's exponentials are being taken.
-    // D = 128 with DT_D128_SHARED_S: S | P0 | P1 | O0 | O1 -- the two query tiles share ONE place for S.  A softmax
-    // thread takes its whole row of S into registers as soon as it arrives, so the place is free again a few dozen
-    // cycles after every Q K^T, and giving the second tile's 128 columns to P0 | P1 takes P_t V_t out of the way of
-    // Q K_{t+1}^T: the S -> P -> S chain of a query tile loses P V's 512 cycles.
-    static constexpr bool SHARED_S = (D == 128) && (DT_D128_SHARED_S != 0);
-    static constexpr bool PREFETCH = (D == 64) || SHARED_S;   // P has columns of its own; one MMA warp per query tile
+    // TMEM columns.  P has columns of its own, so that P_t V_t never stands between a softmax and its next S.
+    // D = 64: S0 | S1 | P0 | P1 | O0 | O1 -- S may be overwritten as soon as the softmax has read it, and the next tile's
+    // Q K^T runs while this tile's exponentials are taken.  D = 128: S | P0 | P1 | O0 | O1 -- 512 columns leave room for
+    // ONE place for S, which the two query tiles share: a softmax thread takes its whole row of S into registers as soon
+    // as it arrives, so the place is free again a few dozen cycles after every Q K^T.
+    static constexpr bool SHARED_S = (D == 128);
+    // Shared place for S: after how many of a tile's four 32-key pieces the softmax asks for the next tile's S.
     static constexpr int S_REQ = SHARED_S ? DT_S_REQ_PIECE : 0;
     static constexpr int POLY_PER_8 = (D == 64) ? DT_POLY_PER_8_D64 : DT_POLY_PER_8_D128;
     static constexpr int S_COL = 0;                                              // S tile q: S_COL + q*S_STRIDE
     static constexpr int S_STRIDE = SHARED_S ? 0 : 128;
     static constexpr int S_TILES = SHARED_S ? 1 : ATTN_NQ;
-    static constexpr int P_COL = PREFETCH ? S_TILES * 128 : 0;                   // P tile q: P_COL + q*P_STRIDE
-    static constexpr int P_STRIDE = PREFETCH ? 64 : 128;
-    static constexpr int O_COL = PREFETCH ? S_TILES * 128 + ATTN_NQ * 64 : ATTN_NQ * 128;   // O tile q: O_COL + q*D
+    static constexpr int P_COL = S_TILES * 128;                                  // P tile q: P_COL + q*P_STRIDE
+    static constexpr int P_STRIDE = 64;
+    static constexpr int O_COL = S_TILES * 128 + ATTN_NQ * 64;                   // O tile q: O_COL + q*D
     static_assert(O_COL + ATTN_NQ * D <= 512, "beyond the tensor memory of an SM");
 };
 
@@ -120,7 +116,7 @@ struct Bars {
     uint32_t s_full, p_full, o_full, o_free, pv_done, s_free, s_req;  // + 8*q
 };
 
-// D = 64 (Cfg::PREFETCH): place of an item's K/V tiles in the order they are loaded and consumed --
+// Place of an item's K/V tiles in the order they are loaded and consumed --
 // K_0, K_1, V_0, K_2, V_1, ..., K_{n-1}, V_{n-2}, V_{n-1}: Q K_{t+1}^T is issued as soon as S_t has been read,
 // before P_t V_t.
 __device__ __forceinline__ uint32_t k_place(int t) { return t == 0 ? 0u : (uint32_t)(2 * t - 1); }
@@ -299,16 +295,15 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         abort_flag = 0;
         mbar_init(bars.q_full, 1);
         // D = 64: each of the two MMA warps hands Q's place and the K/V stages back with a commit of its own
-        mbar_init(bars.q_empty, C::PREFETCH ? 2 : 1);
+        mbar_init(bars.q_empty, 2);
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(bars.kv_full + 8 * s, 1);
-            mbar_init(bars.kv_empty + 8 * s, C::PREFETCH ? 2 : 1);
+            mbar_init(bars.kv_empty + 8 * s, 2);
         }
         for (int q = 0; q < ATTN_NQ; ++q) {
             mbar_init(bars.s_full + 8 * q, 1);
-            // D = 128: P ready (128 threads), tile 0: + the K/V watcher.  D = 64: P stored (128 threads)
-            mbar_init(bars.p_full + 8 * q, C::PREFETCH ? 128 : 128 + (q == 0 ? 1 : 0));
-            mbar_init(bars.s_free + 8 * q, 128);   // D = 64: S read (128 threads)
+            mbar_init(bars.p_full + 8 * q, 128);   // P stored (the tile's 128 softmax threads)
+            mbar_init(bars.s_free + 8 * q, 128);   // S read (D = 128: only [0] is used, by both tiles in turn)
             mbar_init(bars.o_full + 8 * q, 1);
             mbar_init(bars.o_free + 8 * q, 128);
             mbar_init(bars.pv_done + 8 * q, 1);
@@ -352,37 +347,20 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         tma_load_4d(q_smem + q * C::TILE_BYTES + hf * C::HALF_BYTES, &tmap_q, bars.q_full, hf * 64, it.h,
                                     it.qrow[q], it.b);
                 q_phase ^= 1u;
-                if constexpr (C::PREFETCH) {
-                    for (int n = 0; n < 2 * it.tiles && ok; ++n) {
-                        // place n of the item's load order: K_0 | K_{(n+1)/2} for odd n | V_{(n-2)/2} for even n | V_{tiles-1} last
-                        const bool is_k = (n == 0) || ((n & 1) && n + 1 < 2 * it.tiles);
-                        const int t = is_k ? (n + 1) / 2 : (n + 1 == 2 * it.tiles ? it.tiles - 1 : (n - 2) / 2);
-                        const int key0 = it.template tile<FUSED>(t).x;
-                        const uint32_t st = ring.st, ph = ring.ph;
-                        ok = mbar_wait_bounded(bars.kv_empty + 8 * st, ph ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
-                        if (!ok) break;
-                        mbar_arrive_expect_tx(bars.kv_full + 8 * st, C::TILE_BYTES);
-#pragma unroll
-                        for (int hf = 0; hf < C::NHALF; ++hf)
-                            tma_load_4d(kv_smem + st * C::TILE_BYTES + hf * C::HALF_BYTES, is_k ? &tmap_k : &tmap_v,
-                                        bars.kv_full + 8 * st, hf * 64, it.h, key0, it.b);
-                        ring.advance();
-                    }
-                } else
-                for (int t = 0; t < it.tiles && ok; ++t) {
+                for (int n = 0; n < 2 * it.tiles && ok; ++n) {
+                    // place n of the item's load order: K_0 | K_{(n+1)/2} for odd n | V_{(n-2)/2} for even n | V_{tiles-1} last
+                    const bool is_k = (n == 0) || ((n & 1) && n + 1 < 2 * it.tiles);
+                    const int t = is_k ? (n + 1) / 2 : (n + 1 == 2 * it.tiles ? it.tiles - 1 : (n - 2) / 2);
                     const int key0 = it.template tile<FUSED>(t).x;
+                    const uint32_t st = ring.st, ph = ring.ph;
+                    ok = mbar_wait_bounded(bars.kv_empty + 8 * st, ph ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(bars.kv_full + 8 * st, C::TILE_BYTES);
 #pragma unroll
-                    for (int kv = 0; kv < 2; ++kv) {
-                        const uint32_t st = ring.st, ph = ring.ph;
-                        ok = mbar_wait_bounded(bars.kv_empty + 8 * st, ph ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
-                        if (!ok) break;
-                        mbar_arrive_expect_tx(bars.kv_full + 8 * st, C::TILE_BYTES);
-#pragma unroll
-                        for (int hf = 0; hf < C::NHALF; ++hf)
-                            tma_load_4d(kv_smem + st * C::TILE_BYTES + hf * C::HALF_BYTES, kv == 0 ? &tmap_k : &tmap_v,
-                                        bars.kv_full + 8 * st, hf * 64, it.h, key0, it.b);
-                        ring.advance();
-                    }
+                    for (int hf = 0; hf < C::NHALF; ++hf)
+                        tma_load_4d(kv_smem + st * C::TILE_BYTES + hf * C::HALF_BYTES, is_k ? &tmap_k : &tmap_v,
+                                    bars.kv_full + 8 * st, hf * 64, it.h, key0, it.b);
+                    ring.advance();
                 }
             }
             if (!ok) {
@@ -393,7 +371,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         }
-      } else if (warp == MMA_WARP || (C::PREFETCH && warp == WATCH_WARP)) {
+      } else if (warp == MMA_WARP || warp == MMA_WARP_1) {
         // ------------------------------------------------------------ MMA issuer
         {
             const bool leader = (lane == 0);
@@ -404,8 +382,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             };
             constexpr uint32_t IDESC_QK = make_idesc_bf16_f32(128, ATTN_TILE, false, FP16);
             constexpr uint32_t IDESC_PV = make_idesc_bf16_f32(128, D, true, FP16);
-            uint32_t q_phase = 0, p_phase = 0, of_phase = 0;
-            RingPos<C::STAGES> ring;
+            uint32_t q_phase = 0, of_phase = 0;
             bool ok = true;
 
             // Descriptors differ only in their 14-bit start-address field (units of 16 bytes), so each
@@ -433,16 +410,16 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     if (leader) mma_ts(d, a + kk * 8, b0 + (uint64_t)((kk * 2048) >> 4), IDESC_PV, (accumulate || kk > 0) ? 1u : 0u);
             };
 
-            if constexpr (C::PREFETCH) {
-                // D = 64: one MMA warp per query tile (this one: mq), so that the two tiles' chains of wait -> issue ->
-                // commit run side by side; the tensor pipe has room for both (an M = 128 MMA takes 64 cycles whatever
-                // its N, so a K/V tile costs 4 + 8 MMAs per query tile against 2048 cycles of exponentials per pair).
-                // Per K/V tile t: s_free[mq] -- the softmax has read S_t -- lets S_{t+1} = Q K_{t+1}^T overwrite S;
+            {
+                // One MMA warp per query tile (this one: mq), so that the two tiles' chains of wait -> issue -> commit run
+                // side by side: an MMA leaves the issuing thread only as the pipe takes it, and what a single issuing warp
+                // did between two groups (commit, poll, fence) was time the pipe ran dry.
+                // D = 64, per K/V tile t: s_free[mq] -- the softmax has read S_t -- lets S_{t+1} = Q K_{t+1}^T overwrite S;
                 // p_full[mq] -- P_t is stored -- lets O += P_t V_t go (commit pv_done: P's place is free again, or o_full
-                // after the last tile).  This warp waits for the K/V tiles itself and hands them (and Q's place) back with
-                // a commit of its own: a stage is free when both warps' commits have arrived, so neither query tile can
-                // run ahead of the other by more than the ring holds.  Place n of the run of K/V tiles lives in ring
-                // stage (n mod STAGES).
+                // after the last tile).  D = 128: see below.  This warp waits for the K/V tiles itself and hands them (and
+                // Q's place) back with a commit of its own: a stage is free when both warps' commits have arrived, so
+                // neither query tile can run ahead of the other by more than the ring holds.  Place n of the run of K/V
+                // tiles lives in ring stage (n mod STAGES).
                 const int mq = warp - MMA_WARP;
                 uint32_t abs0 = 0, t_phase = 0;   // tiles loaded before this item; parity of s_free / p_full (one phase per tile)
                 auto wait_kv = [&](uint32_t place, uint32_t &st) -> bool {
@@ -530,114 +507,9 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     of_phase ^= 1u;
                     abs0 += 2u * (uint32_t)it.tiles;
                 }
-            } else
-            for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
-                WorkItem it;
-                if (!decode_work<FUSED>(p, npairs, w, it)) continue;
-                ok = wait_all(bars.q_full, q_phase, abort_ptr, WAIT_LIMIT_CYCLES);
-                if (!ok) break;
-                q_phase ^= 1u;
-                // first K tile
-                {
-                    const uint32_t st = ring.st, ph = ring.ph;
-                    ok = wait_all(bars.kv_full + 8 * st, ph, abort_ptr, WAIT_LIMIT_CYCLES);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int q = 0; q < ATTN_NQ; ++q) {
-                        issue_qk(q, st);
-                        if (leader) tc_commit(bars.s_full + 8 * q);
-                    }
-                    ring.advance();
-                }
-                // Steady state.  This thread only waits on p_full: softmax warp 0 checks that V_t and
-                // K_{t+1} have landed before it arrives there, so one wait covers both (every wait here
-                // drains the queue of issued MMAs, and the tensor pipe idles until new ones arrive).
-                for (int t = 0; t < it.tiles && ok; ++t) {
-                    const uint32_t st_v = ring.st;
-                    ring.advance();
-                    const uint32_t st_k = ring.st;
-                    const bool more = (t + 1 < it.tiles);
-#pragma unroll
-                    for (int q = 0; q < ATTN_NQ; ++q) {
-                        ok = wait_all(bars.p_full + 8 * q, p_phase, abort_ptr, WAIT_LIMIT_CYCLES);
-                        if (!ok) break;
-                        if (t == 0) {  // the previous item's epilogue must have drained O[q]
-                            ok = wait_all(bars.o_free + 8 * q, of_phase ^ 1u, abort_ptr, WAIT_LIMIT_CYCLES);
-                            if (!ok) break;
-                        }
-                        tc_fence_after();
-                        issue_pv(q, st_v, t > 0);
-                        if (more) {
-                            issue_qk(q, st_k);
-                            if (leader) tc_commit(bars.s_full + 8 * q);
-                        } else {
-                            if (leader) tc_commit(bars.o_full + 8 * q);
-                        }
-                    }
-                    if (!ok) break;
-                    if (more) ring.advance();
-                    p_phase ^= 1u;
-                }
-                of_phase ^= 1u;
             }
             if (!ok) {
                 if (leader && !*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
-                *abort_ptr = 1;
-            }
-        }
-      } else if (warp == WATCH_WARP) {
-        // ------------------------------------------------------------ K/V watcher
-        // One more arrival on p_full[0] per tile, made once V_t and K_{t+1} are in shared memory: the
-        // MMA thread's single wait then covers P_t and both tiles without a poll of its own.
-        if (lane == 0) {
-            RingPos<C::STAGES> ring;
-            uint32_t p_phase = 0;
-            bool ok = true;
-            if constexpr (C::PREFETCH) {
-                // (D = 64 has no watcher: this warp is the second MMA warp there)
-            } else {
-            // It also hands the ring stages (and Q's place) back to the producer, so that the MMA thread issues no
-            // commit for that: the commit that closes the group of query tile 1 -- s_full[1], or o_full[1] after the
-            // last tile -- tells that every MMA issued before it is done, those of query tile 0 included.  After the
-            // item's first Q K^T that frees K_0; after the groups of tile t, V_t and K_{t+1}.  The release for tile
-            // t - 1 is made between the arrival for tile t and the wait for its phase to close: by then the commit
-            // is due, and the arrival is not held up by it.
-            uint32_t s1_phase = 0, o1_phase = 0;
-            RingPos<C::STAGES> rel;   // next stage to hand back (stages are freed in the order they were filled)
-            for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
-                WorkItem it;
-                if (!decode_work<FUSED>(p, npairs, w, it)) continue;
-                ring.advance();   // K_0 of the item: the MMA thread waits for that one itself
-                for (int t = 0; t < it.tiles && ok; ++t) {
-                    ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_CYCLES);
-                    ring.advance();
-                    if (ok && t + 1 < it.tiles) {
-                        ok = mbar_wait_bounded(bars.kv_full + 8 * ring.st, ring.ph, abort_ptr, WAIT_LIMIT_CYCLES);
-                        ring.advance();
-                    }
-                    if (!ok) break;
-                    mbar_arrive(bars.p_full);
-                    // S_1 of tile t is complete: the first Q K^T (t = 0) or the groups of tile t - 1 are done
-                    ok = mbar_wait_bounded(bars.s_full + 8, s1_phase, abort_ptr, WAIT_LIMIT_CYCLES);
-                    if (!ok) break;
-                    s1_phase ^= 1u;
-                    if (t > 0) { mbar_arrive(bars.kv_empty + 8 * rel.st); rel.advance(); }   // V_{t-1}
-                    mbar_arrive(bars.kv_empty + 8 * rel.st); rel.advance();                   // K_t
-                    if (t + 1 == it.tiles) mbar_arrive(bars.q_empty);                         // that was the item's last Q K^T
-                    // one arrival per phase: wait for the phase to close before the next one
-                    ok = mbar_wait_bounded(bars.p_full, p_phase, abort_ptr, WAIT_LIMIT_CYCLES);
-                    p_phase ^= 1u;
-                }
-                if (!ok) break;
-                ok = mbar_wait_bounded(bars.o_full + 8, o1_phase, abort_ptr, WAIT_LIMIT_CYCLES);   // the last PVs are done
-                if (!ok) break;
-                o1_phase ^= 1u;
-                mbar_arrive(bars.kv_empty + 8 * rel.st); rel.advance();                       // V of the last tile
-            }
-            }
-            if (!ok) {
-                if (!*abort_ptr) atomicOr(p.status, STATUS_WAIT_TIMEOUT);
                 *abort_ptr = 1;
             }
         }
@@ -655,10 +527,11 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         uint32_t s_phase = 0, o_phase = 0, pv_phase = 0;
         bool ok = true;
         StateT *o_state = static_cast<StateT *>(p.o_state);
-        if constexpr (C::PREFETCH) {
+        if constexpr (!C::SHARED_S) {
             // D = 64: the two warpgroups share the MUFU and are otherwise independent (an MMA warp each).  Started
             // half a tile apart, one takes its exponentials while the other waits for S, stores P or runs its epilogue
-            // (measured +1 %); nothing brings them back into step.
+            // (measured +1 %); nothing brings them back into step.  (D = 128: the turns at the one place for S space
+            // the two tiles out by themselves.)
             if (q == 1) {
                 const long long t0 = clock64();
                 while (clock64() - t0 < 1200) {}
@@ -687,13 +560,11 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         // moves up by e = floor(log2(l)) binades and O and l are multiplied by 2^-e, which is exact.  The test
                         // costs one compare on a value that is live anyway; made here, at the top of the next tile, the move
                         // is off the S -> P chain and the logits of a tile never have to be kept for a second pass.
-                        // (S_t complete tells that P_{t-1} V_{t-1} is -- D = 64: pv_done does.)
-                        if constexpr (C::PREFETCH) {
-                            ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_CYCLES));
-                            pv_phase ^= 1u;
-                            pv_waited = true;
-                            tc_fence_after();
-                        }
+                        // (O may only be touched once P_{t-1} V_{t-1} is complete: pv_done.)
+                        ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_CYCLES));
+                        pv_phase ^= 1u;
+                        pv_waited = true;
+                        tc_fence_after();
                         const int e = move_reference<D>(o_tmem, l_sum);
                         m_used += (float)e;
                         l_sum *= __int_as_float((127 - e) << 23);
@@ -706,11 +577,9 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 tmem_ld_x32(s_tmem + 96, s[3]);
                 tmem_wait_ld();
                 [[maybe_unused]] bool s_asked = false;   // (one request per tile, also when P is computed twice)
-                bool p_place_free = !C::PREFETCH || t == 0 || pv_waited;   // D = 64: P's columns may still be read by the previous tile's PV
-                if constexpr (C::PREFETCH) {
-                    tc_fence_before();
-                    mbar_arrive(s_free_bar);   // S_t has been read: the next Q K^T may overwrite it
-                }
+                bool p_place_free = t == 0 || pv_waited;   // P's columns may still be read by the previous tile's PV
+                tc_fence_before();
+                mbar_arrive(s_free_bar);   // S_t has been read: the next Q K^T may overwrite it
                 if (valid < ATTN_TILE) {
 #pragma unroll
                     for (int c = 0; c < 128; ++c)
@@ -763,13 +632,11 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             }
                         }
                         if (LATE_STORE && half == 0) continue;
-                        if constexpr (C::PREFETCH) {
-                            if (!p_place_free) {   // PV of tile t-1 is done with P's columns
-                                ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_CYCLES));
-                                pv_phase ^= 1u;
-                                p_place_free = true;
-                                tc_fence_after();
-                            }
+                        if (!p_place_free) {   // PV of tile t-1 is done with P's columns
+                            ok = __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars.pv_done + 8 * q, pv_phase, abort_ptr, WAIT_LIMIT_CYCLES));
+                            pv_phase ^= 1u;
+                            p_place_free = true;
+                            tc_fence_after();
                         }
                         if (LATE_STORE) tmem_st_x32(p_tmem, pk2[0]);
                         tmem_st_x32(p_tmem + 32 * half, pk);
