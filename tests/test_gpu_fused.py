@@ -25,6 +25,10 @@ def _fused_steps(run, P, S, masks, state_dtype=torch.float32):
     comp_o = torch.empty((wl.B, wl.H, wl.L, wl.D), dtype=state_dtype, device=dev)
     comp_l = torch.empty((wl.B, wl.H, wl.L), dtype=torch.float32, device=dev)
     out = torch.empty_like(run.out); lse = torch.empty_like(run.lse)
+    # The composed reuse state is a state of its own, stored in the cache's type: with a bf16 cache it is rounded to
+    # bf16 once more (relative 2^-9 of values up to about 4, on top of the rounding of the states it was composed from
+    # and of the bf16 output), so those checks allow twice the O bounds, as after an in-place group compose.
+    o_scale = 2.0 if state_dtype == torch.bfloat16 else 1.0
     t = 1
     for mask in masks:
         mask = np.ascontiguousarray(mask, dtype=np.uint8).reshape(P, S)
@@ -49,7 +53,7 @@ def _fused_steps(run, P, S, masks, state_dtype=torch.float32):
             ses.tc = saved_tc
             out_h, lse_h = out.float().cpu().numpy(), lse.cpu().numpy()
             for (b, h), rows in run.rows.items():
-                check_o(out_h[b, rows, h, :], outs[(b, h)], f"fused step {t} head {h}")
+                check_o(out_h[b, rows, h, :], outs[(b, h)], f"fused step {t} head {h}", scale=o_scale)
                 check_lse(lse_h[b, h, rows], lses[(b, h)], f"fused step {t} head {h}")
         assert (ctx.dt_get_tc() == tc_before).all() and torch.equal(ctx.lse_state, cache_before)
 

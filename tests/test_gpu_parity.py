@@ -20,8 +20,9 @@ def _built():
 
 
 def check_o(got, ref, what="", scale=1.0):
-    """scale > 1 only where a bf16 state cache has been composed in place: every composition rounds the state to
-    bf16 once more (relative 2^-9 of values up to about 4), on top of the rounding of the stored states."""
+    """scale > 1 only where states of a bf16 cache have been composed into a state that is stored again (in place by
+    dt_group_compose, or as the composed reuse state that dt_attn_fused reads): every such composition rounds the state
+    to bf16 once more (relative 2^-9 of values up to about 4), on top of the rounding of the stored states."""
     err = np.abs(np.asarray(got, dtype=np.float64) - ref)
     assert err.max() <= scale * O_MAX, f"{what}: O max abs err {err.max():.3e}"
     assert err.mean() <= scale * O_MEAN, f"{what}: O mean abs err {err.mean():.3e}"
