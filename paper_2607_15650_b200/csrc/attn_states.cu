@@ -452,6 +452,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     }
                     for (int k = 0; k < it.tiles && ok; ++k) {
                         const bool more = (k + 1 < it.tiles);
+                        [[maybe_unused]] uint32_t stv = 0; [[maybe_unused]] bool v_waited = false;
                         if constexpr (C::SHARED_S) {
                             // Q K_{k+1}^T first -- the softmax waits for it, and asks for it a little before it has
                             // stored P_k, so that S_{k+1} lands about when it is ready to read it -- then P_k V_k, which
@@ -459,7 +460,15 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                             ok = wait_all((C::S_REQ ? bars.s_req : bars.p_full) + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES);
                             if (!ok) break;
                             if (more) {
-                                ok = wait_kv(k_place(k + 1), st) && wait_all(bars.s_free, s_turn, abort_ptr, WAIT_LIMIT_CYCLES);
+                                {   // K_{k+1}, V_k (loaded right behind it) and the place for S behind one vote: every
+                                    // separate wait costs this warp a poll and a vote, and its loop is what paces the pipe
+                                    const uint32_t ak = abs0 + k_place(k + 1), av = abs0 + v_place(k, it.tiles);
+                                    st = ak % C::STAGES; stv = av % C::STAGES;
+                                    const bool r = mbar_wait_bounded(bars.kv_full + 8 * st, (ak / C::STAGES) & 1u, abort_ptr, WAIT_LIMIT_CYCLES) &&
+                                                   mbar_wait_bounded(bars.kv_full + 8 * stv, (av / C::STAGES) & 1u, abort_ptr, WAIT_LIMIT_CYCLES) &&
+                                                   mbar_wait_bounded(bars.s_free, s_turn, abort_ptr, WAIT_LIMIT_CYCLES);
+                                    ok = __all_sync(0xFFFFFFFFu, r) != 0; v_waited = true;
+                                }
                                 if (!ok) break;
                                 tc_fence_after();
                                 issue_qk(mq, st);
@@ -473,7 +482,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                                 ok = wait_all(bars.p_full + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES);   // P_k is stored
                                 if (!ok) break;
                             }
-                            ok = wait_kv(v_place(k, it.tiles), st);
+                            if (v_waited) st = stv; else ok = wait_kv(v_place(k, it.tiles), st);
                             if (!ok) break;
                         } else {
                             ok = wait_all(bars.s_free + 8 * mq, t_phase, abort_ptr, WAIT_LIMIT_CYCLES);
