@@ -66,8 +66,8 @@ constexpr float LSUM_TRIGGER = 16777216.0f;   // bf16 inputs: a running sum l at
 constexpr float RESCALE_THRESHOLD = 1.0f;  // log2 units: in the slow path the reference moves if the maximum grew by more
 // Key pairs (of every 8) whose exp2 runs as a cubic on the FMA pipe instead of the MUFU.  D = 64 is bound by the
 // exponentials (2048 MUFU cycles per 256 x 128 tile pair against 1536 of MMA issue), and one pair in eight measured
-// +2 % there (two in eight: no further gain); at D = 128 the softmax is a link of the S -> P -> S chain and the extra
-// dependent instructions cost what the MUFU time saves.
+// +2 % there (two in eight: no further gain).  At D = 128 one pair in eight saves 4 % of the cycles and costs 3 % of the
+// time at full size: the GPU runs at its power cap there, and an exponential takes less energy on the MUFU.
 #ifndef DT_POLY_PER_8_D64
 #define DT_POLY_PER_8_D64 1
 #endif
@@ -283,7 +283,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     bars.p_full = bars.s_full + 8 * ATTN_NQ;
     bars.o_full = bars.p_full + 8 * ATTN_NQ;
     bars.o_free = bars.o_full + 8 * ATTN_NQ;
-    bars.pv_done = bars.o_free + 8 * ATTN_NQ;   // D = 64 only: the PV MMAs that read P[q] have completed
+    bars.pv_done = bars.o_free + 8 * ATTN_NQ;   // the PV MMAs that read P[q] have completed
     bars.s_free = bars.pv_done + 8 * ATTN_NQ;   // S[q] has been read (and the next K tile has landed)
     bars.s_req = bars.s_free + 8 * ATTN_NQ;     // shared place for S: query tile q's softmax will be ready for its next S shortly
 
@@ -294,7 +294,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp == TMA_WARP && lane == 0) {
         abort_flag = 0;
         mbar_init(bars.q_full, 1);
-        // D = 64: each of the two MMA warps hands Q's place and the K/V stages back with a commit of its own
+        // each of the two MMA warps hands Q's place and the K/V stages back with a commit of its own
         mbar_init(bars.q_empty, 2);
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(bars.kv_full + 8 * s, 1);
@@ -531,7 +531,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const uint32_t lane_addr = ((uint32_t)((warp % 4) * 32)) << 16;
         const uint32_t s_tmem = tmem_base + lane_addr + C::S_COL + q * C::S_STRIDE;
         const uint32_t s_free_bar = bars.s_free + (C::SHARED_S ? 0 : 8 * q);   // one place for S: one barrier
-        const uint32_t p_tmem = tmem_base + lane_addr + C::P_COL + q * C::P_STRIDE;   // D = 128: the same columns as S
+        const uint32_t p_tmem = tmem_base + lane_addr + C::P_COL + q * C::P_STRIDE;
         const uint32_t o_tmem = tmem_base + lane_addr + C::O_COL + q * D;
         uint32_t s_phase = 0, o_phase = 0, pv_phase = 0;
         bool ok = true;
