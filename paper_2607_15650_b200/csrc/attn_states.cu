@@ -64,8 +64,8 @@ constexpr float ROWSUM_TRIGGER = 512.0f;   // fp16 inputs: a row sum of P at or 
 constexpr float LSUM_TRIGGER = 16777216.0f;   // bf16 inputs: a running sum l at or above 2^24 moves the row's reference
 constexpr float RESCALE_THRESHOLD = 1.0f;  // log2 units: in the slow path the reference moves if the maximum grew by more
 // Key pairs (of every 8) whose exp2 runs as a cubic on the FMA pipe instead of the MUFU.  D = 64 is bound by the
-// exponentials (2048 MUFU cycles per 256 x 128 tile pair against 1536 of MMA issue): two pairs in eight measured
-// +1 % over one and about +10 % over none there (three: -2 %, four: -15 %).  At D = 128 one pair in eight saves 4 %
+// exponentials (2048 MUFU cycles per 256 x 128 tile pair against 1536 of MMA issue): two pairs in eight, every
+// fourth pair, measured +2 % over one and about +10 % over none there (two adjacent pairs: +1 %; three: -8 %).  At D = 128 one pair in eight saves 4 %
 // of the cycles and costs 3 % of the time at full size: the GPU runs at its power cap there, and an exponential takes
 // less energy on the MUFU.
 #ifndef DT_POLY_PER_8_D64
@@ -588,8 +588,9 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         for (int c = half * 64; c < half * 64 + 64; c += 2) {
                             const float s0 = __uint_as_float(s[c >> 5][c & 31]), s1 = __uint_as_float(s[(c + 1) >> 5][(c + 1) & 31]);
                             const float2 x = __ffma2_rn(make_float2(s0, s1), sc2, nm2);
-                            const float2 pp = (((c >> 1) & 7) < C::POLY_PER_8) ? exp2_poly2(x)
-                                                                            : make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                            // POLY_PER_8 key pairs in eight take the polynomial, spread evenly (two in eight: every fourth)
+                            const bool poly = (((c >> 1) * C::POLY_PER_8) & 7) < C::POLY_PER_8;
+                            const float2 pp = poly ? exp2_poly2(x) : make_float2(ex2_approx(x.x), ex2_approx(x.y));
                             rs4[(c >> 1) & 3] = __fadd2_rn(rs4[(c >> 1) & 3], pp);
                             pk[(c >> 1) & 31] = pack_half2<FP16>(pp.x, pp.y);
                             if (c + 2 == C::S_REQ * 32 && !s_asked) {   // this many keys are done: ask for the next tile's S
