@@ -306,7 +306,7 @@ dt_status dt_plan_static(const float *lse_state_dev, const int32_t *part_offsets
 /* One whole step from HOST buffers: copies q, k, v (bf16 [B,L,H,D] contiguous) and the mask to the
  * device workspace, runs dt_attn_states and dt_state_merge, copies out (bf16 [B,L,H,D]) and lse
  * (fp32 [B,H,L], may be NULL) back and synchronises `stream`.  Heads are independent, so the step runs
- * in up to 8 head chunks: the kernels of one chunk (on `stream`) overlap the host-to-device copy of the next
+ * in head chunks (a few heads each): the kernels of one chunk (on `stream`) overlap the host-to-device copy of the next
  * and the device-to-host copy of the previous one, which run on two streams the context owns (ordered against
  * `stream` with events; the call returns with all three idle).  workspace_dev must hold
  * dt_step_host_workspace_bytes() bytes of device memory.  Host buffers should be pinned: pageable memory

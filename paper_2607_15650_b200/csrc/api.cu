@@ -569,6 +569,14 @@ dt_status dt_step_host_workspace_bytes(const dt_config *cfg, size_t *bytes) {
     return DT_OK;
 }
 
+#ifndef DT_CHUNK_DIV
+#define DT_CHUNK_DIV 16
+#endif
+#ifndef DT_CHUNK_MIN
+#define DT_CHUNK_MIN 2
+#endif
+constexpr int DT_MAX_HEAD_CHUNKS = 64;
+
 dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, const void *v_host,
                        const uint8_t *mask_host, int32_t step, void *out_host, float *lse_out_host,
                        void *workspace_dev, size_t workspace_bytes, void *stream) {
@@ -591,7 +599,23 @@ dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, cons
     cudaError_t e;
     // Heads are independent, so the step is cut into head chunks: chunk c + 1 is copied in (copy_in stream) and
     // chunk c - 1 copied out (copy_out stream) while chunk c is in the kernels (the caller's stream).
-    const int nchunks = std::min(c.H, 8);
+    // About H / DT_CHUNK_DIV heads per chunk while many remain, then smaller ones down to DT_CHUNK_MIN heads: the last
+    // chunk's kernels and its copy out overlap nothing, so it should be short, but a chunk of a single head makes for
+    // narrow strided copies and a thin launch.
+    int bounds[DT_MAX_HEAD_CHUNKS + 1];
+    int nchunks = 0;
+    {
+        const int base = std::max(DT_CHUNK_MIN, (c.H + DT_CHUNK_DIV - 1) / DT_CHUNK_DIV);
+        int h = 0;
+        bounds[0] = 0;
+        while (h < c.H) {
+            const int left = c.H - h;
+            int sz = std::min(base, std::max(DT_CHUNK_MIN, left / 2));
+            if (sz > left || nchunks + 1 == DT_MAX_HEAD_CHUNKS) sz = left;
+            h += sz;
+            bounds[++nchunks] = h;
+        }
+    }
     if (!ctx->copy_in) {
         bool ok = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking) == cudaSuccess;
@@ -612,7 +636,7 @@ dt_status dt_step_host(dt_ctx *ctx, const void *q_host, const void *k_host, cons
     const size_t pitch = (size_t)c.H * c.D * 2, rows2d = (size_t)c.B * c.L;
     dt_status s;
     for (int ch = 0; ch < nchunks; ++ch) {
-        const int h0 = (int)((long long)ch * c.H / nchunks), h1 = (int)((long long)(ch + 1) * c.H / nchunks), hc = h1 - h0;
+        const int h0 = bounds[ch], h1 = bounds[ch + 1], hc = h1 - h0;
         const size_t col = (size_t)h0 * c.D * 2, width = (size_t)hc * c.D * 2;
         const void *src[3] = {q_host, k_host, v_host};
         void *dst[3] = {qd, kd, vd};
