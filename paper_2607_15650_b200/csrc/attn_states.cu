@@ -125,11 +125,6 @@ struct RingPos {
     __device__ __forceinline__ void advance() {
         if (++st == STAGES) { st = 0; ph ^= 1u; }
     }
-    __device__ __forceinline__ RingPos next() const {
-        RingPos r = *this;
-        r.advance();
-        return r;
-    }
 };
 
 struct WorkItem {
