@@ -409,7 +409,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 // commits have arrived, so neither query tile can run ahead of the other by more than the ring holds.
                 // Place n of the run of K/V tiles lives in ring stage (n mod STAGES).
                 const int mq = warp - MMA_WARP;
-                uint32_t abs0 = 0, t_phase = 0;   // tiles loaded before this item; parity of s_free / p_full (one phase per tile)
+                uint32_t abs0 = 0, t_phase = 0;   // tiles loaded before this item; parity of s_req / p_full (one phase per tile)
                 auto wait_kv = [&](uint32_t place, uint32_t &st) -> bool {
                     const uint32_t a = abs0 + place;
                     st = a % C::STAGES;
@@ -419,7 +419,7 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 // Q K^T waits until the softmax has read the S before it, and a phase of the one s_free barrier is one
                 // such read.  Tile 0's warp therefore always waits for an odd phase and tile 1's for an even one (for the
                 // very first use that is the phase before the first, which counts as complete).
-                [[maybe_unused]] const uint32_t s_turn = mq ? 0u : 1u;
+                const uint32_t s_turn = mq ? 0u : 1u;
                 for (long long w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
                     WorkItem it;
                     if (!decode_work<FUSED>(p, npairs, w, it)) continue;
@@ -438,7 +438,8 @@ attn_states_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     }
                     for (int k = 0; k < it.tiles && ok; ++k) {
                         const bool more = (k + 1 < it.tiles);
-                        [[maybe_unused]] uint32_t stv = 0; [[maybe_unused]] bool v_waited = false;
+                        uint32_t stv = 0;
+                        bool v_waited = false;   // V_k was waited for together with K_{k+1}
                         // Q K_{k+1}^T first -- the softmax waits for it, and asks for it a little before it has
                         // stored P_k, so that S_{k+1} lands about when it is ready to read it -- then P_k V_k, which
                         // nothing waits for until the next P is to be stored
