@@ -98,6 +98,7 @@ struct Cfg {
     // take at the one place are what keeps their softmaxes half a tile apart, and measured 8 % faster than two places.)
     // After how many of a tile's four 32-key pieces the softmax asks for the next tile's S:
     static constexpr int S_REQ = DT_S_REQ_PIECE;
+    static_assert(S_REQ >= 1 && S_REQ <= 4, "the request for S comes after one to four of a tile's 32-key pieces");
     static constexpr int POLY_PER_8 = (D == 64) ? DT_POLY_PER_8_D64 : DT_POLY_PER_8_D128;
     static constexpr int S_COL = 0;
     static constexpr int P_COL = 128;                                            // P tile q: P_COL + q*P_STRIDE
